@@ -1,0 +1,250 @@
+/*
+ * jv_oracle.c -- float64 CPU oracle for the three JetViT token mixers.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+ * mixers compute; the parity tests, the smoke check and the CPU-baseline leg of
+ * the benchmark are its only callers.  It shares no code, header, table or
+ * helper with the CUDA library and the CUDA library never calls it.
+ *
+ * Everything is double precision, every loop is the definition written out:
+ * no tiling, no fusion, no reordering beyond the one the paper itself states
+ * (Eq. 2: phi(Q) (phi(K)^T V) instead of (phi(Q) phi(K)^T) V).
+ * OpenMP only spreads independent (batch, head) units over the host cores.
+ *
+ * Layout of q, k, v, o: [B*H][N][D] contiguous, D fastest; token t of an
+ * Hg x Wg grid is (y, x) = (t / Wg, t % Wg).
+ *
+ * Pins (tests/test_oracle_pins.py): brute-force N x N forms, closed forms,
+ * library routines (float64 SDPA, float64 depth-wise conv2d), hand-computed
+ * fixtures under tests/golden/.  No function here is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int jvo_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/*
+ * Full softmax attention, Eq. 1 with the row normalisation of softmax:
+ *   s_ij = (q_i . k_j) * scale,  m_i = max_j s_ij,  p_ij = exp(s_ij - m_i),
+ *   O_i  = sum_j p_ij v_j / sum_j p_ij.
+ * Non-causal.  Nq query rows attend Nk key rows (Nq == Nk for self-attention;
+ * Nq < Nk lets a test evaluate a sample of the query rows of a large problem,
+ * rows being independent of one another).
+ * q: [BH][Nq][D], k, v: [BH][Nk][D], o: [BH][Nq][D].
+ */
+void jvo_full_attn(const double* q, const double* k, const double* v, double* o,
+                   int64_t BH, int64_t Nq, int64_t Nk, int64_t D, double scale) {
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)Nk);
+#pragma omp for collapse(2) schedule(dynamic, 16)
+    for (int64_t g = 0; g < BH; ++g) {
+      for (int64_t i = 0; i < Nq; ++i) {
+        const double* qi = q + (g * Nq + i) * D;
+        const double* kg = k + g * Nk * D;
+        const double* vg = v + g * Nk * D;
+        double* oi = o + (g * Nq + i) * D;
+        double m = -INFINITY;
+        for (int64_t j = 0; j < Nk; ++j) {
+          double dot = 0.0;
+          for (int64_t e = 0; e < D; ++e) dot += qi[e] * kg[j * D + e];
+          s[j] = dot * scale;
+          if (s[j] > m) m = s[j];
+        }
+        double denom = 0.0;
+        for (int64_t e = 0; e < D; ++e) oi[e] = 0.0;
+        for (int64_t j = 0; j < Nk; ++j) {
+          double p = exp(s[j] - m);
+          denom += p;
+          for (int64_t e = 0; e < D; ++e) oi[e] += p * vg[j * D + e];
+        }
+        for (int64_t e = 0; e < D; ++e) oi[e] /= denom;
+      }
+    }
+    free(s);
+  }
+}
+
+/*
+ * Window attention (Sec. 3.2.2): the Hg x Wg token grid is cut into
+ * non-overlapping wh x ww windows anchored at the grid origin; softmax
+ * attention (Eq. 1) runs independently inside each window.  When the grid is
+ * not a multiple of the window, the right / bottom windows are simply smaller:
+ * they hold the tokens that exist.  Token (y, x) belongs to window
+ * (y / wh, x / ww); it attends exactly the tokens with the same window id.
+ */
+void jvo_window_attn(const double* q, const double* k, const double* v, double* o,
+                     int64_t BH, int64_t Hg, int64_t Wg, int64_t D,
+                     int64_t wh, int64_t ww, double scale) {
+  const int64_t N = Hg * Wg;
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)(wh * ww));
+#pragma omp for collapse(2) schedule(dynamic, 16)
+    for (int64_t g = 0; g < BH; ++g) {
+      for (int64_t i = 0; i < N; ++i) {
+        const int64_t y = i / Wg, x = i % Wg;
+        const int64_t y0 = (y / wh) * wh, x0 = (x / ww) * ww;
+        const int64_t y1 = (y0 + wh < Hg) ? y0 + wh : Hg;
+        const int64_t x1 = (x0 + ww < Wg) ? x0 + ww : Wg;
+        const double* qi = q + (g * N + i) * D;
+        double* oi = o + (g * N + i) * D;
+        double m = -INFINITY;
+        int64_t c = 0;
+        for (int64_t yy = y0; yy < y1; ++yy)
+          for (int64_t xx = x0; xx < x1; ++xx) {
+            const double* kj = k + (g * N + yy * Wg + xx) * D;
+            double dot = 0.0;
+            for (int64_t e = 0; e < D; ++e) dot += qi[e] * kj[e];
+            s[c] = dot * scale;
+            if (s[c] > m) m = s[c];
+            ++c;
+          }
+        double denom = 0.0;
+        for (int64_t e = 0; e < D; ++e) oi[e] = 0.0;
+        c = 0;
+        for (int64_t yy = y0; yy < y1; ++yy)
+          for (int64_t xx = x0; xx < x1; ++xx) {
+            const double* vj = v + (g * N + yy * Wg + xx) * D;
+            double p = exp(s[c] - m);
+            denom += p;
+            for (int64_t e = 0; e < D; ++e) oi[e] += p * vj[e];
+            ++c;
+          }
+        for (int64_t e = 0; e < D; ++e) oi[e] /= denom;
+      }
+    }
+    free(s);
+  }
+}
+
+static double silu(double x) { return x / (1.0 + exp(-x)); }
+
+/*
+ * Kernel generator of the squeeze dynamic convolution (Sec. 3.2.1): average
+ * pooling of V over the grid, then a two-layer MLP with SiLU.
+ *   s[b][c] = (1/N) sum_j V[b][c][j],  hid = SiLU(W1 s + b1),  w[b] = W2 hid + b2.
+ * v: [B*H][N][D]; w: [B][C*k*k] with C = H*D, channel c = h*D + e.
+ */
+void jvo_dwc_generate(const double* v, double* w, int64_t B, int64_t H, int64_t N, int64_t D,
+                      int64_t dwc_k, int64_t R, const double* W1, const double* b1,
+                      const double* W2, const double* b2) {
+  const int64_t C = H * D, kk = dwc_k * dwc_k;
+  for (int64_t b = 0; b < B; ++b) {
+    double* s = (double*)calloc((size_t)C, sizeof(double));
+    double* hid = (double*)calloc((size_t)R, sizeof(double));
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t e = 0; e < D; ++e) {
+        const double* vg = v + (b * H + h) * N * D;
+        double acc = 0.0;
+        for (int64_t j = 0; j < N; ++j) acc += vg[j * D + e];
+        s[h * D + e] = acc / (double)N;
+      }
+    for (int64_t r = 0; r < R; ++r) {
+      double acc = b1 ? b1[r] : 0.0;
+      for (int64_t c = 0; c < C; ++c) acc += W1[r * C + c] * s[c];
+      hid[r] = silu(acc);
+    }
+    for (int64_t t = 0; t < C * kk; ++t) {
+      double acc = b2 ? b2[t] : 0.0;
+      for (int64_t r = 0; r < R; ++r) acc += W2[t * R + r] * hid[r];
+      w[b * C * kk + t] = acc;
+    }
+    free(s);
+    free(hid);
+  }
+}
+
+/*
+ * JetViT linear-attention block (Sec. 3.2.1, Eqs. 2 and 4).
+ *
+ * Core, per (batch, head), phi = ReLU:
+ *   KV = sum_j phi(k_j)^T v_j   (D x D),     z = sum_j phi(k_j)   (D),
+ *   LA_i = (phi(q_i) KV) / (phi(q_i) . z + eps).
+ * The paper's Eq. 4 prints no denominator; the row normalisation with eps in
+ * the denominator only is the reading this build was given.
+ *
+ * Squeeze dynamic depth-wise convolution on V (used when dwc_k > 0): with
+ * C = H*D value channels, channel c = h*D + e,
+ *   s[b][c]  = mean over the N grid tokens of V[b][c]          (average pooling)
+ *   hid      = SiLU(W1 s + b1)                                 (W1: [R][C])
+ *   w[b]     = W2 hid + b2, viewed as [C][k][k]                (W2: [C*k*k][R])
+ *   DW_i[c]  = sum_{dy,dx in [0,k)} w[b][c][dy][dx] * V[b][c][(y+dy-p, x+dx-p)]
+ *              with p = (k-1)/2 and taps outside the grid contributing zero,
+ *   O_i = LA_i + DW_i                                          (Eq. 4)
+ * b1 / b2 may be NULL (no bias).  One kernel set per batch sample, shared by
+ * all of its tokens.
+ */
+void jvo_linear_attn(const double* q, const double* k, const double* v, double* o,
+                     int64_t B, int64_t H, int64_t Hg, int64_t Wg, int64_t D, double eps,
+                     int64_t dwc_k, int64_t R, const double* W1, const double* b1,
+                     const double* W2, const double* b2) {
+  const int64_t N = Hg * Wg, C = H * D;
+
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t g = 0; g < B * H; ++g) {
+    const double* qg = q + g * N * D;
+    const double* kg = k + g * N * D;
+    const double* vg = v + g * N * D;
+    double* og = o + g * N * D;
+    double* KV = (double*)calloc((size_t)(D * D), sizeof(double));
+    double* z = (double*)calloc((size_t)D, sizeof(double));
+    for (int64_t j = 0; j < N; ++j)
+      for (int64_t a = 0; a < D; ++a) {
+        double pk = kg[j * D + a] > 0.0 ? kg[j * D + a] : 0.0;
+        z[a] += pk;
+        for (int64_t e = 0; e < D; ++e) KV[a * D + e] += pk * vg[j * D + e];
+      }
+    for (int64_t i = 0; i < N; ++i) {
+      double denom = eps;
+      for (int64_t e = 0; e < D; ++e) og[i * D + e] = 0.0;
+      for (int64_t a = 0; a < D; ++a) {
+        double pq = qg[i * D + a] > 0.0 ? qg[i * D + a] : 0.0;
+        denom += pq * z[a];
+        for (int64_t e = 0; e < D; ++e) og[i * D + e] += pq * KV[a * D + e];
+      }
+      for (int64_t e = 0; e < D; ++e) og[i * D + e] /= denom;
+    }
+    free(KV);
+    free(z);
+  }
+
+  if (dwc_k <= 0) return;
+
+  const int64_t kk = dwc_k * dwc_k, p = (dwc_k - 1) / 2;
+  double* wall = (double*)calloc((size_t)(B * C * kk), sizeof(double));
+  jvo_dwc_generate(v, wall, B, H, N, D, dwc_k, R, W1, b1, W2, b2);
+  for (int64_t b = 0; b < B; ++b) {
+    const double* w = wall + b * C * kk;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t y = 0; y < Hg; ++y) {
+        const double* vg = v + (b * H + h) * N * D;
+        double* og = o + (b * H + h) * N * D;
+        for (int64_t x = 0; x < Wg; ++x)
+          for (int64_t e = 0; e < D; ++e) {
+            const double* wc = w + (h * D + e) * kk;
+            double acc = 0.0;
+            for (int64_t dy = 0; dy < dwc_k; ++dy)
+              for (int64_t dx = 0; dx < dwc_k; ++dx) {
+                int64_t yy = y + dy - p, xx = x + dx - p;
+                if (yy < 0 || yy >= Hg || xx < 0 || xx >= Wg) continue;
+                acc += wc[dy * dwc_k + dx] * vg[(yy * Wg + xx) * D + e];
+              }
+            og[(y * Wg + x) * D + e] += acc;
+          }
+      }
+  }
+  free(wall);
+}

@@ -1,0 +1,147 @@
+"""ctypes front end of the float64 CPU oracle (``jv_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+CPU-baseline / reference legs of the benchmark.  Nothing here touches the CUDA
+library, and the CUDA binding never imports this module.
+
+Every function takes array-likes, converts them exactly to float64 and returns
+a float64 ``numpy`` array.  Shapes follow the mixers' ``[B, H, N, D]`` layout.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "jv_oracle.c")
+_SO = os.path.join(_HERE, "libjv_oracle.so")
+_lib = None
+
+_c_dp = ctypes.POINTER(ctypes.c_double)
+_i64 = ctypes.c_int64
+
+
+def build(force: bool = False) -> str:
+    """Compile ``jv_oracle.c`` with gcc (no fast-math: fp64 in source order)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".tmp{os.getpid()}"
+        subprocess.check_call(
+            ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.jvo_num_threads.restype = ctypes.c_int
+        lib.jvo_full_attn.argtypes = [_c_dp] * 4 + [_i64] * 4 + [ctypes.c_double]
+        lib.jvo_window_attn.argtypes = [_c_dp] * 4 + [_i64] * 6 + [ctypes.c_double]
+        lib.jvo_dwc_generate.argtypes = [_c_dp] * 2 + [_i64] * 6 + [_c_dp] * 4
+        lib.jvo_linear_attn.argtypes = ([_c_dp] * 4 + [_i64] * 5 + [ctypes.c_double]
+                                        + [_i64] * 2 + [_c_dp] * 4)
+        for f in (lib.jvo_full_attn, lib.jvo_window_attn, lib.jvo_dwc_generate,
+                  lib.jvo_linear_attn):
+            f.restype = None
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the oracle's OpenMP loops use on this host."""
+    return int(_load().jvo_num_threads())
+
+
+def _f64(a) -> np.ndarray:
+    if hasattr(a, "detach"):  # torch tensor (bf16 has no numpy dtype: widen first)
+        a = a.detach().cpu().double().numpy()
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(_c_dp)
+
+
+def full_attn(q, k, v, scale=None) -> np.ndarray:
+    """Eq. 1.  q: [B,H,Nq,D]; k, v: [B,H,Nk,D] -> [B,H,Nq,D]."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, Nq, D = q.shape
+    Nk = k.shape[2]
+    assert k.shape == (B, H, Nk, D) and v.shape == (B, H, Nk, D)
+    if scale is None or scale <= 0:
+        scale = 1.0 / np.sqrt(D)
+    o = np.empty_like(q)
+    _load().jvo_full_attn(_p(q), _p(k), _p(v), _p(o), B * H, Nq, Nk, D, float(scale))
+    return o
+
+
+def window_attn(q, k, v, Hg, Wg, win_h, win_w, scale=None) -> np.ndarray:
+    """Sec. 3.2.2 window attention.  q, k, v: [B,H,Hg*Wg,D]."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, N, D = q.shape
+    assert N == Hg * Wg and k.shape == q.shape and v.shape == q.shape
+    if scale is None or scale <= 0:
+        scale = 1.0 / np.sqrt(D)
+    o = np.empty_like(q)
+    _load().jvo_window_attn(_p(q), _p(k), _p(v), _p(o), B * H, Hg, Wg, D,
+                            win_h, win_w, float(scale))
+    return o
+
+
+def dwc_generate(v, dwc) -> np.ndarray:
+    """Dynamic depth-wise kernels [B, C, k, k] from V [B,H,N,D] (Sec. 3.2.1)."""
+    v = _f64(v)
+    B, H, N, D = v.shape
+    kk, R = int(dwc["k"]), int(dwc["R"])
+    W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
+    b1 = None if dwc.get("b1") is None else _f64(dwc["b1"])
+    b2 = None if dwc.get("b2") is None else _f64(dwc["b2"])
+    C = H * D
+    assert W1.shape == (R, C) and W2.shape == (C * kk * kk, R)
+    w = np.empty((B, C, kk, kk), dtype=np.float64)
+    _load().jvo_dwc_generate(_p(v), _p(w), B, H, N, D, kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+    return w
+
+
+def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None) -> np.ndarray:
+    """JetViT linear-attention block (Eqs. 2, 4).  ``dwc``: None or a dict with
+    keys k, R, W1 [R,C], b1 [R] or None, W2 [C*k*k,R], b2 [C*k*k] or None."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, N, D = q.shape
+    assert N == Hg * Wg and k.shape == q.shape and v.shape == q.shape
+    o = np.empty_like(q)
+    if dwc is None:
+        _load().jvo_linear_attn(_p(q), _p(k), _p(v), _p(o), B, H, Hg, Wg, D, float(eps),
+                                0, 0, None, None, None, None)
+        return o
+    kk, R = int(dwc["k"]), int(dwc["R"])
+    W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
+    b1 = None if dwc.get("b1") is None else _f64(dwc["b1"])
+    b2 = None if dwc.get("b2") is None else _f64(dwc["b2"])
+    C = H * D
+    assert kk % 2 == 1 and W1.shape == (R, C) and W2.shape == (C * kk * kk, R)
+    _load().jvo_linear_attn(_p(q), _p(k), _p(v), _p(o), B, H, Hg, Wg, D, float(eps),
+                            kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+    return o
+
+
+def hybrid_mixers(schedule, q, k, v, Hg, Wg, win_h, win_w, scale=None, eps=1e-6, dwc=None):
+    """Per-layer L/W/F schedule over a stack of independent layers.
+    q, k, v: sequences of [B,H,N,D] arrays, one per layer; dwc: None or a
+    per-layer sequence whose entries may be None."""
+    out = []
+    for l, m in enumerate(schedule):
+        if m == "L":
+            out.append(linear_attn(q[l], k[l], v[l], Hg, Wg, eps,
+                                   None if dwc is None else dwc[l]))
+        elif m == "W":
+            out.append(window_attn(q[l], k[l], v[l], Hg, Wg, win_h, win_w, scale))
+        elif m == "F":
+            out.append(full_attn(q[l], k[l], v[l], scale))
+        else:
+            raise ValueError(f"schedule[{l}] = {m!r}: expected one of L, W, F")
+    return out

@@ -1,0 +1,397 @@
+"""Pins for the float64 CPU oracle: every oracle function is checked against
+something other than itself -- brute-force N x N forms written with matrix
+algebra, closed forms, invariants, library routines (float64 SDPA, float64
+depth-wise conv2d) and the hand-worked fixtures under tests/golden/.
+CPU only.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+TOL = 1e-11
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+def _golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, vals = line.split(":")
+            out[key.strip()] = np.array([float(x) for x in vals.split()])
+    return out
+
+
+def _softmax_bruteforce(q, k, v, scale, mask=None):
+    """Explicit N x N score matrix, Eq. 1, for one head."""
+    S = (q @ k.T) * scale
+    if mask is not None:
+        S = np.where(mask, S, -np.inf)
+    P = np.exp(S - S.max(axis=1, keepdims=True))
+    return (P / P.sum(axis=1, keepdims=True)) @ v
+
+
+# --------------------------------------------------------------------------- F
+def test_full_golden_two_tokens(oracle):
+    g = _golden("full_attn_2tok.txt")
+    shp = tuple(int(x) for x in g["shape"])
+    o = oracle.full_attn(g["q"].reshape(shp), g["k"].reshape(shp), g["v"].reshape(shp),
+                         scale=float(g["scale"][0]))
+    np.testing.assert_allclose(o.reshape(-1), g["o"], rtol=0, atol=1e-14)
+
+
+def test_full_equals_bruteforce_matrix(oracle):
+    r = _rng(1)
+    B, H, N, D = 2, 3, 37, 16
+    q, k, v = (r.standard_normal((B, H, N, D)) for _ in range(3))
+    o = oracle.full_attn(q, k, v)
+    for b in range(B):
+        for h in range(H):
+            ref = _softmax_bruteforce(q[b, h], k[b, h], v[b, h], 1 / np.sqrt(D))
+            np.testing.assert_allclose(o[b, h], ref, rtol=0, atol=TOL)
+
+
+def test_full_equals_library_sdpa_float64(oracle):
+    r = _rng(2)
+    q, k, v = (r.standard_normal((1, 4, 50, 64)) for _ in range(3))
+    o = oracle.full_attn(q, k, v)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v)).numpy()
+    np.testing.assert_allclose(o, ref, rtol=0, atol=TOL)
+
+
+def test_full_explicit_scale_is_used(oracle):
+    r = _rng(3)
+    q, k, v = (r.standard_normal((1, 1, 9, 8)) for _ in range(3))
+    o = oracle.full_attn(q, k, v, scale=0.7)
+    np.testing.assert_allclose(o[0, 0], _softmax_bruteforce(q[0, 0], k[0, 0], v[0, 0], 0.7),
+                               rtol=0, atol=TOL)
+
+
+def test_full_rows_sum_to_one_and_constant_keys_give_mean(oracle):
+    r = _rng(4)
+    q, k, v = (r.standard_normal((1, 2, 33, 8)) for _ in range(3))
+    ones = np.ones_like(v)
+    np.testing.assert_allclose(oracle.full_attn(q, k, ones), ones, rtol=0, atol=1e-13)
+    kconst = np.broadcast_to(k[:, :, :1, :], k.shape).copy()
+    mean_v = np.broadcast_to(v.mean(axis=2, keepdims=True), v.shape)
+    np.testing.assert_allclose(oracle.full_attn(q, kconst, v), mean_v, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(oracle.full_attn(np.zeros_like(q), k, v), mean_v, rtol=0, atol=1e-12)
+
+
+def test_full_permutation_and_shift_invariance(oracle):
+    r = _rng(5)
+    q, k, v = (r.standard_normal((1, 2, 29, 8)) for _ in range(3))
+    o = oracle.full_attn(q, k, v)
+    pi = r.permutation(29)
+    # joint permutation of all rows permutes the output rows
+    np.testing.assert_allclose(oracle.full_attn(q[:, :, pi], k[:, :, pi], v[:, :, pi]),
+                               o[:, :, pi], rtol=0, atol=TOL)
+    # permuting only the (key, value) pairs changes nothing
+    np.testing.assert_allclose(oracle.full_attn(q, k[:, :, pi], v[:, :, pi]), o, rtol=0, atol=TOL)
+    # q.(k + c) = q.k + q.c: a per-row constant, removed by softmax
+    c = r.standard_normal((1, 2, 1, 8))
+    np.testing.assert_allclose(oracle.full_attn(q, k + c, v), o, rtol=0, atol=1e-10)
+
+
+def test_full_query_subset_equals_rows_of_full(oracle):
+    r = _rng(6)
+    q, k, v = (r.standard_normal((2, 2, 41, 8)) for _ in range(3))
+    o = oracle.full_attn(q, k, v)
+    rows = np.array([0, 7, 40, 13])
+    np.testing.assert_allclose(oracle.full_attn(q[:, :, rows], k, v), o[:, :, rows], rtol=0, atol=0)
+
+
+def test_full_large_logits_do_not_overflow(oracle):
+    q = np.full((1, 1, 3, 4), 40.0)
+    k = np.array([[[[40.0] * 4, [0.0] * 4, [-40.0] * 4]]])
+    v = np.array([[[[1.0] * 4, [2.0] * 4, [3.0] * 4]]])
+    o = oracle.full_attn(q, k, v, scale=1.0)
+    assert np.all(np.isfinite(o))
+    np.testing.assert_allclose(o, 1.0, rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- W
+def _window_ids(Hg, Wg, wh, ww):
+    y, x = np.divmod(np.arange(Hg * Wg), Wg)
+    return (y // wh) * 10_000 + (x // ww)
+
+
+def test_window_covering_grid_equals_full(oracle):
+    r = _rng(10)
+    Hg, Wg = 5, 7
+    q, k, v = (r.standard_normal((1, 2, Hg * Wg, 8)) for _ in range(3))
+    o = oracle.window_attn(q, k, v, Hg, Wg, 8, 8)
+    for h in range(2):
+        np.testing.assert_allclose(o[0, h], _softmax_bruteforce(q[0, h], k[0, h], v[0, h], 8 ** -0.5),
+                                   rtol=0, atol=TOL)
+    np.testing.assert_allclose(o, oracle.full_attn(q, k, v), rtol=0, atol=TOL)
+
+
+@pytest.mark.parametrize("Hg,Wg,wh,ww", [(8, 8, 4, 4), (6, 10, 3, 5), (7, 9, 4, 4), (9, 5, 2, 4),
+                                         (16, 16, 8, 8)])
+def test_window_equals_block_masked_full(oracle, Hg, Wg, wh, ww):
+    r = _rng(11)
+    q, k, v = (r.standard_normal((2, 2, Hg * Wg, 8)) for _ in range(3))
+    o = oracle.window_attn(q, k, v, Hg, Wg, wh, ww)
+    ids = _window_ids(Hg, Wg, wh, ww)
+    mask = ids[:, None] == ids[None, :]
+    for b in range(2):
+        for h in range(2):
+            ref = _softmax_bruteforce(q[b, h], k[b, h], v[b, h], 8 ** -0.5, mask)
+            np.testing.assert_allclose(o[b, h], ref, rtol=0, atol=TOL)
+
+
+def test_window_equals_full_on_extracted_windows(oracle):
+    r = _rng(12)
+    Hg, Wg, wh, ww, D = 7, 10, 3, 4, 8          # ragged in both directions, wh != ww
+    q, k, v = (r.standard_normal((1, 1, Hg * Wg, D)) for _ in range(3))
+    o = oracle.window_attn(q, k, v, Hg, Wg, wh, ww).reshape(Hg, Wg, D)
+    g = lambda a: a.reshape(Hg, Wg, D)
+    for y0 in range(0, Hg, wh):
+        for x0 in range(0, Wg, ww):
+            sl = (slice(y0, min(y0 + wh, Hg)), slice(x0, min(x0 + ww, Wg)))
+            qq, kk, vv = (g(a)[sl].reshape(-1, D) for a in (q, k, v))
+            ref = _softmax_bruteforce(qq, kk, vv, D ** -0.5)
+            np.testing.assert_allclose(o[sl].reshape(-1, D), ref, rtol=0, atol=TOL)
+
+
+def test_window_ragged_equals_pad_and_mask(oracle):
+    """Truncated edge windows == zero-pad the grid to a multiple of the window,
+    mask the padded keys to -inf, drop the padded query rows."""
+    r = _rng(13)
+    Hg, Wg, w, D = 9, 11, 4, 8
+    Hp, Wp = 12, 12
+    q, k, v = (r.standard_normal((1, 1, Hg * Wg, D)) for _ in range(3))
+    o = oracle.window_attn(q, k, v, Hg, Wg, w, w).reshape(Hg, Wg, D)
+
+    def pad(a):
+        p = np.zeros((Hp, Wp, D))
+        p[:Hg, :Wg] = a.reshape(Hg, Wg, D)
+        return p.reshape(-1, D)
+    valid = np.zeros((Hp, Wp), dtype=bool)
+    valid[:Hg, :Wg] = True
+    ids = _window_ids(Hp, Wp, w, w)
+    mask = (ids[:, None] == ids[None, :]) & valid.reshape(-1)[None, :]
+    ref = _softmax_bruteforce(pad(q), pad(k), pad(v), D ** -0.5, mask).reshape(Hp, Wp, D)
+    np.testing.assert_allclose(o, ref[:Hg, :Wg], rtol=0, atol=TOL)
+
+
+def test_window_of_one_token_returns_v(oracle):
+    r = _rng(14)
+    q, k, v = (r.standard_normal((1, 2, 12, 4)) for _ in range(3))
+    np.testing.assert_allclose(oracle.window_attn(q, k, v, 3, 4, 1, 1), v, rtol=0, atol=1e-14)
+
+
+# --------------------------------------------------------------------------- L
+def _linear_naive(q, k, v, eps):
+    """O(N^2) form: sum_j (phi(q_i).phi(k_j)) v_j / (sum_j phi(q_i).phi(k_j) + eps)."""
+    A = np.maximum(q, 0) @ np.maximum(k, 0).T
+    return (A @ v) / (A.sum(axis=1, keepdims=True) + eps)
+
+
+def test_linear_golden_two_tokens(oracle):
+    g = _golden("linear_attn_2tok.txt")
+    shp = tuple(int(x) for x in g["shape"])
+    Hg, Wg = (int(x) for x in g["grid"])
+    o = oracle.linear_attn(g["q"].reshape(shp), g["k"].reshape(shp), g["v"].reshape(shp),
+                           Hg, Wg, eps=float(g["eps"][0]))
+    np.testing.assert_allclose(o.reshape(-1), g["o"], rtol=0, atol=1e-15)
+
+
+def test_linear_equals_naive_quadratic_form(oracle):
+    r = _rng(20)
+    B, H, Hg, Wg, D = 2, 3, 5, 7, 16
+    q, k, v = (r.standard_normal((B, H, Hg * Wg, D)) for _ in range(3))
+    for eps in (1e-6, 0.5):     # eps large enough that its placement matters
+        o = oracle.linear_attn(q, k, v, Hg, Wg, eps=eps)
+        for b in range(B):
+            for h in range(H):
+                np.testing.assert_allclose(o[b, h], _linear_naive(q[b, h], k[b, h], v[b, h], eps),
+                                           rtol=0, atol=1e-12)
+
+
+def test_linear_closed_forms(oracle):
+    r = _rng(21)
+    Hg, Wg, D = 4, 6, 8
+    q, k, v = (r.standard_normal((1, 2, Hg * Wg, D)) for _ in range(3))
+    eps = 1e-3
+    # V = 1 -> O_i = D_i / (D_i + eps) with D_i = phi(q_i) . sum_j phi(k_j)
+    Di = np.einsum("bhnd,bhd->bhn", np.maximum(q, 0), np.maximum(k, 0).sum(axis=2))
+    o1 = oracle.linear_attn(q, k, np.ones_like(v), Hg, Wg, eps=eps)
+    np.testing.assert_allclose(o1, np.broadcast_to((Di / (Di + eps))[..., None], v.shape),
+                               rtol=0, atol=1e-13)
+    # q_i <= 0 componentwise -> phi(q_i) = 0 -> O_i = 0 exactly
+    qn = q.copy()
+    qn[0, 0, 5] = -np.abs(qn[0, 0, 5])
+    assert np.all(oracle.linear_attn(qn, k, v, Hg, Wg, eps=eps)[0, 0, 5] == 0.0)
+    # Q >= 0 and K >= 0: ReLU is the identity -> normalised (Q K^T) V
+    qa, ka = np.abs(q), np.abs(k)
+    A = np.einsum("bhid,bhjd->bhij", qa, ka)
+    ref = np.einsum("bhij,bhjd->bhid", A, v) / (A.sum(-1, keepdims=True) + eps)
+    np.testing.assert_allclose(oracle.linear_attn(qa, ka, v, Hg, Wg, eps=eps), ref, rtol=0, atol=1e-12)
+
+
+def test_linear_scale_and_permutation_invariance(oracle):
+    r = _rng(22)
+    Hg, Wg, D = 3, 9, 8
+    q, k, v = (r.standard_normal((1, 2, Hg * Wg, D)) for _ in range(3))
+    o = oracle.linear_attn(q, k, v, Hg, Wg, eps=0.0)
+    np.testing.assert_allclose(oracle.linear_attn(3.0 * q, k, v, Hg, Wg, eps=0.0), o, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(oracle.linear_attn(q, 0.25 * k, v, Hg, Wg, eps=0.0), o, rtol=0, atol=1e-12)
+    pi = r.permutation(Hg * Wg)
+    np.testing.assert_allclose(oracle.linear_attn(q, k[:, :, pi], v[:, :, pi], Hg, Wg, eps=0.0), o,
+                               rtol=0, atol=1e-12)
+    np.testing.assert_allclose(oracle.linear_attn(q[:, :, pi], k, v, Hg, Wg, eps=0.0), o[:, :, pi],
+                               rtol=0, atol=1e-12)
+
+
+# ------------------------------------------------------------------------ L4 DWC
+def _static_dwc(C, k, kernel):
+    """Generator that emits a fixed kernel: W2 = 0, b2 = kernel, any W1."""
+    R = 3
+    return {"k": k, "R": R, "W1": np.ones((R, C)), "b1": None,
+            "W2": np.zeros((C * k * k, R)), "b2": np.asarray(kernel, dtype=np.float64).reshape(-1)}
+
+
+def _to_image(v, Hg, Wg):
+    """[B,H,N,D] -> [B, C=H*D, Hg, Wg] with channel c = h*D + e."""
+    B, H, N, D = v.shape
+    return v.reshape(B, H, Hg, Wg, D).transpose(0, 1, 4, 2, 3).reshape(B, H * D, Hg, Wg)
+
+
+def _from_image(img, H, D):
+    B, C, Hg, Wg = img.shape
+    return img.reshape(B, H, D, Hg, Wg).transpose(0, 1, 3, 4, 2).reshape(B, H, Hg * Wg, D)
+
+
+def test_dwc_golden_3x3(oracle):
+    g = _golden("dwc_3x3.txt")
+    shp = tuple(int(x) for x in g["shape"])
+    Hg, Wg = (int(x) for x in g["grid"])
+    v = g["v"].reshape(shp)
+    q = -np.ones(shp)
+    o = oracle.linear_attn(q, np.ones(shp), v, Hg, Wg, dwc=_static_dwc(1, 3, g["w"]))
+    np.testing.assert_allclose(o.reshape(-1), g["o"], rtol=0, atol=1e-13)
+
+
+@pytest.mark.parametrize("ksz", [3, 5])
+def test_dwc_static_equals_library_depthwise_conv(oracle, ksz):
+    r = _rng(30)
+    B, H, Hg, Wg, D = 2, 3, 6, 7, 4
+    C = H * D
+    q, k, v = (r.standard_normal((B, H, Hg * Wg, D)) for _ in range(3))
+    kernel = r.standard_normal((C, ksz, ksz))
+    la = oracle.linear_attn(q, k, v, Hg, Wg)
+    o = oracle.linear_attn(q, k, v, Hg, Wg, dwc=_static_dwc(C, ksz, kernel))
+    conv = torch.nn.functional.conv2d(torch.from_numpy(_to_image(v, Hg, Wg)),
+                                      torch.from_numpy(kernel)[:, None], padding=ksz // 2, groups=C)
+    np.testing.assert_allclose(o - la, _from_image(conv.numpy(), H, D), rtol=0, atol=1e-12)
+
+
+def test_dwc_delta_kernel_adds_v_and_constant_v_shows_padding(oracle):
+    r = _rng(31)
+    B, H, Hg, Wg, D = 1, 2, 5, 6, 4
+    C = H * D
+    q, k, v = (r.standard_normal((B, H, Hg * Wg, D)) for _ in range(3))
+    la = oracle.linear_attn(q, k, v, Hg, Wg)
+    delta = np.zeros((C, 3, 3))
+    delta[:, 1, 1] = 1.0
+    np.testing.assert_allclose(oracle.linear_attn(q, k, v, Hg, Wg, dwc=_static_dwc(C, 3, delta)),
+                               la + v, rtol=0, atol=1e-13)
+    # constant V, all-ones kernel: interior = 9 c, edges = 6 c, corners = 4 c
+    vc = np.full_like(v, 2.0)
+    lac = oracle.linear_attn(q, k, vc, Hg, Wg)
+    dw = (oracle.linear_attn(q, k, vc, Hg, Wg, dwc=_static_dwc(C, 3, np.ones((C, 3, 3)))) - lac)
+    dw = dw.reshape(B, H, Hg, Wg, D)
+    np.testing.assert_allclose(dw[:, :, 1:-1, 1:-1], 18.0, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dw[:, :, 0, 1:-1], 12.0, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dw[:, :, 1:-1, -1], 12.0, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dw[:, :, 0, 0], 8.0, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(dw[:, :, -1, -1], 8.0, rtol=0, atol=1e-12)
+
+
+def test_dwc_generator_special_cases(oracle):
+    r = _rng(32)
+    B, H, N, D, ksz, R = 2, 2, 12, 4, 3, 5
+    C = H * D
+    v = r.standard_normal((B, H, N, D))
+    W1 = r.standard_normal((R, C))
+    W2 = r.standard_normal((C * 9, R))
+    b2 = r.standard_normal(C * 9)
+    # SiLU(0) = 0: with W1 = 0 and no b1 the hidden layer vanishes, w = b2
+    w = oracle.dwc_generate(v, {"k": ksz, "R": R, "W1": 0 * W1, "b1": None, "W2": W2, "b2": b2})
+    np.testing.assert_allclose(w.reshape(B, -1), np.broadcast_to(b2, (B, C * 9)), rtol=0, atol=0)
+    # SiLU(x) -> x for large x: pre-activation 40 gives hid = 40 / (1 + e^-40)
+    b1 = np.full(R, 40.0)
+    w = oracle.dwc_generate(v, {"k": ksz, "R": R, "W1": 0 * W1, "b1": b1, "W2": W2, "b2": None})
+    np.testing.assert_allclose(w.reshape(B, -1), np.broadcast_to(W2.sum(1) * 40.0, (B, C * 9)),
+                               rtol=1e-15, atol=1e-12)
+    # average pooling: V constant per channel -> s = that constant, whatever N
+    vch = np.broadcast_to(r.standard_normal((B, H, 1, D)), (B, H, N, D)).copy()
+    w = oracle.dwc_generate(vch, {"k": ksz, "R": R, "W1": W1, "b1": None, "W2": W2, "b2": b2})
+    s = torch.from_numpy(vch[:, :, 0, :].reshape(B, C))
+    hid = torch.nn.functional.silu(torch.nn.functional.linear(s, torch.from_numpy(W1)))
+    ref = torch.nn.functional.linear(hid, torch.from_numpy(W2), torch.from_numpy(b2)).numpy()
+    np.testing.assert_allclose(w.reshape(B, -1), ref, rtol=0, atol=1e-12)
+
+
+def test_dwc_generator_equals_library_mlp_and_pooling(oracle):
+    r = _rng(33)
+    B, H, Hg, Wg, D, ksz, R = 2, 3, 4, 5, 4, 3, 6
+    C = H * D
+    v = r.standard_normal((B, H, Hg * Wg, D))
+    dwc = {"k": ksz, "R": R, "W1": r.standard_normal((R, C)), "b1": r.standard_normal(R),
+           "W2": r.standard_normal((C * 9, R)), "b2": r.standard_normal(C * 9)}
+    w = oracle.dwc_generate(v, dwc)
+    img = torch.from_numpy(_to_image(v, Hg, Wg))
+    s = torch.nn.functional.adaptive_avg_pool2d(img, 1).reshape(B, C)
+    hid = torch.nn.functional.silu(torch.nn.functional.linear(
+        s, torch.from_numpy(dwc["W1"]), torch.from_numpy(dwc["b1"])))
+    ref = torch.nn.functional.linear(hid, torch.from_numpy(dwc["W2"]), torch.from_numpy(dwc["b2"]))
+    np.testing.assert_allclose(w.reshape(B, -1), ref.numpy(), rtol=0, atol=1e-12)
+    # and the whole block: LA + conv2d with those per-sample kernels
+    q, k = (r.standard_normal(v.shape) for _ in range(2))
+    o = oracle.linear_attn(q, k, v, Hg, Wg, dwc=dwc)
+    la = oracle.linear_attn(q, k, v, Hg, Wg)
+    for b in range(B):
+        conv = torch.nn.functional.conv2d(img[b:b + 1], ref[b].reshape(C, 1, ksz, ksz), padding=1, groups=C)
+        np.testing.assert_allclose((o - la)[b:b + 1], _from_image(conv.numpy(), H, D), rtol=0, atol=1e-12)
+
+
+# --------------------------------------------------------------------------- S
+def test_hybrid_schedule_runs_each_layer_with_its_mixer(oracle):
+    r = _rng(40)
+    Hg, Wg, D, L = 6, 6, 8, 4
+    qs, ks, vs = ([r.standard_normal((1, 2, Hg * Wg, D)) for _ in range(L)] for _ in range(3))
+    out = oracle.hybrid_mixers("LWFL", qs, ks, vs, Hg, Wg, 3, 3)
+    np.testing.assert_array_equal(out[0], oracle.linear_attn(qs[0], ks[0], vs[0], Hg, Wg))
+    np.testing.assert_array_equal(out[1], oracle.window_attn(qs[1], ks[1], vs[1], Hg, Wg, 3, 3))
+    np.testing.assert_array_equal(out[2], oracle.full_attn(qs[2], ks[2], vs[2]))
+    np.testing.assert_array_equal(out[3], oracle.linear_attn(qs[3], ks[3], vs[3], Hg, Wg))
+    with pytest.raises(ValueError):
+        oracle.hybrid_mixers("LX", qs, ks, vs, Hg, Wg, 3, 3)
+
+
+def test_tiny_config_invariants(oracle):
+    """The tiny workload itself (16x16 grid, 6 heads, D = 64): L vs the naive form,
+    W with one window vs F, F rows summing to one."""
+    from paper_2605_26636_b200 import inputs
+    w = inputs.WORKLOADS["tiny"]
+    q, k, v = (t.double().numpy() for t in inputs.qkv(w))
+    ol = oracle.linear_attn(q, k, v, w.Hg, w.Wg)
+    for h in range(w.H):
+        np.testing.assert_allclose(ol[0, h], _linear_naive(q[0, h], k[0, h], v[0, h], 1e-6), rtol=0, atol=1e-12)
+    of = oracle.full_attn(q, k, v)
+    np.testing.assert_allclose(oracle.window_attn(q, k, v, w.Hg, w.Wg, 16, 16), of, rtol=0, atol=TOL)
+    np.testing.assert_allclose(oracle.full_attn(q, k, np.ones_like(v)), 1.0, rtol=0, atol=1e-13)
+    ow = oracle.window_attn(q, k, v, w.Hg, w.Wg, 8, 8)
+    assert np.abs(ow - of).max() > 1e-3      # 8x8 windows are a different operator
