@@ -1,0 +1,161 @@
+/*
+ * jetvit.h -- C ABI of libjetvit: the token mixers of a JetViT hybrid Vision
+ * Transformer as CUDA kernels for NVIDIA B200 (sm_100a).
+ *
+ * Three mixers and a schedule driver (JetViT, Sec. 3.2):
+ *   L  linear-attention block: ReLU-kernel linear attention (Eq. 2) with the row
+ *      normalisation, plus the optional squeeze dynamic depth-wise convolution
+ *      on V (Sec. 3.2.1, Eq. 4);
+ *   W  2D window attention over non-overlapping windows (Sec. 3.2.2);
+ *   F  full softmax attention (Eq. 1);
+ *   S  a per-layer L/W/F schedule over a stack of independent layers
+ *      (Sec. 3.2.3, Fig. 1b).
+ *
+ * Conventions shared by every call
+ *   Tensors   q, k, v, o are DEVICE pointers to [B, H, N, D] contiguous arrays,
+ *             D fastest, N = Hg * Wg, token t at grid position (t / Wg, t % Wg).
+ *             All four have the element type jv_shape.dtype; o must not alias an
+ *             input.  Pointers must be 16-byte aligned.
+ *   Ownership The caller owns every buffer and the stream.  The library never
+ *             allocates or frees device memory; scratch comes from the caller
+ *             through (ws, ws_bytes), sized by jv_workspace_bytes(), 256-byte
+ *             aligned.  ws may be NULL when jv_workspace_bytes() returns 0.
+ *   Stream    cuda_stream is a cudaStream_t passed as void* (NULL = default
+ *             stream).  Calls only enqueue work and return; results are valid
+ *             once the caller has synchronised the stream.  Calls that share a
+ *             workspace must be ordered on one stream.
+ *   Errors    Return codes only.  Every argument error is found on the host
+ *             before anything is launched.  There is no CPU fallback: without a
+ *             usable sm_100 device the calls return JV_ERR_CUDA/JV_ERR_UNSUPPORTED.
+ *             Kernels bound every wait; one that gives up records
+ *             JV_ERR_TIMEOUT, which jv_device_status() reports.
+ *   Precision bf16 tensors: bf16 tensor-core products with fp32 accumulation,
+ *             fp32 softmax / state, round-to-nearest-even output.  f32 tensors:
+ *             fp32 arithmetic throughout (no tf32).
+ */
+#ifndef JETVIT_H_
+#define JETVIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  JV_OK = 0,
+  JV_ERR_INVALID_ARG = 1,  /* null / misaligned pointer, non-positive size, bad schedule character */
+  JV_ERR_UNSUPPORTED = 2,  /* shape or dtype outside what the kernels cover (e.g. D > 256) */
+  JV_ERR_WORKSPACE = 3,    /* ws is NULL, misaligned or smaller than jv_workspace_bytes() */
+  JV_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed */
+  JV_ERR_TIMEOUT = 5       /* a kernel gave up on a bounded wait */
+} jv_status;
+
+typedef enum { JV_F32 = 0, JV_BF16 = 1 } jv_dtype;
+
+/* Problem shape.  N = Hg * Wg tokens per (batch, head). */
+typedef struct {
+  int32_t B, H, Hg, Wg, D;
+  int32_t dtype; /* jv_dtype */
+} jv_shape;
+
+/*
+ * Kernel generator of the squeeze dynamic depth-wise convolution (Sec. 3.2.1):
+ * a two-layer MLP with SiLU fed by the average-pooled V.  All pointers are
+ * DEVICE pointers to fp32, row-major; C = H * D, channel c = h * D + e.
+ */
+typedef struct {
+  int32_t k;       /* odd kernel edge: 3 or 5 */
+  int32_t R;       /* hidden width of the generator, 1..1024 */
+  const float* W1; /* [R, C] */
+  const float* b1; /* [R] or NULL */
+  const float* W2; /* [C*k*k, R] */
+  const float* b2; /* [C*k*k] or NULL */
+} jv_dwc;
+
+/*
+ * Bytes of scratch the given mixer needs for this shape.  mixer is 'L', 'W', 'F'
+ * or 'S' (the maximum over the three, for jv_hybrid_mixers).  dwc may be NULL;
+ * pass the descriptor that the L call will get, since it enlarges the scratch.
+ * Returns 0 on invalid arguments as well as when no scratch is needed.
+ */
+size_t jv_workspace_bytes(char mixer, const jv_shape* shape, const jv_dwc* dwc);
+
+/*
+ * L -- JetViT linear-attention block (Sec. 3.2.1; Eq. 2 reordered, Eq. 4).
+ *   KV = sum_j relu(k_j)^T v_j,  z = sum_j relu(k_j)          per (batch, head)
+ *   o_i = relu(q_i) KV / (relu(q_i) . z + eps)
+ *   and, when dwc != NULL:  s = mean_j v_j (per sample and channel),
+ *   w = W2 SiLU(W1 s + b1) + b2 viewed as [C, k, k],
+ *   o_i += depth-wise k x k convolution of V (as an Hg x Wg image, zero padding
+ *   (k-1)/2, stride 1) with the sample's kernels w.
+ * eps is added to the denominator only (1e-6 in the paper's setting; must be >= 0).
+ * Phase 1 reduces the state over token chunks into ws; a second pass sums the
+ * chunk partials in a fixed order (no floating-point atomics: results are
+ * bit-reproducible); phase 2 streams q -> o.
+ */
+jv_status jv_linear_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
+                         float eps, const jv_dwc* dwc, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * W -- window attention (Sec. 3.2.2): the grid is cut into non-overlapping
+ * win_h x win_w windows anchored at (0, 0); softmax attention (Eq. 1) runs
+ * inside each window.  When the grid is not a multiple of the window the
+ * right / bottom windows hold only the tokens that exist (their missing keys are
+ * masked out, their missing query rows are never written).  A window at least as
+ * large as the grid is full attention.  scale <= 0 selects 1/sqrt(D).
+ */
+jv_status jv_window_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
+                         int32_t win_h, int32_t win_w, float scale, void* ws, size_t ws_bytes,
+                         void* cuda_stream);
+
+/*
+ * F -- full softmax attention (Eq. 1): o = softmax(q k^T * scale) v over all N
+ * tokens of each (batch, head), non-causal, computed flash-style with an fp32
+ * online softmax.  scale <= 0 selects 1/sqrt(D).
+ */
+jv_status jv_full_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
+                       float scale, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * S -- hybrid stack (Sec. 3.2.3): for l in [0, n_layers) run mixer schedule[l]
+ * ('L', 'W' or 'F') on layer l's tensors.  q, k, v, o are HOST arrays of n_layers
+ * DEVICE pointers; all layers share one shape.  dwc is NULL or a HOST array of
+ * n_layers entries (each NULL or a host pointer to a jv_dwc) used by the L layers.
+ * Layers are independent; they are enqueued in order on one stream with no host
+ * synchronisation in between.  ws must cover jv_workspace_bytes('S', ...).
+ * The schedule is validated completely before the first launch.
+ */
+jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* const* q,
+                           const void* const* k, const void* const* v, void* const* o,
+                           const jv_shape* shape, int32_t win_h, int32_t win_w, float scale, float eps,
+                           const jv_dwc* const* dwc, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Synchronises the stream, then returns and clears the sticky device status:
+ * JV_OK, JV_ERR_TIMEOUT if a kernel abandoned a bounded wait since the last
+ * call, or JV_ERR_CUDA if the stream reports a CUDA error.
+ */
+jv_status jv_device_status(void* cuda_stream);
+
+/*
+ * Tuning / dispatch switch, mainly for tests: 0 (default) lets every call pick
+ * its fastest kernel for the shape; 1 forces the shape-generic fp32-arithmetic
+ * kernels for every call.  Returns the previous value.  Process-wide.
+ */
+int32_t jv_set_force_generic(int32_t on);
+
+/*
+ * Number of kernel launches the library has enqueued since it was loaded
+ * (process-wide counter; used to report launches per benchmark step).
+ */
+uint64_t jv_launch_count(void);
+
+const char* jv_status_string(jv_status s);
+const char* jv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JETVIT_H_ */

@@ -1,0 +1,233 @@
+// C ABI of libjetvit: argument validation, dispatch, device status.
+// Every argument error is reported before anything is launched.
+#include <atomic>
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace jv {
+namespace {
+
+__device__ int g_status_word = 0;          // sticky error bits written by kernels
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int32_t> g_force_generic{0};
+
+bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+jv_status check_shape(const jv_shape* s) {
+  if (!s) return JV_ERR_INVALID_ARG;
+  if (s->B <= 0 || s->H <= 0 || s->Hg <= 0 || s->Wg <= 0 || s->D <= 0) return JV_ERR_INVALID_ARG;
+  if (s->dtype != JV_F32 && s->dtype != JV_BF16) return JV_ERR_INVALID_ARG;
+  if ((int64_t)s->Hg * s->Wg > (1 << 24)) return JV_ERR_UNSUPPORTED;
+  if ((int64_t)s->B * s->H > 65535) return JV_ERR_UNSUPPORTED;
+  if (s->D > 128) return JV_ERR_UNSUPPORTED;
+  // rows must keep 16-byte alignment for the vector loads
+  const int esz = s->dtype == JV_F32 ? 4 : 2;
+  if ((s->D * esz) % 16 != 0) return JV_ERR_UNSUPPORTED;
+  return JV_OK;
+}
+
+jv_status check_tensors(const void* q, const void* k, const void* v, const void* o, const jv_shape* s) {
+  if (!q || !k || !v || !o) return JV_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return JV_ERR_INVALID_ARG;
+  if (o == q || o == k || o == v) return JV_ERR_INVALID_ARG;
+  (void)s;
+  return JV_OK;
+}
+
+jv_status check_dwc(const jv_dwc* d) {
+  if (!d) return JV_OK;
+  if (d->k != 3 && d->k != 5) return JV_ERR_INVALID_ARG;
+  if (d->R <= 0 || d->R > 1024) return JV_ERR_INVALID_ARG;
+  if (!d->W1 || !d->W2) return JV_ERR_INVALID_ARG;
+  return JV_OK;
+}
+
+jv_status check_ws(const void* ws, size_t ws_bytes, size_t need) {
+  if (need == 0) return JV_OK;
+  if (!ws || !aligned(ws, 256) || ws_bytes < need) return JV_ERR_WORKSPACE;
+  return JV_OK;
+}
+
+jv_status check_window(const jv_shape* s, int wh, int ww) {
+  if (wh <= 0 || ww <= 0) return JV_ERR_INVALID_ARG;
+  const int64_t nwin = (int64_t)ceil_div(s->Hg, wh < s->Hg ? wh : s->Hg) * ceil_div(s->Wg, ww < s->Wg ? ww : s->Wg);
+  if (nwin > 65535) return JV_ERR_UNSUPPORTED;
+  return JV_OK;
+}
+
+jv_status check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return JV_ERR_CUDA; }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return JV_ERR_CUDA;
+  }
+  return major == 10 ? JV_OK : JV_ERR_UNSUPPORTED;
+}
+
+jv_status from_cuda(cudaError_t e) { return e == cudaSuccess ? JV_OK : JV_ERR_CUDA; }
+
+float pick_scale(float scale, int D) { return scale > 0.f ? scale : 1.f / sqrtf((float)D); }
+
+// ---- enqueue helpers (arguments already validated) ---------------------------
+jv_status run_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* s, int wh, int ww,
+                   float scale, bool full, cudaStream_t st) {
+  AttnArgs a{q, k, v, o, s->B * s->H, s->Hg, s->Wg, s->D, wh, ww, pick_scale(scale, s->D), s->dtype};
+  if (!g_force_generic.load() && attn_tc_supported(a, full)) {
+    int* status = device_status_ptr();
+    if (!status) return JV_ERR_CUDA;
+    return from_cuda(launch_attn_tc(a, full, status, st));
+  }
+  return from_cuda(launch_attn_generic(a, st));
+}
+
+jv_status run_linear(const void* q, const void* k, const void* v, void* o, const jv_shape* s, float eps,
+                     const jv_dwc* dwc, void* ws, cudaStream_t st) {
+  LinArgs a{q, k, v, o, *s, eps, dwc, ws};
+  const LinPlan p = lin_plan(*s, dwc);
+  if (!g_force_generic.load() && linear_fast_supported(a)) return from_cuda(launch_linear_fast(a, p, st));
+  return from_cuda(launch_linear_generic(a, p, st));
+}
+
+}  // namespace
+
+int* device_status_ptr() {
+  // One address per device; looked up once per device and cached.
+  static int* cache[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cache[dev]) {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_status_word) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    cache[dev] = p;
+  }
+  return cache[dev];
+}
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+}  // namespace jv
+
+using namespace jv;
+
+extern "C" {
+
+size_t jv_workspace_bytes(char mixer, const jv_shape* shape, const jv_dwc* dwc) {
+  if (check_shape(shape) != JV_OK || check_dwc(dwc) != JV_OK) return 0;
+  switch (mixer) {
+    case 'L':
+    case 'S':
+      return lin_plan(*shape, dwc).total;   // W and F need no scratch
+    case 'W':
+    case 'F':
+      return 0;
+    default:
+      return 0;
+  }
+}
+
+jv_status jv_linear_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape, float eps,
+                         const jv_dwc* dwc, void* ws, size_t ws_bytes, void* cuda_stream) {
+  jv_status st = check_shape(shape);
+  if (st != JV_OK) return st;
+  if ((st = check_tensors(q, k, v, o, shape)) != JV_OK) return st;
+  if (!(eps >= 0.f)) return JV_ERR_INVALID_ARG;
+  if ((st = check_dwc(dwc)) != JV_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, lin_plan(*shape, dwc).total)) != JV_OK) return st;
+  if ((st = check_device()) != JV_OK) return st;
+  return run_linear(q, k, v, o, shape, eps, dwc, ws, (cudaStream_t)cuda_stream);
+}
+
+jv_status jv_window_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
+                         int32_t win_h, int32_t win_w, float scale, void* ws, size_t ws_bytes,
+                         void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  jv_status st = check_shape(shape);
+  if (st != JV_OK) return st;
+  if ((st = check_tensors(q, k, v, o, shape)) != JV_OK) return st;
+  if ((st = check_window(shape, win_h, win_w)) != JV_OK) return st;
+  if ((st = check_device()) != JV_OK) return st;
+  return run_attn(q, k, v, o, shape, win_h, win_w, scale, false, (cudaStream_t)cuda_stream);
+}
+
+jv_status jv_full_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape, float scale,
+                       void* ws, size_t ws_bytes, void* cuda_stream) {
+  (void)ws; (void)ws_bytes;
+  jv_status st = check_shape(shape);
+  if (st != JV_OK) return st;
+  if ((st = check_tensors(q, k, v, o, shape)) != JV_OK) return st;
+  if ((st = check_device()) != JV_OK) return st;
+  return run_attn(q, k, v, o, shape, shape->Hg, shape->Wg, scale, true, (cudaStream_t)cuda_stream);
+}
+
+jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* const* q, const void* const* k,
+                           const void* const* v, void* const* o, const jv_shape* shape, int32_t win_h,
+                           int32_t win_w, float scale, float eps, const jv_dwc* const* dwc, void* ws,
+                           size_t ws_bytes, void* cuda_stream) {
+  if (n_layers <= 0 || !schedule || !q || !k || !v || !o) return JV_ERR_INVALID_ARG;
+  jv_status st = check_shape(shape);
+  if (st != JV_OK) return st;
+  if (!(eps >= 0.f)) return JV_ERR_INVALID_ARG;
+  size_t need = 0;
+  bool any_w = false;
+  for (int l = 0; l < n_layers; ++l) {
+    const char m = schedule[l];
+    if (m != 'L' && m != 'W' && m != 'F') return JV_ERR_INVALID_ARG;   // also catches an early '\0'
+    if ((st = check_tensors(q[l], k[l], v[l], o[l], shape)) != JV_OK) return st;
+    if (m == 'W') any_w = true;
+    if (m == 'L') {
+      const jv_dwc* d = dwc ? dwc[l] : nullptr;
+      if ((st = check_dwc(d)) != JV_OK) return st;
+      const size_t n = lin_plan(*shape, d).total;
+      if (n > need) need = n;
+    }
+  }
+  if (any_w && (st = check_window(shape, win_h, win_w)) != JV_OK) return st;
+  if ((st = check_ws(ws, ws_bytes, need)) != JV_OK) return st;
+  if ((st = check_device()) != JV_OK) return st;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  for (int l = 0; l < n_layers; ++l) {
+    switch (schedule[l]) {
+      case 'L': st = run_linear(q[l], k[l], v[l], o[l], shape, eps, dwc ? dwc[l] : nullptr, ws, stream); break;
+      case 'W': st = run_attn(q[l], k[l], v[l], o[l], shape, win_h, win_w, scale, false, stream); break;
+      default:  st = run_attn(q[l], k[l], v[l], o[l], shape, shape->Hg, shape->Wg, scale, true, stream); break;
+    }
+    if (st != JV_OK) return st;
+  }
+  return JV_OK;
+}
+
+jv_status jv_device_status(void* cuda_stream) {
+  if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) { cudaGetLastError(); return JV_ERR_CUDA; }
+  int word = 0;
+  if (cudaMemcpyFromSymbol(&word, g_status_word, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return JV_ERR_CUDA; }
+  if (word != 0) {
+    const int zero = 0;
+    cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int));
+    return JV_ERR_TIMEOUT;
+  }
+  return JV_OK;
+}
+
+int32_t jv_set_force_generic(int32_t on) { return g_force_generic.exchange(on ? 1 : 0); }
+
+uint64_t jv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* jv_status_string(jv_status s) {
+  switch (s) {
+    case JV_OK: return "ok";
+    case JV_ERR_INVALID_ARG: return "invalid argument";
+    case JV_ERR_UNSUPPORTED: return "unsupported shape, dtype or device";
+    case JV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case JV_ERR_CUDA: return "CUDA call failed";
+    case JV_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+    default: return "unknown status";
+  }
+}
+
+const char* jv_version(void) { return "jetvit-b200 0.1.0 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,82 @@
+// Shared host/device helpers of libjetvit (internal; not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "jetvit.h"
+
+namespace jv {
+
+// ---- device status word ---------------------------------------------------
+// One int per device context lives in status.cu; kernels receive its device
+// address and OR error bits into it.  Bit 0: a bounded wait ran out.
+constexpr int kStatusTimeout = 1;
+
+int* device_status_ptr();        // device address of the status word (nullptr on failure)
+void count_launch(int n = 1);    // launch counter behind jv_launch_count()
+
+// ---- element access -------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void from_f32(float* p, float x) { *p = x; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- plan of the linear-attention workspace --------------------------------
+// State per (batch, head): (D+1) x (D+1) fp32, S[a][e] = sum_j pk[j][a] * pv[j][e]
+// with pk = [relu(k) | 1], pv = [v | 1]:  S[a<D][e<D] = KV, S[a][D] = z (k-sum),
+// S[D][e] = v-sum, S[D][D] = N.
+struct LinPlan {
+  int D1;            // D + 1
+  int state_elems;   // D1 * D1 rounded up to a multiple of 4
+  int chunk_tokens;  // tokens per phase-1 chunk
+  int nchunk;        // chunks per (batch, head)
+  size_t off_partial, off_state, off_hidden, off_kernel, total;  // byte offsets into ws
+};
+LinPlan lin_plan(const jv_shape& s, const jv_dwc* dwc);
+
+// ---- kernels' host launchers (each returns a cudaError_t from the launch) ---
+struct AttnArgs {
+  const void *q, *k, *v;
+  void* o;
+  int BH, Hg, Wg, D;
+  int wh, ww;  // window size (wh >= Hg and ww >= Wg: one window = full attention)
+  float scale;
+  int dtype;
+};
+cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st);
+// tcgen05 path: bf16, D == 64.  full = true: F over all N tokens; else W with
+// (wh, ww) windows, ww a power of two dividing 128, wh*ww a multiple of 128 and <= 256...
+bool attn_tc_supported(const AttnArgs& a, bool full);
+cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream_t st);
+
+struct LinArgs {
+  const void *q, *k, *v;
+  void* o;
+  jv_shape s;
+  float eps;
+  const jv_dwc* dwc;  // host struct holding device pointers, or nullptr
+  void* ws;
+};
+cudaError_t launch_linear_generic(const LinArgs& a, const LinPlan& p, cudaStream_t st);
+bool linear_fast_supported(const LinArgs& a);
+cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t st);
+// shared by both linear paths: hidden = SiLU(W1 s + b1), w = W2 hidden + b2
+cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, cudaStream_t st);
+
+}  // namespace jv

@@ -1,0 +1,228 @@
+"""ctypes binding of libjetvit.so: same names as the C ABI, argument marshalling
+only.  Tensors are CUDA ``torch`` tensors (device memory and streams come from
+PyTorch); every step of every mixer runs in the library's CUDA kernels.  There
+is no CPU path: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+JV_OK, JV_ERR_INVALID_ARG, JV_ERR_UNSUPPORTED, JV_ERR_WORKSPACE, JV_ERR_CUDA, JV_ERR_TIMEOUT = range(6)
+JV_F32, JV_BF16 = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libjetvit.so")
+
+
+class JvShape(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("Hg", ctypes.c_int32),
+                ("Wg", ctypes.c_int32), ("D", ctypes.c_int32), ("dtype", ctypes.c_int32)]
+
+
+class JvDwc(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_int32), ("R", ctypes.c_int32), ("W1", ctypes.c_void_p),
+                ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
+
+
+class JetVitError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (jv_status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libjetvit.so (built in-tree by ``paper_2605_26636_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2605_26636_b200.build` "
+                              "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, i32, f32 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int32, ctypes.c_float
+        shp, dwc = ctypes.POINTER(JvShape), ctypes.POINTER(JvDwc)
+        L.jv_workspace_bytes.argtypes = [ctypes.c_char, shp, dwc]
+        L.jv_workspace_bytes.restype = sz
+        L.jv_linear_attn.argtypes = [vp, vp, vp, vp, shp, f32, dwc, vp, sz, vp]
+        L.jv_window_attn.argtypes = [vp, vp, vp, vp, shp, i32, i32, f32, vp, sz, vp]
+        L.jv_full_attn.argtypes = [vp, vp, vp, vp, shp, f32, vp, sz, vp]
+        L.jv_hybrid_mixers.argtypes = [i32, ctypes.c_char_p, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                       ctypes.POINTER(vp), ctypes.POINTER(vp), shp, i32, i32, f32, f32,
+                                       ctypes.POINTER(dwc), vp, sz, vp]
+        L.jv_device_status.argtypes = [vp]
+        for f in (L.jv_linear_attn, L.jv_window_attn, L.jv_full_attn, L.jv_hybrid_mixers, L.jv_device_status):
+            f.restype = ctypes.c_int
+        L.jv_set_force_generic.argtypes = [i32]
+        L.jv_set_force_generic.restype = i32
+        L.jv_launch_count.restype = ctypes.c_uint64
+        L.jv_status_string.argtypes = [ctypes.c_int]
+        L.jv_status_string.restype = ctypes.c_char_p
+        L.jv_version.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().jv_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return lib().jv_version().decode()
+
+
+def launch_count() -> int:
+    return int(lib().jv_launch_count())
+
+
+def set_force_generic(on: bool) -> bool:
+    return bool(lib().jv_set_force_generic(1 if on else 0))
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return JV_F32
+    if t.dtype == torch.bfloat16:
+        return JV_BF16
+    raise TypeError(f"dtype {t.dtype}: the mixers take float32 or bfloat16")
+
+
+def make_shape(t: torch.Tensor, Hg: int, Wg: int) -> JvShape:
+    B, H, N, D = t.shape
+    if N != Hg * Wg:
+        raise ValueError(f"N = {N} is not Hg*Wg = {Hg}*{Wg}")
+    return JvShape(B, H, Hg, Wg, D, _dtype_code(t))
+
+
+def _check_tensors(*ts: torch.Tensor):
+    ref = ts[0]
+    for t in ts:
+        if not t.is_cuda:
+            raise ValueError("tensors must live on a CUDA device (there is no CPU path)")
+        if not t.is_contiguous() or t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device:
+            raise ValueError("q, k, v, o must be contiguous [B,H,N,D] tensors of one shape, dtype and device")
+
+
+def make_dwc(d: Optional[dict], device) -> Optional[JvDwc]:
+    """dict(k, R, W1, b1, W2, b2) of fp32 CUDA tensors -> jv_dwc.  The dict must stay
+    alive until the call has been enqueued."""
+    if d is None:
+        return None
+    for key in ("W1", "W2"):
+        t = d[key]
+        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise ValueError(f"dwc[{key!r}] must be a contiguous fp32 CUDA tensor")
+    ptr = lambda t: None if t is None else t.data_ptr()
+    return JvDwc(int(d["k"]), int(d["R"]), ptr(d["W1"]), ptr(d.get("b1")), ptr(d["W2"]), ptr(d.get("b2")))
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def workspace_bytes(mixer: str, shape: JvShape, dwc: Optional[JvDwc] = None) -> int:
+    return int(lib().jv_workspace_bytes(mixer.encode()[:1], ctypes.byref(shape),
+                                        ctypes.byref(dwc) if dwc is not None else None))
+
+
+def alloc_workspace(mixer: str, shape: JvShape, dwc: Optional[JvDwc], device) -> Optional[torch.Tensor]:
+    n = workspace_bytes(mixer, shape, dwc)
+    return torch.empty(max(n, 256), dtype=torch.uint8, device=device) if n else None
+
+
+def _ws_args(ws: Optional[torch.Tensor]):
+    return (None, 0) if ws is None else (ws.data_ptr(), ws.numel() * ws.element_size())
+
+
+def _raise(status: int, where: str):
+    if status != JV_OK:
+        raise JetVitError(status, where)
+
+
+def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict] = None, out=None,
+                ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """jv_linear_attn.  Allocates ``out`` / ``ws`` with torch when not given."""
+    out = torch.empty_like(q) if out is None else out
+    _check_tensors(q, k, v, out)
+    shape = make_shape(q, Hg, Wg)
+    d = make_dwc(dwc, q.device)
+    with torch.cuda.device(q.device):
+        if ws is None:
+            ws = alloc_workspace("L", shape, d, q.device)
+        wp, wn = _ws_args(ws)
+        st = lib().jv_linear_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
+                                  float(eps), ctypes.byref(d) if d is not None else None, wp, wn, _stream(stream))
+    _raise(st, "jv_linear_attn")
+    return out
+
+
+def window_attn(q, k, v, Hg: int, Wg: int, win_h: int, win_w: int, scale: float = 0.0, out=None,
+                stream=None) -> torch.Tensor:
+    """jv_window_attn (scale <= 0: 1/sqrt(D))."""
+    out = torch.empty_like(q) if out is None else out
+    _check_tensors(q, k, v, out)
+    shape = make_shape(q, Hg, Wg)
+    with torch.cuda.device(q.device):
+        st = lib().jv_window_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
+                                  int(win_h), int(win_w), float(scale), None, 0, _stream(stream))
+    _raise(st, "jv_window_attn")
+    return out
+
+
+def full_attn(q, k, v, Hg: Optional[int] = None, Wg: Optional[int] = None, scale: float = 0.0, out=None,
+              stream=None) -> torch.Tensor:
+    """jv_full_attn (scale <= 0: 1/sqrt(D)).  The grid split of N is irrelevant to F."""
+    out = torch.empty_like(q) if out is None else out
+    _check_tensors(q, k, v, out)
+    if Hg is None or Wg is None:
+        Hg, Wg = 1, q.shape[2]
+    shape = make_shape(q, Hg, Wg)
+    with torch.cuda.device(q.device):
+        st = lib().jv_full_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
+                                float(scale), None, 0, _stream(stream))
+    _raise(st, "jv_full_attn")
+    return out
+
+
+def hybrid_mixers(schedule: str, q: Sequence[torch.Tensor], k, v, Hg: int, Wg: int, win_h: int, win_w: int,
+                  scale: float = 0.0, eps: float = 1e-6, dwc: Optional[Sequence[Optional[dict]]] = None,
+                  out: Optional[Sequence[torch.Tensor]] = None, ws: Optional[torch.Tensor] = None, stream=None):
+    """jv_hybrid_mixers: one mixer per layer, schedule[l] in 'L', 'W', 'F'."""
+    n = len(schedule)
+    if not (len(q) == len(k) == len(v) == n):
+        raise ValueError("need one q, k, v per schedule entry")
+    out = [torch.empty_like(t) for t in q] if out is None else list(out)
+    for l in range(n):
+        _check_tensors(q[l], k[l], v[l], out[l])
+        if q[l].shape != q[0].shape or q[l].dtype != q[0].dtype:
+            raise ValueError("all layers share one shape and dtype")
+    shape = make_shape(q[0], Hg, Wg)
+    arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
+    dstructs = [make_dwc(d, q[0].device) for d in dwc] if dwc is not None else None
+    dptr = None
+    if dstructs is not None:
+        dptr = (ctypes.POINTER(JvDwc) * n)(*[ctypes.pointer(d) if d is not None else ctypes.POINTER(JvDwc)()
+                                             for d in dstructs])
+    with torch.cuda.device(q[0].device):
+        if ws is None:
+            need = 0
+            for l, m in enumerate(schedule):
+                if m == "L":
+                    need = max(need, workspace_bytes("L", shape, dstructs[l] if dstructs else None))
+            ws = torch.empty(max(need, 256), dtype=torch.uint8, device=q[0].device) if need else None
+        wp, wn = _ws_args(ws)
+        st = lib().jv_hybrid_mixers(n, schedule.encode(), arr(q), arr(k), arr(v), arr(out), ctypes.byref(shape),
+                                    int(win_h), int(win_w), float(scale), float(eps), dptr, wp, wn, _stream(stream))
+    _raise(st, "jv_hybrid_mixers")
+    return out
+
+
+def device_status(stream=None) -> int:
+    """jv_device_status: synchronises the stream and returns the sticky status."""
+    return int(lib().jv_device_status(_stream(stream)))

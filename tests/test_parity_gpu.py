@@ -1,0 +1,256 @@
+"""GPU parity: the CUDA mixers (through the C ABI binding) against the float64
+CPU oracle on the same seeded inputs.  Bar: max-abs error / rms(oracle) <= 1e-4
+for fp32 tensors, <= 2e-2 for bf16 tensors with fp32 accumulation."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_26636_b200 import inputs
+from tests._util import TOL, dwc_to_device, guarded_empty, rel_err, sample_heads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def jv():
+    from paper_2605_26636_b200 import jetvit
+    jetvit.lib()
+    assert torch.cuda.is_available()
+    yield jetvit
+    assert jetvit.device_status() == jetvit.JV_OK
+
+
+@pytest.fixture(params=[False, True], ids=["fast", "generic"])
+def both_paths(request, jv):
+    prev = jv.set_force_generic(request.param)
+    yield request.param
+    jv.set_force_generic(prev)
+
+
+DEV = "cuda:0"
+
+
+def _dev(ts):
+    return tuple(t.to(DEV) for t in ts)
+
+
+# ------------------------------------------------------------------ config 1: tiny, fp32
+def test_tiny_fp32_all_mixers(jv, oracle, both_paths):
+    w = inputs.WORKLOADS["tiny"]
+    q, k, v = inputs.qkv(w)
+    dq, dk, dv = _dev((q, k, v))
+    assert rel_err(jv.linear_attn(dq, dk, dv, w.Hg, w.Wg), oracle.linear_attn(q, k, v, w.Hg, w.Wg)) <= TOL["f32"]
+    assert rel_err(jv.window_attn(dq, dk, dv, w.Hg, w.Wg, 8, 8),
+                   oracle.window_attn(q, k, v, w.Hg, w.Wg, 8, 8)) <= TOL["f32"]
+    assert rel_err(jv.full_attn(dq, dk, dv), oracle.full_attn(q, k, v)) <= TOL["f32"]
+    # one window covering the grid is full attention
+    assert rel_err(jv.window_attn(dq, dk, dv, w.Hg, w.Wg, 16, 16), oracle.full_attn(q, k, v)) <= TOL["f32"]
+    assert rel_err(jv.window_attn(dq, dk, dv, w.Hg, w.Wg, 64, 64), oracle.full_attn(q, k, v)) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("ksz", [3, 5])
+def test_tiny_fp32_linear_with_squeeze_dynamic_dwc(jv, oracle, both_paths, ksz):
+    w = inputs.WORKLOADS["tiny"]
+    q, k, v = inputs.qkv(w)
+    C = w.H * w.D
+    d = inputs.dwc_weights(C, C // 8, ksz, inputs.seed_for(w.cfg, 0, 3))
+    ref = oracle.linear_attn(q, k, v, w.Hg, w.Wg, dwc=d)
+    out = jv.linear_attn(*_dev((q, k, v)), w.Hg, w.Wg, dwc=dwc_to_device(d, DEV))
+    assert rel_err(out, ref) <= TOL["f32"]
+    # without biases
+    d2 = dict(d, b1=None, b2=None)
+    ref = oracle.linear_attn(q, k, v, w.Hg, w.Wg, dwc=d2)
+    out = jv.linear_attn(*_dev((q, k, v)), w.Hg, w.Wg, dwc=dwc_to_device(d2, DEV))
+    assert rel_err(out, ref) <= TOL["f32"]
+
+
+# ------------------------------------------------------------------ shape sweep with canaries
+SWEEP = [  # B, H, Hg, Wg, D, win_h, win_w
+    (1, 1, 7, 5, 64, 4, 4),
+    (2, 3, 17, 33, 64, 16, 16),
+    (1, 2, 73, 73, 64, 16, 16),
+    (2, 2, 16, 48, 64, 16, 16),
+    (1, 2, 40, 24, 64, 8, 16),
+    (1, 2, 9, 9, 32, 3, 5),
+    (1, 1, 12, 20, 128, 8, 8),
+    (3, 1, 1, 1, 64, 1, 1),
+    (1, 2, 33, 16, 64, 16, 16),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", SWEEP, ids=lambda c: "x".join(map(str, c)))
+def test_shape_sweep(jv, oracle, both_paths, case, dtype):
+    B, H, Hg, Wg, D, wh, ww = case
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, D, dtype, seed=Hg * 100 + Wg)
+    dq, dk, dv = _dev((q, k, v))
+    tol = TOL[dtype]
+    for name in ("L", "W", "F"):
+        out, check = guarded_empty(q.shape, dq.dtype, DEV)
+        if name == "L":
+            jv.linear_attn(dq, dk, dv, Hg, Wg, out=out)
+            ref = oracle.linear_attn(q, k, v, Hg, Wg)
+        elif name == "W":
+            jv.window_attn(dq, dk, dv, Hg, Wg, wh, ww, out=out)
+            ref = oracle.window_attn(q, k, v, Hg, Wg, wh, ww)
+        else:
+            jv.full_attn(dq, dk, dv, Hg, Wg, out=out)
+            ref = oracle.full_attn(q, k, v)
+        check()
+        assert rel_err(out, ref) <= tol, f"{name} {case} {dtype}"
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sweep_linear_dwc_ragged(jv, oracle, both_paths, dtype):
+    B, H, Hg, Wg, D = 2, 2, 19, 13, 64
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, D, dtype, seed=5)
+    d = inputs.dwc_weights(H * D, 16, 3, 99)
+    out, check = guarded_empty(q.shape, _dev((q,))[0].dtype, DEV)
+    jv.linear_attn(*_dev((q, k, v)), Hg, Wg, dwc=dwc_to_device(d, DEV), out=out)
+    check()
+    assert rel_err(out, oracle.linear_attn(q, k, v, Hg, Wg, dwc=d)) <= TOL[dtype]
+
+
+def test_explicit_scale_and_eps(jv, oracle, both_paths):
+    q, k, v = inputs.custom_qkv(1, 2, 16 * 16, 64, "bf16", seed=8)
+    dq, dk, dv = _dev((q, k, v))
+    assert rel_err(jv.full_attn(dq, dk, dv, scale=0.3), oracle.full_attn(q, k, v, scale=0.3)) <= TOL["bf16"]
+    assert rel_err(jv.window_attn(dq, dk, dv, 16, 16, 16, 16, scale=0.05),
+                   oracle.window_attn(q, k, v, 16, 16, 16, 16, scale=0.05)) <= TOL["bf16"]
+    assert rel_err(jv.linear_attn(dq, dk, dv, 16, 16, eps=50.0),
+                   oracle.linear_attn(q, k, v, 16, 16, eps=50.0)) <= TOL["bf16"]
+
+
+def test_degenerate_inputs(jv, oracle, both_paths):
+    """All-negative q in L gives exactly 0; large logits do not overflow in F / W."""
+    q, k, v = inputs.custom_qkv(1, 2, 16 * 16, 64, "bf16", seed=9)
+    qn = -q.abs()
+    out = jv.linear_attn(*_dev((qn, k, v)), 16, 16)
+    assert float(out.abs().max()) == 0.0
+    qb, kb = q * 12, k * 12          # logits of a few hundred: softmax is nearly one-hot
+    dq, dk, dv = _dev((qb, kb, v))
+    assert rel_err(jv.full_attn(dq, dk, dv), oracle.full_attn(qb, kb, v)) <= TOL["bf16"]
+    assert rel_err(jv.window_attn(dq, dk, dv, 16, 16, 16, 16), oracle.window_attn(qb, kb, v, 16, 16, 16, 16)) <= TOL["bf16"]
+
+
+def test_bit_determinism(jv):
+    w = inputs.WORKLOADS["dinov3_l"]
+    q, k, v = _dev(inputs.custom_qkv(2, 4, 64 * 64, 64, "bf16", seed=3))
+    d = dwc_to_device(inputs.dwc_weights(4 * 64, 32, 3, 7), DEV)
+    for fn in (lambda: jv.linear_attn(q, k, v, 64, 64, dwc=d), lambda: jv.window_attn(q, k, v, 64, 64, 16, 16),
+               lambda: jv.full_attn(q, k, v)):
+        a, b = fn(), fn()
+        torch.cuda.synchronize()
+        assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ configs 2-5 at full size
+def test_cfg2_linear_dinov3_full_size(jv, oracle):
+    w = inputs.WORKLOADS["dinov3_l"]
+    q, k, v = inputs.qkv(w)
+    out = jv.linear_attn(*_dev((q, k, v)), w.Hg, w.Wg)
+    torch.cuda.synchronize()
+    assert rel_err(out, oracle.linear_attn(q, k, v, w.Hg, w.Wg)) <= TOL["bf16"]
+
+
+def test_cfg2d_linear_with_dwc_full_size(jv, oracle):
+    w = inputs.WORKLOADS["dinov3_l"]
+    q, k, v = inputs.qkv(w)
+    C = w.H * w.D
+    d = inputs.dwc_weights(C, C // 8, 3, inputs.seed_for(w.cfg, 0, 3))
+    out = jv.linear_attn(*_dev((q, k, v)), w.Hg, w.Wg, dwc=dwc_to_device(d, DEV))
+    torch.cuda.synchronize()
+    assert rel_err(out, oracle.linear_attn(q, k, v, w.Hg, w.Wg, dwc=d)) <= TOL["bf16"]
+
+
+def test_cfg3_window_dinov3_full_size_sampled_heads(jv, oracle):
+    w = inputs.WORKLOADS["dinov3_w"]
+    q, k, v = inputs.qkv(w)
+    out = jv.window_attn(*_dev((q, k, v)), w.Hg, w.Wg, 16, 16).cpu()
+    for b, h in sample_heads(w.B, w.H, 12, 3):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        ref = oracle.window_attn(q[sl], k[sl], v[sl], w.Hg, w.Wg, 16, 16)
+        assert rel_err(out[sl], ref) <= TOL["bf16"], (b, h)
+
+
+def _sample_rows(N, n, seed, tail=160):
+    rng = np.random.default_rng(seed)
+    rows = set(rng.choice(N, size=n, replace=False).tolist())
+    rows.update(range(max(0, N - tail), N, 7))      # always cover the ragged last tile
+    rows.update((0, N - 1))
+    return np.array(sorted(rows))
+
+
+def test_cfg4_dav2_ragged_full_and_window(jv, oracle):
+    w = inputs.WORKLOADS["dav2_l"]
+    q, k, v = inputs.qkv(w)
+    dq, dk, dv = _dev((q, k, v))
+    of = jv.full_attn(dq, dk, dv, w.Hg, w.Wg).cpu()
+    ow = jv.window_attn(dq, dk, dv, w.Hg, w.Wg, 16, 16).cpu()
+    rows = _sample_rows(w.N, 192, 4)
+    for b, h in sample_heads(w.B, w.H, 6, 4):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        ref = oracle.full_attn(q[sl][:, :, rows], k[sl], v[sl])
+        assert rel_err(of[sl][:, :, rows], ref) <= TOL["bf16"], ("F", b, h)
+        ref = oracle.window_attn(q[sl], k[sl], v[sl], w.Hg, w.Wg, 16, 16)
+        assert rel_err(ow[sl], ref) <= TOL["bf16"], ("W", b, h)
+
+
+def test_cfg5_hybrid_stack_and_all_full(jv, oracle):
+    w = inputs.WORKLOADS["hybrid24"]
+    sched = inputs.HYBRID_SCHEDULE
+    assert len(sched) == w.n_layers and [i for i, c in enumerate(sched) if c == "F"] == [5, 11, 17, 23]
+    host = [inputs.qkv(w, layer=l) for l in range(w.n_layers)]
+    dq, dk, dv = ([t[i].to(DEV) for t in host] for i in range(3))
+    outs = jv.hybrid_mixers(sched, dq, dk, dv, w.Hg, w.Wg, 16, 16)
+    torch.cuda.synchronize()
+    rows = _sample_rows(w.N, 96, 5, tail=0)
+    for l, m in enumerate(sched):
+        q, k, v = host[l]
+        o = outs[l].cpu()
+        for b, h in sample_heads(w.B, w.H, 2, 50 + l):
+            sl = (slice(b, b + 1), slice(h, h + 1))
+            if m == "L":
+                err = rel_err(o[sl], oracle.linear_attn(q[sl], k[sl], v[sl], w.Hg, w.Wg))
+            elif m == "W":
+                err = rel_err(o[sl], oracle.window_attn(q[sl], k[sl], v[sl], w.Hg, w.Wg, 16, 16))
+            else:
+                err = rel_err(o[sl][:, :, rows], oracle.full_attn(q[sl][:, :, rows], k[sl], v[sl]))
+            assert err <= TOL["bf16"], (l, m, b, h, err)
+    del outs
+    # the comparison run: the same stack with every layer F
+    outs = jv.hybrid_mixers("F" * w.n_layers, dq, dk, dv, w.Hg, w.Wg, 16, 16)
+    torch.cuda.synchronize()
+    rows = rows[::3]
+    for l in range(0, w.n_layers, 5):
+        q, k, v = host[l]
+        o = outs[l].cpu()
+        b, h = sample_heads(w.B, w.H, 1, 80 + l)[0]
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        assert rel_err(o[sl][:, :, rows], oracle.full_attn(q[sl][:, :, rows], k[sl], v[sl])) <= TOL["bf16"], l
+
+
+def test_hybrid_small_with_dwc_layers(jv, oracle, both_paths):
+    B, H, Hg, Wg, D = 1, 2, 32, 32, 64
+    sched = "LWFL"
+    host = [inputs.custom_qkv(B, H, Hg * Wg, D, "bf16", seed=20 + l) for l in range(4)]
+    dws = [inputs.dwc_weights(H * D, 16, 3, 5), None, None, None]
+    dq, dk, dv = ([t[i].to(DEV) for t in host] for i in range(3))
+    outs = jv.hybrid_mixers(sched, dq, dk, dv, Hg, Wg, 16, 16,
+                            dwc=[None if d is None else dwc_to_device(d, DEV) for d in dws])
+    refs = oracle.hybrid_mixers(sched, [t[0] for t in host], [t[1] for t in host], [t[2] for t in host],
+                                Hg, Wg, 16, 16, dwc=dws)
+    for l in range(4):
+        assert rel_err(outs[l], refs[l]) <= TOL["bf16"], l
+
+
+def test_runtime_errors_on_device(jv):
+    q, k, v = _dev(inputs.custom_qkv(1, 2, 64, 64, "f32", seed=1))
+    with pytest.raises(jv.JetVitError) as e:
+        jv.linear_attn(q, k, v, 8, 8, ws=torch.empty(256, dtype=torch.uint8, device=DEV))
+    assert e.value.status == jv.JV_ERR_WORKSPACE
+    with pytest.raises(jv.JetVitError):
+        jv.window_attn(q, k, v, 8, 8, 0, 4)
+    with pytest.raises(jv.JetVitError):
+        jv.full_attn(q, k, v, out=q)
+    assert jv.device_status() == jv.JV_OK
