@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the JetViT token mixers on B200.
+
+One "step" is one pass of the whole hot path at the DINOv3-L high-resolution
+shape (B=8, heads=16, 64x64 token grid, head_dim 64, bf16): jv_hybrid_mixers with
+schedule "LWF" over three layers of fresh synthetic Q/K/V -- the linear-attention
+block (with its squeeze dynamic convolution), 16x16 window attention and full
+attention.  `value` is mixer tokens/s (layers x B x N per step) with inputs
+resident in HBM; `e2e` is the same step with host buffers (pinned), host<->device
+copies inside the timed region.  Each mixer is also timed on its own (tokens/s,
+achieved GB/s or TFLOP/s against the measured peaks), and the 24-layer 128x128
+hybrid stack is timed against the same stack run all-F.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Under torchrun (N > 1) every rank runs the same per-GPU workload on its own GPU
+(the path shards over independent (batch, head) units: no data-path collective).
+`--impl reference` times the float64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2605_26636_b200 import inputs
+
+METRIC = "mixer tokens/sec (L+W+F stack at ViT-L shapes)"
+UNIT = "tokens/s"
+STEP_SCHEDULE = "LWF"
+WIN = 16
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- algorithmic work
+def alg_bytes(B, H, N, D, esz=2, dwc=False):
+    """Q, K, V read once, O written once (V read twice with the convolution)."""
+    return B * H * N * D * esz * (5 if dwc else 4)
+
+
+def alg_flops_attn(B, H, Hg, Wg, D, wh, ww):
+    """2 flops per MAC over valid (query, key) pairs only, QK^T and PV."""
+    pairs = 0
+    for y0 in range(0, Hg, wh):
+        for x0 in range(0, Wg, ww):
+            n = min(wh, Hg - y0) * min(ww, Wg - x0)
+            pairs += n * n
+    return 4 * D * pairs * B * H
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            f = [x.strip() for x in s.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = max(mx, float(f[1]))
+            except ValueError:
+                continue
+            for n, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- timing helpers
+def time_calls(fn, steps, warmup, stream):
+    """Device time per call (ms): CUDA events on the launching stream around `steps` calls."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        fn(warmup + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ----------------------------------------------------------------------------- oracle legs
+def oracle_sample_step(w, scale=1.0):
+    """A bounded sample of one step for the CPU oracle (about 10 s on 8 cores at
+    scale 1): L with the dynamic convolution and W on ceil(scale * B) batch samples,
+    F on all query rows of round(32 * scale) of the B*H (batch, head) pairs; each
+    mixer's time is extrapolated to the whole step by its sampled fraction.
+    Returns (seconds spent, extrapolated seconds of a whole step, description,
+    threads used)."""
+    from oracle import jv_oracle
+    C = w.H * w.D
+    d = inputs.dwc_weights(C, C // 8, 3, inputs.seed_for(w.cfg, 0, 3))
+    nB = max(1, min(w.B, int(np.ceil(scale * w.B))))
+    q, k, v = inputs.qkv(w, layer=0, shape=(nB, w.H, w.N, w.D))
+    t0 = time.perf_counter()
+    jv_oracle.linear_attn(q, k, v, w.Hg, w.Wg, dwc=d)
+    tL = time.perf_counter() - t0
+    q, k, v = inputs.qkv(w, layer=1, shape=(nB, w.H, w.N, w.D))
+    t0 = time.perf_counter()
+    jv_oracle.window_attn(q, k, v, w.Hg, w.Wg, WIN, WIN)
+    tW = time.perf_counter() - t0
+    nF = max(1, min(w.B * w.H, int(round(32 * scale))))
+    q, k, v = inputs.qkv(w, layer=2, shape=(1, nF, w.N, w.D))
+    t0 = time.perf_counter()
+    jv_oracle.full_attn(q, k, v)
+    tF = time.perf_counter() - t0
+    full_step_s = (tL + tW) * w.B / nB + tF * (w.B * w.H) / nF
+    desc = (f"L+DWC on {nB}/{w.B} of the batch ({tL:.2f}s), W on {nB}/{w.B} of the batch ({tW:.2f}s), "
+            f"F on {nF} of {w.B * w.H} (batch, head) pairs ({tF:.2f}s); each extrapolated by its fraction")
+    return tL + tW + tF, full_step_s, desc, jv_oracle.num_threads()
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    w = inputs.WORKLOADS["dinov3_l"]
+    step_tokens = len(STEP_SCHEDULE) * w.tokens
+    # size the per-step sample so that the whole run stays near two minutes
+    n_warm = min(args.warmup, 1)
+    scale = min(1.0, 120.0 / (10.5 * (args.steps + n_warm)))
+    for _ in range(n_warm):
+        oracle_sample_step(w, scale)
+    spent, full = [], []
+    for _ in range(args.steps):
+        s, f, desc, cores = oracle_sample_step(w, scale)
+        spent.append(s)
+        full.append(f)
+    step_s = float(np.mean(full))
+    value = step_tokens / step_s
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "dinov3_l 64x64 grid B=8 H=16 D=64, schedule LWF (CPU oracle, sampled)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+def run_cuda(args):
+    from paper_2605_26636_b200 import jetvit as jv
+    rank, world, local = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    jv.lib()
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+    w = inputs.WORKLOADS["dinov3_l"]
+    nL = len(STEP_SCHEDULE)
+    C = w.H * w.D
+
+    # ---- inputs: three layers of Q/K/V in pinned host memory and on the device
+    host = [[t.pin_memory() for t in inputs.qkv(w, layer=100 * rank + l)] for l in range(nL)]
+    dq, dk, dv = ([host[l][i].to(dev, non_blocking=True) for l in range(nL)] for i in range(3))
+    outs = [torch.empty_like(t) for t in dq]
+    host_out = [torch.empty(w.shape, dtype=torch.bfloat16).pin_memory() for _ in range(nL)]
+    dwc_host = inputs.dwc_weights(C, C // 8, 3, inputs.seed_for(w.cfg, 0, 3))
+    dwc_dev = {k: (v.to(dev) if hasattr(v, "to") else v) for k, v in dwc_host.items()}
+    dwcs = [dwc_dev if m == "L" else None for m in STEP_SCHEDULE]
+    shape = jv.make_shape(dq[0], w.Hg, w.Wg)
+    ws = jv.alloc_workspace("S", shape, jv.make_dwc(dwc_dev, dev), dev)
+    torch.cuda.synchronize()
+
+    def step(_i=0):
+        jv.hybrid_mixers(STEP_SCHEDULE, dq, dk, dv, w.Hg, w.Wg, WIN, WIN, dwc=dwcs, out=outs, ws=ws)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- the timed region: exactly K steps between barrier + synchronize
+    for i in range(args.warmup):
+        step()
+    barrier()
+    l0 = jv.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        e0.record(stream)
+        for i in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+    launches = jv.launch_count() - l0
+    ms = e0.elapsed_time(e1) / args.steps
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    assert jv.device_status() == jv.JV_OK, "a kernel reported a timeout"
+    step_tokens = nL * w.tokens
+    value = world * step_tokens / (ms * 1e-3)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    def e2e_step(_i=0):
+        for l in range(nL):
+            for i, dst in enumerate((dq, dk, dv)):
+                dst[l].copy_(host[l][i], non_blocking=True)
+        step()
+        for l in range(nL):
+            host_out[l].copy_(outs[l], non_blocking=True)
+    n_e2e = max(2, min(args.steps, 5))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0.record(stream)
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / n_e2e
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    tensor_bytes = int(np.prod(w.shape)) * 2
+    e2e = {"value": world * step_tokens / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+           "h2d_bytes_per_step": 3 * nL * tensor_bytes, "d2h_bytes_per_step": nL * tensor_bytes}
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- per-mixer timings (rank 0; rotating over the three layers' tensors: 805 MB > L2)
+    per = {}
+    K, W = max(args.steps, 10), max(args.warmup, 3)
+    hbm, tf = peaks["hbm_gbs"], peaks["bf16_tflops"]
+
+    def add(name, fn, bytes_, flops, bound):
+        t_ms = time_calls(fn, K, W, stream)
+        gbs, tfl = bytes_ / t_ms / 1e6, flops / t_ms / 1e9
+        per[name] = {"ms": t_ms, "tokens_per_s": w.tokens / (t_ms * 1e-3), "GBps": gbs, "TFLOPs": tfl,
+                     "frac_hbm": gbs / hbm, "frac_tensor": tfl / tf, "bound": bound}
+
+    r = lambda i: i % nL
+    add("L", lambda i: jv.linear_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, out=outs[r(i)], ws=ws),
+        alg_bytes(*w.shape), 0.0, "hbm")
+    add("L+dwc", lambda i: jv.linear_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, dwc=dwc_dev, out=outs[r(i)], ws=ws),
+        alg_bytes(*w.shape, dwc=True), 0.0, "hbm")
+    add("W", lambda i: jv.window_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, WIN, WIN, out=outs[r(i)]),
+        alg_bytes(*w.shape), alg_flops_attn(w.B, w.H, w.Hg, w.Wg, w.D, WIN, WIN), "hbm")
+    f_flops = alg_flops_attn(w.B, w.H, w.Hg, w.Wg, w.D, w.Hg, w.Wg)
+    add("F", lambda i: jv.full_attn(dq[r(i)], dk[r(i)], dv[r(i)], out=outs[r(i)]),
+        alg_bytes(*w.shape), f_flops, "tensor")
+
+    # ragged DepthAnythingV2-L grid (73x73, B=4): F and W with masked edge windows
+    w4 = inputs.WORKLOADS["dav2_l"]
+    q4 = [[t.to(dev) for t in inputs.qkv(w4, layer=l)] for l in range(3)]
+    o4 = [torch.empty_like(q4[0][0]) for _ in range(3)]
+
+    def add4(name, fn, bytes_, flops, bound):
+        t_ms = time_calls(fn, K, W, stream)
+        per[name] = {"ms": t_ms, "tokens_per_s": w4.tokens / (t_ms * 1e-3), "GBps": bytes_ / t_ms / 1e6,
+                     "TFLOPs": flops / t_ms / 1e9, "frac_hbm": bytes_ / t_ms / 1e6 / hbm,
+                     "frac_tensor": flops / t_ms / 1e9 / tf, "bound": bound}
+    add4("F@dav2_73x73", lambda i: jv.full_attn(*q4[r(i)], out=o4[r(i)]),
+         alg_bytes(*w4.shape), alg_flops_attn(w4.B, w4.H, w4.Hg, w4.Wg, w4.D, w4.Hg, w4.Wg), "tensor")
+    add4("W@dav2_73x73", lambda i: jv.window_attn(*q4[r(i)], w4.Hg, w4.Wg, WIN, WIN, out=o4[r(i)]),
+         alg_bytes(*w4.shape), alg_flops_attn(w4.B, w4.H, w4.Hg, w4.Wg, w4.D, WIN, WIN), "hbm")
+    del q4, o4
+
+    # 24-layer hybrid stack at 128x128 against the same stack run all-F
+    w5 = inputs.WORKLOADS["hybrid24"]
+    base = [t.to(dev) for t in inputs.qkv(w5, layer=0)]
+    q5 = [[torch.roll(t, l, dims=2) if l else t for t in base] for l in range(4)]   # 4 distinct layer inputs
+    lq, lk, lv = ([q5[l % 4][i] for l in range(w5.n_layers)] for i in range(3))
+    lo = [torch.empty_like(base[0]) for _ in range(4)]
+    louts = [lo[l % 4] for l in range(w5.n_layers)]
+    ws5 = jv.alloc_workspace("S", jv.make_shape(base[0], w5.Hg, w5.Wg), None, dev)
+    hyb = time_calls(lambda i: jv.hybrid_mixers(inputs.HYBRID_SCHEDULE, lq, lk, lv, w5.Hg, w5.Wg, WIN, WIN,
+                                                out=louts, ws=ws5), 3, 2, stream)
+    allf = time_calls(lambda i: jv.hybrid_mixers("F" * w5.n_layers, lq, lk, lv, w5.Hg, w5.Wg, WIN, WIN,
+                                                 out=louts, ws=ws5), 2, 1, stream)
+    f5_flops = alg_flops_attn(w5.B, w5.H, w5.Hg, w5.Wg, w5.D, w5.Hg, w5.Wg)
+    hybrid = {"schedule": inputs.HYBRID_SCHEDULE, "hybrid_ms": hyb, "all_full_ms": allf, "speedup": allf / hyb,
+              "tokens_per_s_hybrid": w5.n_layers * w5.tokens / (hyb * 1e-3),
+              "all_full_TFLOPs": w5.n_layers * f5_flops / allf / 1e9,
+              "note": "4 distinct layer inputs reused round-robin over the 24 layers (134 MB each: larger than L2)"}
+    del q5, lo, base
+    assert jv.device_status() == jv.JV_OK, "a kernel reported a timeout"
+
+    # ---- roofline of the dominant kernel of the step (full attention)
+    dom = per["F"]
+    roofline = {"kernel": "full attention (jv_full_attn)", "bound": "tensor", "achieved": dom["TFLOPs"],
+                "peak": tf, "unit": "TFLOP/s", "frac": dom["TFLOPs"] / tf, "traffic": None,
+                "peak_source": peaks["source"] + " bf16 burst",
+                "linear": {"bound": "hbm", "achieved": per["L"]["GBps"], "peak": hbm, "unit": "GB/s",
+                           "frac": per["L"]["GBps"] / hbm},
+                "window": {"bound": "hbm", "achieved": per["W"]["GBps"], "peak": hbm, "unit": "GB/s",
+                           "frac": per["W"]["GBps"] / hbm, "tensor_frac": per["W"]["TFLOPs"] / tf}}
+
+    # ---- CPU baseline: the oracle, as it stands, on a bounded sample
+    cpu = None
+    if not args.no_cpu_baseline:
+        spent, full_s, desc, cores = oracle_sample_step(w)
+        cpu = {"value": step_tokens / full_s, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+               "seconds_spent": spent}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "dinov3_l: 64x64 token grid (1024x1024 px, patch 16), B=8, H=16, D=64, bf16; "
+                                   "one step = jv_hybrid_mixers('LWF'): L with squeeze dynamic DWC (k=3, R=128), "
+                                   "W 16x16, F", "l2": "three layers' tensors (805 MB) exceed L2; "
+                                   "per-mixer loops rotate over three tensor sets"},
+            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu, "per_mixer": per, "hybrid24": hybrid,
+            "peaks": peaks}
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

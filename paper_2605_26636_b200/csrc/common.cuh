@@ -76,7 +76,11 @@ struct LinArgs {
 cudaError_t launch_linear_generic(const LinArgs& a, const LinPlan& p, cudaStream_t st);
 bool linear_fast_supported(const LinArgs& a);
 cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t st);
-// shared by both linear paths: hidden = SiLU(W1 s + b1), w = W2 hidden + b2
-cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, cudaStream_t st);
+// shared by both linear paths: hidden = SiLU(W1 s + b1), w = W2 hidden + b2, with
+// s = vsum / N read from vsum[bh * bh_stride + e]
+cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float* vsum, int bh_stride,
+                                 cudaStream_t st);
+cudaError_t launch_lin_reduce(const float* partial, float* state, int nchunk, int state_elems, size_t total,
+                              cudaStream_t st);
 
 }  // namespace jv

@@ -144,17 +144,19 @@ lin_apply_generic_kernel(const T* __restrict__ q, const T* __restrict__ v, T* __
 
 // ---- kernel generator of the squeeze dynamic convolution ---------------------
 // hidden[b][r] = SiLU(b1[r] + sum_c W1[r][c] * mean_v[b][c]); one warp per (b, r).
-__global__ void dwc_hidden_kernel(const float* __restrict__ state, const float* __restrict__ W1,
+// vsum points at the v-sum of (batch 0, head 0); consecutive (batch, head) pairs are
+// bh_stride floats apart.
+__global__ void dwc_hidden_kernel(const float* __restrict__ vsum, const float* __restrict__ W1,
                                   const float* __restrict__ b1, float* __restrict__ hidden,
-                                  int H, int D, int R, int state_elems, float inv_n) {
+                                  int H, int D, int R, int bh_stride, float inv_n) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y;
   if (warp >= R) return;
-  const int C = H * D, D1 = D + 1;
+  const int C = H * D;
   float s = 0.f;
   for (int c = lane; c < C; c += 32) {
     const int h = c / D, e = c % D;
-    const float mean = state[((size_t)b * H + h) * state_elems + D * D1 + e] * inv_n;   // v-sum row
+    const float mean = vsum[((size_t)b * H + h) * bh_stride + e] * inv_n;
     s = fmaf(__ldg(&W1[(size_t)warp * C + c]), mean, s);
   }
   s = warp_sum(s);
@@ -198,7 +200,7 @@ cudaError_t launch_generic_t(const LinArgs& a, const LinPlan& p, cudaStream_t st
   count_launch();
   const float* dw = nullptr;
   if (a.dwc) {
-    cudaError_t e = launch_dwc_generator(a, p, st);
+    cudaError_t e = launch_dwc_generator(a, p, state + s.D * p.D1, p.state_elems, st);
     if (e != cudaSuccess) return e;
     dw = (const float*)(ws + p.off_kernel);
   }
@@ -219,16 +221,16 @@ cudaError_t launch_lin_reduce(const float* partial, float* state, int nchunk, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, cudaStream_t st) {
+cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float* vsum, int bh_stride,
+                                 cudaStream_t st) {
   const jv_shape& s = a.s;
   const jv_dwc& d = *a.dwc;
   char* ws = (char*)a.ws;
-  const float* state = (const float*)(ws + p.off_state);
   float* hidden = (float*)(ws + p.off_hidden);
   float* w = (float*)(ws + p.off_kernel);
   const int N = s.Hg * s.Wg;
   dim3 g1(ceil_div(d.R * 32, 256), s.B);
-  dwc_hidden_kernel<<<g1, 256, 0, st>>>(state, d.W1, d.b1, hidden, s.H, s.D, d.R, p.state_elems, 1.f / (float)N);
+  dwc_hidden_kernel<<<g1, 256, 0, st>>>(vsum, d.W1, d.b1, hidden, s.H, s.D, d.R, bh_stride, 1.f / (float)N);
   count_launch();
   const int T = s.H * s.D * d.k * d.k;
   dwc_out_kernel<<<ceil_div(T * 32, 256), 256, 0, st>>>(hidden, d.W2, d.b2, w, s.B, T, d.R);
