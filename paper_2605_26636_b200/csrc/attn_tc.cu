@@ -1,7 +1,546 @@
-// tcgen05 / TMEM path of full and window attention (placeholder until the
-// kernel lands: reports "not supported" so the generic kernel runs).
+// Full (Eq. 1) and window (Sec. 3.2.2) softmax attention on the 5th-generation
+// tensor cores: tcgen05.mma with accumulators in tensor memory, operands staged by
+// TMA.  bf16 tensors, head_dim 64.
+//
+// One kernel serves both mixers.  The token grid is described to TMA as a 4-D tensor
+// (d, x, y, batch*head); a "tile" is a box of 128 tokens: 128 consecutive tokens for
+// F (x = token index, y = 0), ww x (128/ww) tokens of a window for W.  Keys outside
+// the grid arrive as zeros from TMA's out-of-bounds fill and are masked to -inf before
+// the softmax; query rows outside the grid / window are never stored.
+//
+// Per CTA: two 128-row query tiles (ping-pong) against all key tiles of their
+// window.  Warp roles:
+//   warp 0        TMA producer: Q tiles once, then K and V tiles through 3-stage rings
+//   warp 1        MMA issuer (one elected thread): S_t = Q_t K^T (SS, M128 N128 K64),
+//                 O_t += P_t V (A = P from tensor memory, B = V MN-major, M128 N64 K128)
+//   warps 4-7     softmax of query tile 0   } one thread per query row: fp32 online
+//   warps 8-11    softmax of query tile 1   } softmax (exp2 domain, lazy rescale),
+//                 P as bf16 back into tensor memory, final 1/l scaling and the store.
+// While one tile's softmax runs on the ALUs, the tensor pipe works on the other tile.
+//
+// Tensor memory (512 columns): S0 [0,128) S1 [128,256) O0 [256,320) O1 [320,384)
+// P0 [384,448) P1 [448,512).
+//
+// Every mbarrier wait is bounded: a wait that runs out sets the device status word,
+// raises a CTA-wide abort flag, and every role falls through to the common teardown
+// (tensor memory is always released).
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace jv {
-bool attn_tc_supported(const AttnArgs&, bool) { return false; }
-cudaError_t launch_attn_tc(const AttnArgs&, bool, int*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int kD = 64;
+constexpr int kTile = 128;                 // tokens per tile (MMA M and key-tile N)
+constexpr int kTileBytes = kTile * kD * 2; // 16 KB
+constexpr int kStages = 3;
+constexpr int kThreads = 384;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+struct TcParams {
+  __nv_bfloat16* o;
+  int* status;
+  int gridW, gridH;      // token grid as TMA sees it (F: N x 1)
+  int tokens_per_head;   // N
+  int win_w, win_h;      // window extent in (x, y) (F: N x 1)
+  int box_w, box_h;      // tile box: box_w * box_h == 128
+  int step_x, step_y;    // origin step from one tile of a window to the next
+  int nwx;               // windows per grid row
+  float scale_log2;      // softmax scale * log2(e)
+};
+
+// ---- shared-memory layout -------------------------------------------------------
+struct __align__(8) Barriers {
+  uint64_t q_full;
+  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t s_full[2], p_full[2], o_full[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  volatile uint32_t abort_flag;
+};
+constexpr size_t kSmemTiles = (2 + 2 * kStages) * (size_t)kTileBytes;          // Q0 Q1 K[3] V[3]
+constexpr size_t kSmemBytes = kSmemTiles + sizeof(Barriers) + 1024;            // + alignment slack
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (after flagging the status word and the CTA abort flag)
+// if the phase did not complete in time or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* b, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try(bar, parity)) return true;
+    if ((spin & 63u) == 63u) {
+      if (b->abort_flag) return false;
+      const unsigned long long now = globaltimer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) {
+        b->abort_flag = 1;
+        atomicOr(status, kStatusTimeout);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+// ---- tcgen05 wrappers -------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Shared-memory matrix descriptors (128-byte swizzle; 8-row groups 1024 bytes apart).
+//   K-major operand  ([rows][64 bf16], used for Q and K): advance 32 bytes per K step of 16.
+//   MN-major operand ([keys][64 bf16] used as B = V):      advance 2048 bytes per K step of 16 keys.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) /* LBO (unused) */ | (64ull << 32) /* SBO = 1024 B */ |
+         (1ull << 46) /* descriptor version */ | (2ull << 61) /* SWIZZLE_128B */;
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16.
+constexpr uint32_t idesc(uint32_t M, uint32_t N, uint32_t b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+constexpr uint32_t kIdescQK = idesc(kTile, kTile, 0);
+constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
+
+// ---- the kernel ------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+               const __grid_constant__ CUtensorMap mapV, const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
+  const uint32_t sQ = smem_u32(smem), sK = sQ + 2 * kTileBytes, sV = sK + kStages * kTileBytes;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.z;
+  const int wy = blockIdx.y / p.nwx, wx = blockIdx.y % p.nwx;
+  const int x0 = wx * p.win_w, y0 = wy * p.win_h;
+  const int x_end = min(x0 + p.win_w, p.gridW), y_end = min(y0 + p.win_h, p.gridH);
+  // key tiles of this window, and the two query tiles of this CTA
+  const int ntiles = p.step_x ? (x_end - x0 + kTile - 1) / kTile : (y_end - y0 + p.box_h - 1) / p.box_h;
+  const int qt0 = 2 * blockIdx.x;
+  if (qt0 >= ntiles) return;   // uniform: nothing of this window left for this CTA
+
+  // Once any CTA has flagged a timeout the rest of the grid (and later launches, until the
+  // host reads the status) leave at once instead of each running into the same limit.
+  if (threadIdx.x == 0) bar->tmem_base = *reinterpret_cast<volatile int*>(p.status);
+  __syncthreads();
+  if (bar->tmem_base != 0) return;
+  __syncthreads();
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bar->q_full, 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&bar->k_full[s], 1);
+      mbar_init(&bar->k_empty[s], 1);
+      mbar_init(&bar->v_full[s], 1);
+      mbar_init(&bar->v_empty[s], 1);
+    }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&bar->s_full[t], 1);
+      mbar_init(&bar->p_full[t], 128);
+      mbar_init(&bar->o_full[t], 1);
+    }
+    mbar_init(&bar->drain, 1);
+    bar->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar->tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bar->tmem_base;
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      mbar_expect_tx(&bar->q_full, 2 * kTileBytes);
+      for (int t = 0; t < 2; ++t)
+        tma_load_4d(sQ + t * kTileBytes, &mapQ, &bar->q_full, 0, x0 + (qt0 + t) * p.step_x,
+                    y0 + (qt0 + t) * p.step_y, bh);
+      bool ok = true;
+      int issued = 0;
+      for (int j = 0; j < ntiles && ok; ++j) {
+        const int s = j % kStages;
+        const uint32_t par = ((j / kStages) & 1) ^ 1;
+        ok = mbar_wait(&bar->k_empty[s], par, bar, p.status);
+        if (!ok) break;
+        mbar_expect_tx(&bar->k_full[s], kTileBytes);
+        tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, x0 + j * p.step_x, y0 + j * p.step_y, bh);
+        ok = mbar_wait(&bar->v_empty[s], par, bar, p.status);
+        if (!ok) { issued = j; break; }
+        mbar_expect_tx(&bar->v_full[s], kTileBytes);
+        tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, x0 + j * p.step_x, y0 + j * p.step_y, bh);
+        issued = j + 1;
+      }
+      if (!ok) {
+        // let the copies still in flight land before the CTA leaves (bounded by the same limit)
+        const unsigned long long t0 = globaltimer();
+        for (int j = max(0, issued - kStages); j < issued; ++j)
+          while (!mbar_try(&bar->v_full[j % kStages], (j / kStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      bool ok = mbar_wait(&bar->q_full, 0, bar, p.status);
+      auto issue_qk = [&](int t, int j) {
+        const uint32_t kb = sK + (j % kStages) * kTileBytes, qb = sQ + t * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks)
+          mma_ss(tmem + kColS + t * kTile, smem_desc(qb + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
+        tc_commit(&bar->s_full[t]);
+      };
+      if (ok) ok = mbar_wait(&bar->k_full[0], 0, bar, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, 0);
+        issue_qk(1, 0);
+        tc_commit(&bar->k_empty[0]);
+      }
+      for (int j = 0; j < ntiles && ok; ++j) {
+        const int s = j % kStages;
+        ok = mbar_wait(&bar->v_full[s], (j / kStages) & 1, bar, p.status);
+        for (int t = 0; t < 2 && ok; ++t) {
+          ok = mbar_wait(&bar->p_full[t], j & 1, bar, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t vb = sV + s * kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < kTile / 16; ++ks)
+            mma_ts(tmem + kColO + t * kD, tmem + kColP + t * (kTile / 2) + ks * 8, smem_desc(vb + ks * 2048), kIdescPV,
+                   (j > 0 || ks > 0) ? 1u : 0u);
+          if (j + 1 < ntiles) {
+            if (t == 0) {
+              ok = mbar_wait(&bar->k_full[(j + 1) % kStages], ((j + 1) / kStages) & 1, bar, p.status);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_qk(t, j + 1);
+            if (t == 1) tc_commit(&bar->k_empty[(j + 1) % kStages]);
+          } else {
+            tc_commit(&bar->o_full[t]);
+          }
+        }
+        if (ok) tc_commit(&bar->v_empty[s]);
+      }
+      // Teardown: every MMA issued so far must have retired before tensor memory is released.
+      tc_commit(&bar->drain);
+      const unsigned long long t0 = globaltimer();
+      while (!mbar_try(&bar->drain, 0) && globaltimer() - t0 < kWaitLimitNs) {}
+    }
+  } else if (warp >= 4) {
+    // ================= softmax + epilogue: one thread per query row =================
+    const int t = (warp - 4) >> 2;                 // query tile of this warpgroup
+    const int row = ((warp & 3) << 5) + lane;      // row of the tile == tensor-memory lane
+    const uint32_t lane_base = (uint32_t)((warp & 3) << 5) << 16;
+    const uint32_t tS = tmem + lane_base + kColS + t * kTile;
+    const uint32_t tO = tmem + lane_base + kColO + t * kD;
+    const uint32_t tP = tmem + lane_base + kColP + t * (kTile / 2);
+    const float sl2 = p.scale_log2;
+    const float kLazy = 8.f / sl2;                 // rescale only when the max grew by > 2^8
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+
+    for (int j = 0; j < ntiles && ok; ++j) {
+      ok = mbar_wait(&bar->s_full[t], j & 1, bar, p.status);
+      if (!ok) break;
+      tc_fence_after();
+      // which keys of this tile exist?
+      const int kx = x0 + j * p.step_x, ky = y0 + j * p.step_y;
+      const bool full_tile = (kx + p.box_w <= x_end) && (ky + p.box_h <= y_end);
+      uint32_t valid[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+      if (!full_tile) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t bits = 0;
+          for (int i = 0; i < 32; ++i) {
+            const int key = 32 * c + i;
+            const int lx = key % p.box_w, ly = key / p.box_w;
+            if (kx + lx < x_end && ky + ly < y_end) bits |= 1u << i;
+          }
+          valid[c] = bits;
+        }
+      }
+      // pass 1: row maximum
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tS + 32 * c, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+          if (full_tile || ((valid[c] >> i) & 1u)) mx = fmaxf(mx, __uint_as_float(v[i]));
+      }
+      float alpha = 1.f;
+      bool rescale = false;
+      if (mx > m + kLazy) {          // always true on the first tile (m = -inf, mx finite)
+        alpha = ex2((m - mx) * sl2); // first tile: exp2(-inf) = 0
+        l *= alpha;
+        m = mx;
+        rescale = j > 0;
+      }
+      if (__any_sync(0xffffffffu, rescale)) {
+        // PV of the previous key tile has retired (its commit preceded this S tile's): O is ours
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tO + 32 * c, v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+          tmem_st32(tO + 32 * c, v);
+        }
+      }
+      // pass 2: p = exp2(s*scale - m*scale), row sum, P (bf16) into tensor memory
+      const float mneg = -m * sl2;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tS + 32 * c, v);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), sl2, mneg));
+          float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), sl2, mneg));
+          if (!full_tile) {
+            if (!((valid[c] >> (2 * i)) & 1u)) p0 = 0.f;
+            if (!((valid[c] >> (2 * i + 1)) & 1u)) p1 = 0.f;
+          }
+          l += p0 + p1;
+          pk[i] = pack_bf16(p0, p1);
+        }
+        tmem_st16(tP + 16 * c, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bar->p_full[t]);
+    }
+
+    if (ok) ok = mbar_wait(&bar->o_full[t], 0, bar, p.status);
+    if (ok) {
+      tc_fence_after();
+      // this row's token
+      const int qx = x0 + (qt0 + t) * p.step_x + row % p.box_w, qy = y0 + (qt0 + t) * p.step_y + row / p.box_w;
+      const bool row_ok = (qt0 + t < ntiles) && qx < x_end && qy < y_end;
+      const float inv = 1.f / l;
+      __nv_bfloat16* dst = p.o + ((size_t)bh * p.tokens_per_head + (size_t)qy * p.gridW + qx) * kD;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tO + 32 * c, v);
+        tmem_wait_ld();
+        if (row_ok) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + 32 * c + 8 * i) = w;
+          }
+        }
+      }
+    }
+  }
+
+  // ================= common teardown =================
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+// ---- host side ----------------------------------------------------------------------
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = (EncodeFn)ptr;
+  }
+  return fn;
+}
+
+struct Geometry {
+  int gridW, gridH, win_w, win_h, box_w, box_h, step_x, step_y, nwx, nwy, tiles_per_window;
+};
+
+bool geometry(const AttnArgs& a, bool full, Geometry* g) {
+  const int N = a.Hg * a.Wg;
+  if (full || (a.wh >= a.Hg && a.ww >= a.Wg)) {
+    *g = Geometry{N, 1, N, 1, kTile, 1, kTile, 0, 1, 1, ceil_div(N, kTile)};
+    return true;
+  }
+  const int ww = a.ww;
+  if (ww > kTile || (ww & (ww - 1)) != 0) return false;   // box width must divide 128
+  const int bh = kTile / ww;
+  const int wh = a.wh < a.Hg ? a.wh : a.Hg;
+  *g = Geometry{a.Wg, a.Hg, ww, wh, ww, bh, 0, bh, ceil_div(a.Wg, ww), ceil_div(a.Hg, wh), ceil_div(wh, bh)};
+  return true;
+}
+
+}  // namespace
+
+bool attn_tc_supported(const AttnArgs& a, bool full) {
+  if (a.dtype != JV_BF16 || a.D != kD) return false;
+  Geometry g;
+  if (!geometry(a, full, &g)) return false;
+  if ((int64_t)g.nwx * g.nwy > 65535) return false;
+  // 128-byte rows keep every TMA stride a multiple of 16 bytes; the base must be 16-byte aligned (checked by the ABI)
+  return encode_fn() != nullptr;
+}
+
+cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream_t st) {
+  Geometry g;
+  if (!geometry(a, full, &g)) return cudaErrorInvalidValue;
+  EncodeFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  const int N = a.Hg * a.Wg;
+  CUtensorMap maps[3];
+  const void* ptrs[3] = {a.q, a.k, a.v};
+  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.gridW, (cuuint64_t)g.gridH, (cuuint64_t)a.BH};
+  const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.gridW * kD * 2, (cuuint64_t)N * kD * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 3; ++i) {
+    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  TcParams p;
+  p.o = (__nv_bfloat16*)a.o;
+  p.status = status;
+  p.gridW = g.gridW;
+  p.gridH = g.gridH;
+  p.tokens_per_head = N;
+  p.win_w = g.win_w;
+  p.win_h = g.win_h;
+  p.box_w = g.box_w;
+  p.box_h = g.box_h;
+  p.step_x = g.step_x;
+  p.step_y = g.step_y;
+  p.nwx = g.nwx;
+  p.scale_log2 = a.scale * 1.4426950408889634f;
+  dim3 grid(ceil_div(g.tiles_per_window, 2), g.nwx * g.nwy, a.BH);
+  attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], p);
+  count_launch();
+  return cudaGetLastError();
+}
+
 }  // namespace jv
