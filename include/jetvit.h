@@ -99,6 +99,39 @@ jv_status jv_linear_attn(const void* q, const void* k, const void* v, void* o, c
                          float eps, const jv_dwc* dwc, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * L without caller scratch.  (The paper has no counterpart: this entry point exists for
+ * integration, not for the method.)
+ *
+ * Some callers cannot allocate device memory at the point where they run a mixer: a
+ * serving engine whose own pool already owns the whole GPU, a real-time loop that must
+ * not hit the device-wide synchronisation of cudaMalloc / cudaFree, a plug-in interface
+ * that offers a stream and nothing else.  jv_linear_attn_static computes exactly what
+ * jv_linear_attn computes (same kernels, bit-identical output) but takes its scratch from
+ * a fixed array of JV_STATIC_SCRATCH_BYTES that is part of the library image; the caller
+ * passes only inputs and outputs.  The call allocates nothing and frees nothing.
+ *
+ *   Limit     jv_workspace_bytes('L', shape, dwc) must not exceed JV_STATIC_SCRATCH_BYTES
+ *             (16 MiB: enough for B*H*N up to about 3.9 M token-heads at D = 64, e.g.
+ *             B=8, H=16, 64x64 grid, or B=1, H=16, 128x128 grid).  Larger problems are
+ *             refused with JV_ERR_WORKSPACE before anything is launched; use
+ *             jv_linear_attn with your own buffer for those.
+ *   Cost      every GPU on which the library is loaded carries the 16 MiB array until the
+ *             process exits, whether or not this function is ever called.
+ *   Set-up    the first call on each device looks up the array's device address (that
+ *             device must be current, as for every call).  Make that first call during
+ *             initialisation, before any stream capture begins.
+ *   Sharing   there is one array per device and every call uses it.  It keeps whatever
+ *             the previous call left; nothing in it needs clearing, because every value
+ *             a call consumes is written earlier in that same call.  Two calls that may overlap on the
+ *             GPU (different streams, no ordering between them) race on the array and
+ *             corrupt each other: order them on one stream or with events.
+ * Other arguments and return codes are those of jv_linear_attn.
+ */
+#define JV_STATIC_SCRATCH_BYTES (16u << 20)
+jv_status jv_linear_attn_static(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
+                                float eps, const jv_dwc* dwc, void* cuda_stream);
+
+/*
  * W -- window attention (Sec. 3.2.2): the grid is cut into non-overlapping
  * win_h x win_w windows anchored at (0, 0); softmax attention (Eq. 1) runs
  * inside each window.  When the grid is not a multiple of the window the

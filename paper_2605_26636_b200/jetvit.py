@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
         L.jv_workspace_bytes.argtypes = [ctypes.c_char, shp, dwc]
         L.jv_workspace_bytes.restype = sz
         L.jv_linear_attn.argtypes = [vp, vp, vp, vp, shp, f32, dwc, vp, sz, vp]
+        L.jv_linear_attn_static.argtypes = [vp, vp, vp, vp, shp, f32, dwc, vp]
+        L.jv_linear_attn_static.restype = ctypes.c_int
         L.jv_window_attn.argtypes = [vp, vp, vp, vp, shp, i32, i32, f32, vp, sz, vp]
         L.jv_full_attn.argtypes = [vp, vp, vp, vp, shp, f32, vp, sz, vp]
         L.jv_hybrid_mixers.argtypes = [i32, ctypes.c_char_p, ctypes.POINTER(vp), ctypes.POINTER(vp),
@@ -159,6 +161,26 @@ def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict
         st = lib().jv_linear_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
                                   float(eps), ctypes.byref(d) if d is not None else None, wp, wn, _stream(stream))
     _raise(st, "jv_linear_attn")
+    return out
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def linear_attn_static(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict] = None, *, out,
+                       stream=None) -> torch.Tensor:
+    """jv_linear_attn_static: the linear block with the library's built-in scratch, for
+    callers that must not allocate.  This wrapper allocates nothing either: ``out`` is
+    required.  Problems needing more than STATIC_SCRATCH_BYTES raise JV_ERR_WORKSPACE;
+    calls that can overlap on the GPU must be ordered by the caller (they share the scratch)."""
+    _check_tensors(q, k, v, out)
+    shape = make_shape(q, Hg, Wg)
+    d = make_dwc(dwc, q.device)
+    with torch.cuda.device(q.device):
+        st = lib().jv_linear_attn_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                         ctypes.byref(shape), float(eps),
+                                         ctypes.byref(d) if d is not None else None, _stream(stream))
+    _raise(st, "jv_linear_attn_static")
     return out
 
 
