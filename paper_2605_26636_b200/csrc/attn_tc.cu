@@ -239,6 +239,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 0) {
+    __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar->tmem_base)),
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -340,7 +341,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     bool ok = true;
 
     for (int j = 0; j < ntiles && ok; ++j) {
-      ok = mbar_wait(&bar->s_full[t], j & 1, bar, p.status);
+      // warp-uniform outcome: the tensor-memory accesses below are warp-collective
+      ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], j & 1, bar, p.status));
       if (!ok) break;
       tc_fence_after();
       // which keys of this tile exist?
@@ -416,7 +418,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       mbar_arrive(&bar->p_full[t]);
     }
 
-    if (ok) ok = mbar_wait(&bar->o_full[t], 0, bar, p.status);
+    ok = __all_sync(0xffffffffu, ok && mbar_wait(&bar->o_full[t], 0, bar, p.status));
     if (ok) {
       tc_fence_after();
       // this row's token
@@ -445,6 +447,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   }
 
   // ================= common teardown =================
+  __syncwarp();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
