@@ -387,6 +387,37 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_single(args):
+    """One mixer alone at a named workload shape (the command the profiler captures)."""
+    from paper_2605_26636_b200 import jetvit as jv
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    w = inputs.WORKLOADS[args.workload]
+    stream = torch.cuda.current_stream()
+    sets = [[t.to(dev) for t in inputs.qkv(w, layer=l)] for l in range(3)]
+    outs = [torch.empty_like(s[0]) for s in sets]
+    C = w.H * w.D
+    dwc = None
+    if args.single == "L+dwc":
+        d = inputs.dwc_weights(C, C // 8, 3, inputs.seed_for(w.cfg, 0, 3))
+        dwc = {k: (v.to(dev) if hasattr(v, "to") else v) for k, v in d.items()}
+    ws = jv.alloc_workspace("L", jv.make_shape(sets[0][0], w.Hg, w.Wg), jv.make_dwc(dwc, dev), dev)
+
+    def fn(i):
+        q, k, v = sets[i % 3]
+        o = outs[i % 3]
+        if args.single in ("L", "L+dwc"):
+            jv.linear_attn(q, k, v, w.Hg, w.Wg, dwc=dwc, out=o, ws=ws)
+        elif args.single == "W":
+            jv.window_attn(q, k, v, w.Hg, w.Wg, WIN, WIN, out=o)
+        else:
+            jv.full_attn(q, k, v, out=o)
+    ms = time_calls(fn, args.steps, args.warmup, stream)
+    assert jv.device_status() == jv.JV_OK
+    print(json.dumps({"single": args.single, "workload": args.workload, "ms": ms,
+                      "tokens_per_s": w.tokens / (ms * 1e-3)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -394,8 +425,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--single", choices=["L", "L+dwc", "W", "F"], default=None,
+                    help="time one mixer alone (used for profiler captures)")
+    ap.add_argument("--workload", default="dinov3_l", choices=sorted(inputs.WORKLOADS))
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.single:
+        run_single(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)
