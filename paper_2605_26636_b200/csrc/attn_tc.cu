@@ -167,8 +167,17 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Waits for this thread's outstanding tensor-memory loads.  The registers of the load are
+// threaded through the statement so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :: "memory");
+}
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -176,8 +185,57 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Two fp32 values in one 64-bit register: the packed fp32x2 arithmetic of sm_100.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// ---- softmax building blocks: 32 scores of one query row at a time -------------------
+constexpr uint32_t kNegInf = 0xff800000u;
+__device__ __forceinline__ void max32(const uint32_t (&v)[32], float (&mx)[4]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      mx[u] = max3(mx[u], __uint_as_float(v[8 * i + 2 * u]), __uint_as_float(v[8 * i + 2 * u + 1]));
+}
+// p = exp2(s * sl2 + mneg) for 32 scores; adds them into four packed partial sums and
+// packs them to bf16 pairs (even key in the low half).
+__device__ __forceinline__ void exp32(const uint32_t (&v)[32], uint64_t sl2x2, uint64_t mnegx2, uint64_t (&lsum)[4],
+                                      uint32_t (&pk)[16]) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const uint64_t x = fma2(pack2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2x2, mnegx2);
+    float x0, x1;
+    unpack2(x, x0, x1);
+    const float p0 = ex2(x0), p1 = ex2(x1);
+    lsum[i & 3] = add2(lsum[i & 3], pack2(p0, p1));
+    pk[i] = pack_bf16(p0, p1);
+  }
 }
 
 // Shared-memory matrix descriptors (128-byte swizzle; 8-row groups 1024 bytes apart).
@@ -340,79 +398,109 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     float m = -INFINITY, l = 0.f;
     bool ok = true;
 
-    for (int j = 0; j < ntiles && ok; ++j) {
-      // warp-uniform outcome: the tensor-memory accesses below are warp-collective
-      ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], j & 1, bar, p.status));
-      if (!ok) break;
-      tc_fence_after();
-      // which keys of this tile exist?
-      const int kx = x0 + j * p.step_x, ky = y0 + j * p.step_y;
-      const bool full_tile = (kx + p.box_w <= x_end) && (ky + p.box_h <= y_end);
-      uint32_t valid[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-      if (!full_tile) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t bits = 0;
-          for (int i = 0; i < 32; ++i) {
-            const int key = 32 * c + i;
-            const int lx = key % p.box_w, ly = key / p.box_w;
-            if (kx + lx < x_end && ky + ly < y_end) bits |= 1u << i;
-          }
-          valid[c] = bits;
-        }
-      }
-      // pass 1: row maximum
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tS + 32 * c, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (full_tile || ((valid[c] >> i) & 1u)) mx = fmaxf(mx, __uint_as_float(v[i]));
-      }
+    const uint64_t sl2x2 = pack2(sl2, sl2);
+    const int lg_bw = 31 - __clz(p.box_w);          // box_w is a power of two
+
+    // One key tile: two passes over the 128 scores of this thread's row (maximum, then
+    // exponentials), reading tensor memory 32 columns at a time with the next read in flight.
+    auto tile = [&](int j) {
+      uint32_t va[32], vb[32];
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      tmem_ld32(tS, va);
+      tmem_wait_ld(va);
+      tmem_ld32(tS + 32, vb);
+      max32(va, mx4);
+      tmem_wait_ld(vb);
+      tmem_ld32(tS + 64, va);
+      max32(vb, mx4);
+      tmem_wait_ld(va);
+      tmem_ld32(tS + 96, vb);
+      max32(va, mx4);
+      tmem_wait_ld(vb);
+      tmem_ld32(tS, va);                             // first read of pass 2
+      max32(vb, mx4);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));   // finite: >= 1 valid key per tile
+
       float alpha = 1.f;
       bool rescale = false;
-      if (mx > m + kLazy) {          // always true on the first tile (m = -inf, mx finite)
+      if (mx > m + kLazy) {          // always true on the first tile (m = -inf)
         alpha = ex2((m - mx) * sl2); // first tile: exp2(-inf) = 0
         l *= alpha;
         m = mx;
         rescale = j > 0;
       }
+      tmem_wait_ld(va);
       if (__any_sync(0xffffffffu, rescale)) {
         // PV of the previous key tile has retired (its commit preceded this S tile's): O is ours
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
-          uint32_t v[32];
-          tmem_ld32(tO + 32 * c, v);
-          tmem_wait_ld();
+          tmem_ld32(tO + 32 * c, vb);
+          tmem_wait_ld(vb);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-          tmem_st32(tO + 32 * c, v);
+          for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
+          tmem_st32(tO + 32 * c, vb);
         }
       }
-      // pass 2: p = exp2(s*scale - m*scale), row sum, P (bf16) into tensor memory
       const float mneg = -m * sl2;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tS + 32 * c, v);
-        tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = ex2(fmaf(__uint_as_float(v[2 * i]), sl2, mneg));
-          float p1 = ex2(fmaf(__uint_as_float(v[2 * i + 1]), sl2, mneg));
-          if (!full_tile) {
-            if (!((valid[c] >> (2 * i)) & 1u)) p0 = 0.f;
-            if (!((valid[c] >> (2 * i + 1)) & 1u)) p1 = 0.f;
+      const uint64_t mnegx2 = pack2(mneg, mneg);
+      uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
+      uint32_t pk[16];
+      tmem_ld32(tS + 32, vb);
+      exp32(va, sl2x2, mnegx2, lsum, pk);
+      tmem_st16(tP, pk);
+      tmem_wait_ld(vb);
+      tmem_ld32(tS + 64, va);
+      exp32(vb, sl2x2, mnegx2, lsum, pk);
+      tmem_st16(tP + 16, pk);
+      tmem_wait_ld(va);
+      tmem_ld32(tS + 96, vb);
+      exp32(va, sl2x2, mnegx2, lsum, pk);
+      tmem_st16(tP + 32, pk);
+      tmem_wait_ld(vb);
+      exp32(vb, sl2x2, mnegx2, lsum, pk);
+      tmem_st16(tP + 48, pk);
+      float a0, a1, b0, b1;
+      unpack2(add2(lsum[0], lsum[1]), a0, a1);
+      unpack2(add2(lsum[2], lsum[3]), b0, b1);
+      l += (a0 + a1) + (b0 + b1);
+    };
+
+    for (int j = 0; j < ntiles && ok; ++j) {
+      // warp-uniform outcome: the tensor-memory accesses below are warp-collective
+      ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], j & 1, bar, p.status));
+      if (!ok) break;
+      tc_fence_after();
+      // which keys of this tile exist?  vx, vy: valid extent of the box along x and y
+      const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
+      if (vx < p.box_w || vy < p.box_h) {
+        // Edge tile: overwrite the scores of keys that do not exist (outside the grid or the
+        // window) with -inf in tensor memory, then treat the tile like any other.
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t bits = 0;
+          if (p.box_w >= 32) {                       // the 32 keys lie in one box row
+            const int ly = (32 * c) >> lg_bw, lx0 = (32 * c) & (p.box_w - 1);
+            const int n = min(32, vx - lx0);
+            if (ly < vy && n > 0) bits = n >= 32 ? 0xffffffffu : ((1u << n) - 1u);
+          } else {                                   // 32 / box_w whole box rows
+            const uint32_t rowbits = (1u << min(vx, p.box_w)) - 1u;
+            const int ly0 = (32 * c) >> lg_bw;
+            for (int r = 0; r < (32 >> lg_bw); ++r)
+              if (ly0 + r < vy) bits |= rowbits << (r << lg_bw);
           }
-          l += p0 + p1;
-          pk[i] = pack_bf16(p0, p1);
+          if (bits != 0xffffffffu) {                 // warp-uniform: the mask depends on the tile only
+            uint32_t v[32];
+            tmem_ld32(tS + 32 * c, v);
+            tmem_wait_ld(v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (!((bits >> i) & 1u)) v[i] = kNegInf;   // exp2(-inf) = 0 and -inf never wins the maximum
+            tmem_st32(tS + 32 * c, v);
+          }
         }
-        tmem_st16(tP + 16 * c, pk);
+        tmem_wait_st();
       }
+      tile(j);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bar->p_full[t]);
@@ -430,7 +518,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int c = 0; c < 2; ++c) {
         uint32_t v[32];
         tmem_ld32(tO + 32 * c, v);
-        tmem_wait_ld();
+        tmem_wait_ld(v);
         if (row_ok) {
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
