@@ -110,6 +110,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barrie
   }
 }
 
+// The same for a whole converged warp, with a warp-uniform outcome.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Barriers* b, int* status) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, b, status));
+}
+
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
                                             int c2, int c3) {
   asm volatile(
@@ -120,11 +125,21 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
 // ---- tcgen05 wrappers -------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// One lane of a converged warp (the same one every time for a full warp).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
+  return pred != 0;
+}
+// The tcgen05 issue wrappers below are called by a whole converged warp; one elected lane issues.
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+  if (elect_one())
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+  __syncwarp();
 }
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  if (elect_one())
   asm volatile(
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
@@ -132,6 +147,7 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t
 }
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  if (elect_one())
   asm volatile(
       "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
@@ -223,16 +239,52 @@ __device__ __forceinline__ void max32(const uint32_t (&v)[32], float (&mx)[4]) {
     for (int u = 0; u < 4; ++u)
       mx[u] = max3(mx[u], __uint_as_float(v[8 * i + 2 * u]), __uint_as_float(v[8 * i + 2 * u + 1]));
 }
-// p = exp2(s * sl2 + mneg) for 32 scores; adds them into four packed partial sums and
-// packs them to bf16 pairs (even key in the low half).
+// exp2 on the FMA pipe, for part of the scores (the MUFU unit, 16 results per clock and SM,
+// is the tightest resource of softmax attention at head_dim 64).  x = n + f with n = round(x),
+// f in [-0.5, 0.5]; 2^f by a degree-3 minimax polynomial (relative error 7.5e-5, well below
+// the bf16 rounding of P); n goes straight into the exponent field.  Valid for x in [-126, 126].
+constexpr float kPolyC0 = 0.9999280571937561f, kPolyC1 = 0.6932609677314758f;
+constexpr float kPolyC2 = 0.2426111251115799f, kPolyC3 = 0.0551716685295105f;
+constexpr float kRoundMagic = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+__device__ __forceinline__ void exp2_poly2(uint64_t x, float& p0, float& p1) {
+  float x0, x1;
+  unpack2(x, x0, x1);
+  x = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t t = add2(x, pack2(kRoundMagic, kRoundMagic));
+  const uint64_t n = add2(t, pack2(-kRoundMagic, -kRoundMagic));
+  const uint64_t f = fma2(n, pack2(-1.f, -1.f), x);
+  uint64_t q = fma2(f, pack2(kPolyC3, kPolyC3), pack2(kPolyC2, kPolyC2));
+  q = fma2(q, f, pack2(kPolyC1, kPolyC1));
+  q = fma2(q, f, pack2(kPolyC0, kPolyC0));
+  float q0, q1, t0, t1;
+  unpack2(q, q0, q1);
+  unpack2(t, t0, t1);
+  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
+#ifndef JV_POLY_PAIRS_OF_8
+#define JV_POLY_PAIRS_OF_8 2   // of every 8 score pairs, this many take the polynomial path
+#endif
+// p = exp2(s * sl2 + mneg) for 32 scores; adds them into four packed partial sums and packs
+// them to bf16 pairs (even key in the low half).  kTrack also folds the scores into mx.
+template <bool kTrack>
 __device__ __forceinline__ void exp32(const uint32_t (&v)[32], uint64_t sl2x2, uint64_t mnegx2, uint64_t (&lsum)[4],
-                                      uint32_t (&pk)[16]) {
+                                      uint32_t (&pk)[16], float (&mx)[4]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const uint64_t x = fma2(pack2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), sl2x2, mnegx2);
-    float x0, x1;
-    unpack2(x, x0, x1);
-    const float p0 = ex2(x0), p1 = ex2(x1);
+    const float s0 = __uint_as_float(v[2 * i]), s1 = __uint_as_float(v[2 * i + 1]);
+    if (kTrack) mx[i & 3] = max3(mx[i & 3], s0, s1);
+    const uint64_t x = fma2(pack2(s0, s1), sl2x2, mnegx2);
+    float p0, p1;
+    if ((i & 7) < JV_POLY_PAIRS_OF_8) {
+      exp2_poly2(x, p0, p1);
+    } else {
+      float x0, x1;
+      unpack2(x, x0, x1);
+      p0 = ex2(x0);
+      p1 = ex2(x1);
+    }
     lsum[i & 3] = add2(lsum[i & 3], pack2(p0, p1));
     pk[i] = pack_bf16(p0, p1);
   }
@@ -307,84 +359,99 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = bar->tmem_base;
 
+  // Warps 0 and 1 run their loops with all 32 lanes (waits included) so that stage counters,
+  // addresses and descriptors stay warp-uniform; only the TMA / tcgen05 instructions themselves
+  // are issued by one elected lane (always the same one: the election is deterministic for a
+  // full warp, and tcgen05.commit has to come from the thread that issued the MMAs).
   if (warp == 0) {
     // ================= TMA producer =================
-    if (lane == 0) {
+    if (elect_one()) {
       mbar_expect_tx(&bar->q_full, 2 * kTileBytes);
       for (int t = 0; t < 2; ++t)
         tma_load_4d(sQ + t * kTileBytes, &mapQ, &bar->q_full, 0, x0 + (qt0 + t) * p.step_x,
                     y0 + (qt0 + t) * p.step_y, bh);
-      bool ok = true;
-      int issued = 0;
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % kStages;
-        const uint32_t par = ((j / kStages) & 1) ^ 1;
-        ok = mbar_wait(&bar->k_empty[s], par, bar, p.status);
-        if (!ok) break;
+    }
+    __syncwarp();
+    bool ok = true;
+    int issued = 0, s = 0;
+    uint32_t par = 1;                       // parity of the "empty" phase this pass over the ring waits for
+    for (int j = 0; j < ntiles; ++j) {
+      ok = warp_wait(&bar->k_empty[s], par, bar, p.status);
+      if (!ok) break;
+      if (elect_one()) {
         mbar_expect_tx(&bar->k_full[s], kTileBytes);
         tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, x0 + j * p.step_x, y0 + j * p.step_y, bh);
-        ok = mbar_wait(&bar->v_empty[s], par, bar, p.status);
-        if (!ok) { issued = j; break; }
+      }
+      __syncwarp();
+      ok = warp_wait(&bar->v_empty[s], par, bar, p.status);
+      if (!ok) break;
+      if (elect_one()) {
         mbar_expect_tx(&bar->v_full[s], kTileBytes);
         tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, x0 + j * p.step_x, y0 + j * p.step_y, bh);
-        issued = j + 1;
       }
-      if (!ok) {
-        // let the copies still in flight land before the CTA leaves (bounded by the same limit)
-        const unsigned long long t0 = globaltimer();
-        for (int j = max(0, issued - kStages); j < issued; ++j)
-          while (!mbar_try(&bar->v_full[j % kStages], (j / kStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
-      }
+      __syncwarp();
+      issued = j + 1;
+      if (++s == kStages) { s = 0; par ^= 1; }
+    }
+    if (!ok && lane == 0) {
+      // let the copies still in flight land before the CTA leaves (bounded by the same limit)
+      const unsigned long long t0 = globaltimer();
+      for (int j = max(0, issued - kStages); j < issued; ++j)
+        while (!mbar_try(&bar->v_full[j % kStages], (j / kStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
     }
   } else if (warp == 1) {
     // ================= MMA issuer =================
-    if (lane == 0) {
-      bool ok = mbar_wait(&bar->q_full, 0, bar, p.status);
-      auto issue_qk = [&](int t, int j) {
-        const uint32_t kb = sK + (j % kStages) * kTileBytes, qb = sQ + t * kTileBytes;
+    bool ok = warp_wait(&bar->q_full, 0, bar, p.status);
+    auto issue_qk = [&](int t, int stage) {
+      const uint32_t kb = sK + stage * kTileBytes, qb = sQ + t * kTileBytes;
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks)
-          mma_ss(tmem + kColS + t * kTile, smem_desc(qb + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
-        tc_commit(&bar->s_full[t]);
-      };
-      if (ok) ok = mbar_wait(&bar->k_full[0], 0, bar, p.status);
-      if (ok) {
+      for (int ks = 0; ks < kD / 16; ++ks)
+        mma_ss(tmem + kColS + t * kTile, smem_desc(qb + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
+      tc_commit(&bar->s_full[t]);
+    };
+    if (ok) ok = warp_wait(&bar->k_full[0], 0, bar, p.status);
+    if (ok) {
+      tc_fence_after();
+      issue_qk(0, 0);
+      issue_qk(1, 0);
+      tc_commit(&bar->k_empty[0]);
+    }
+    int s = 0, s1 = 1 % kStages;            // ring stage of key tile j and of key tile j + 1
+    uint32_t ph = 0, ph1 = (kStages == 1);  // and their "full" parities
+    for (int j = 0; j < ntiles && ok; ++j) {
+      ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
+      for (int t = 0; t < 2 && ok; ++t) {
+        ok = warp_wait(&bar->p_full[t], j & 1, bar, p.status);
+        if (!ok) break;
         tc_fence_after();
-        issue_qk(0, 0);
-        issue_qk(1, 0);
-        tc_commit(&bar->k_empty[0]);
-      }
-      for (int j = 0; j < ntiles && ok; ++j) {
-        const int s = j % kStages;
-        ok = mbar_wait(&bar->v_full[s], (j / kStages) & 1, bar, p.status);
-        for (int t = 0; t < 2 && ok; ++t) {
-          ok = mbar_wait(&bar->p_full[t], j & 1, bar, p.status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t vb = sV + s * kTileBytes;
+        const uint32_t vb = sV + s * kTileBytes;
 #pragma unroll
-          for (int ks = 0; ks < kTile / 16; ++ks)
-            mma_ts(tmem + kColO + t * kD, tmem + kColP + t * (kTile / 2) + ks * 8, smem_desc(vb + ks * 2048), kIdescPV,
-                   (j > 0 || ks > 0) ? 1u : 0u);
-          if (j + 1 < ntiles) {
-            if (t == 0) {
-              ok = mbar_wait(&bar->k_full[(j + 1) % kStages], ((j + 1) / kStages) & 1, bar, p.status);
-              if (!ok) break;
-              tc_fence_after();
-            }
-            issue_qk(t, j + 1);
-            if (t == 1) tc_commit(&bar->k_empty[(j + 1) % kStages]);
-          } else {
-            tc_commit(&bar->o_full[t]);
+        for (int ks = 0; ks < kTile / 16; ++ks)
+          mma_ts(tmem + kColO + t * kD, tmem + kColP + t * (kTile / 2) + ks * 8, smem_desc(vb + ks * 2048), kIdescPV,
+                 (j > 0 || ks > 0) ? 1u : 0u);
+        if (j + 1 < ntiles) {
+          if (t == 0) {
+            ok = warp_wait(&bar->k_full[s1], ph1, bar, p.status);
+            if (!ok) break;
+            tc_fence_after();
           }
+          issue_qk(t, s1);
+          if (t == 1) tc_commit(&bar->k_empty[s1]);
+        } else {
+          tc_commit(&bar->o_full[t]);
         }
-        if (ok) tc_commit(&bar->v_empty[s]);
       }
-      // Teardown: every MMA issued so far must have retired before tensor memory is released.
-      tc_commit(&bar->drain);
+      if (ok) tc_commit(&bar->v_empty[s]);
+      if (++s == kStages) { s = 0; ph ^= 1; }
+      if (++s1 == kStages) { s1 = 0; ph1 ^= 1; }
+    }
+    // Teardown: every MMA issued so far must have retired before tensor memory is released.
+    tc_commit(&bar->drain);
+    if (lane == 0) {
       const unsigned long long t0 = globaltimer();
       while (!mbar_try(&bar->drain, 0) && globaltimer() - t0 < kWaitLimitNs) {}
     }
+    __syncwarp();
   } else if (warp >= 4) {
     // ================= softmax + epilogue: one thread per query row =================
     const int t = (warp - 4) >> 2;                 // query tile of this warpgroup
@@ -446,23 +513,83 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
       uint32_t pk[16];
       tmem_ld32(tS + 32, vb);
-      exp32(va, sl2x2, mnegx2, lsum, pk);
+      exp32<false>(va, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tP, pk);
       tmem_wait_ld(vb);
       tmem_ld32(tS + 64, va);
-      exp32(vb, sl2x2, mnegx2, lsum, pk);
+      exp32<false>(vb, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tP + 16, pk);
       tmem_wait_ld(va);
       tmem_ld32(tS + 96, vb);
-      exp32(va, sl2x2, mnegx2, lsum, pk);
+      exp32<false>(va, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tP + 32, pk);
       tmem_wait_ld(vb);
-      exp32(vb, sl2x2, mnegx2, lsum, pk);
+      exp32<false>(vb, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tP + 48, pk);
       float a0, a1, b0, b1;
       unpack2(add2(lsum[0], lsum[1]), a0, a1);
       unpack2(add2(lsum[2], lsum[3]), b0, b1);
       l += (a0 + a1) + (b0 + b1);
+    };
+
+    // Later key tiles, one pass: the exponentials are taken against the maximum known so far
+    // while the tile's own maximum is tracked on the side.  Any reference value gives the same
+    // softmax as long as nothing overflows, so a larger maximum only matters for the tiles
+    // that follow: O and l are rescaled at the start of the next tile, once this tile's PV
+    // has retired.  A tile whose scores exceed the reference by more than 2^kSpecLimit is redone
+    // with the two-pass routine above (P has not been published yet).
+    constexpr float kSpecLimit = 64.f;
+    float pend_alpha = 1.f, pend_m = 0.f;
+    bool pending = false;
+    auto spec_tile = [&](int j) -> bool {
+      uint32_t va[32], vb[32];
+      if (__any_sync(0xffffffffu, pending)) {
+        // the previous tile's PV has retired (its commit preceded this S tile's): O is ours
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          tmem_ld32(tO + 32 * c, vb);
+          tmem_wait_ld(vb);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * pend_alpha);
+          tmem_st32(tO + 32 * c, vb);
+        }
+        if (pending) { l *= pend_alpha; m = pend_m; }
+        pending = false;
+        pend_alpha = 1.f;
+      }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      const float mneg = -m * sl2;
+      const uint64_t mnegx2 = pack2(mneg, mneg);
+      uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
+      uint32_t pk[16];
+      tmem_ld32(tS, va);
+      tmem_wait_ld(va);
+      tmem_ld32(tS + 32, vb);
+      exp32<true>(va, sl2x2, mnegx2, lsum, pk, mx4);
+      tmem_st16(tP, pk);
+      tmem_wait_ld(vb);
+      tmem_ld32(tS + 64, va);
+      exp32<true>(vb, sl2x2, mnegx2, lsum, pk, mx4);
+      tmem_st16(tP + 16, pk);
+      tmem_wait_ld(va);
+      tmem_ld32(tS + 96, vb);
+      exp32<true>(va, sl2x2, mnegx2, lsum, pk, mx4);
+      tmem_st16(tP + 32, pk);
+      tmem_wait_ld(vb);
+      exp32<true>(vb, sl2x2, mnegx2, lsum, pk, mx4);
+      tmem_st16(tP + 48, pk);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      if (__any_sync(0xffffffffu, (mx - m) * sl2 > kSpecLimit)) return false;   // redo (whole warp)
+      float a0, a1, b0, b1;
+      unpack2(add2(lsum[0], lsum[1]), a0, a1);
+      unpack2(add2(lsum[2], lsum[3]), b0, b1);
+      l += (a0 + a1) + (b0 + b1);
+      if (mx > m + kLazy) {
+        pending = true;
+        pend_alpha = ex2((m - mx) * sl2);
+        pend_m = mx;
+      }
+      return true;
     };
 
     for (int j = 0; j < ntiles && ok; ++j) {
@@ -500,7 +627,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         tmem_wait_st();
       }
-      tile(j);
+      if (j == 0 || !spec_tile(j)) {
+        tile(j);
+      }
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bar->p_full[t]);

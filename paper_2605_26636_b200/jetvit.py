@@ -15,7 +15,8 @@ JV_OK, JV_ERR_INVALID_ARG, JV_ERR_UNSUPPORTED, JV_ERR_WORKSPACE, JV_ERR_CUDA, JV
 JV_F32, JV_BF16 = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libjetvit.so")
+# JETVIT_LIB selects another build of the same library (e.g. one compiled with other tuning macros)
+LIB_PATH = os.environ.get("JETVIT_LIB") or os.path.join(_HERE, "libjetvit.so")
 
 
 class JvShape(ctypes.Structure):
