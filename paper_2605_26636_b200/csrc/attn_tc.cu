@@ -8,18 +8,20 @@
 // the grid arrive as zeros from TMA's out-of-bounds fill and are masked to -inf before
 // the softmax; query rows outside the grid / window are never stored.
 //
-// Per CTA: two 128-row query tiles (ping-pong) against all key tiles of their
-// window.  Warp roles:
+// Per CTA: two 128-row query tiles against all key tiles of their window.  Warp roles:
 //   warp 0        TMA producer: Q tiles once, then K and V tiles through 3-stage rings
-//   warp 1        MMA issuer (one elected thread): S_t = Q_t K^T (SS, M128 N128 K64),
-//                 O_t += P_t V (A = P from tensor memory, B = V MN-major, M128 N64 K128)
+//   warps 1, 2    MMA issuers (one elected lane each; warp 1 + t serves query tile t), in steps of 64 keys:
+//                 S_t = Q_t K^T (operands in smem, M128 N64 K64),
+//                 O_t += P_t V (A = P from tensor memory, B = V MN-major, M128 N64 K64)
 //   warps 4-7     softmax of query tile 0   } one thread per query row: fp32 online
 //   warps 8-11    softmax of query tile 1   } softmax (exp2 domain, lazy rescale),
 //                 P as bf16 back into tensor memory, final 1/l scaling and the store.
-// While one tile's softmax runs on the ALUs, the tensor pipe works on the other tile.
+// Scores and probabilities are double-buffered per query tile, so the score MMA of step
+// u + 2 is issued as soon as the probabilities of step u are published and the softmax
+// warps never wait for the tensor pipe in steady state.
 //
-// Tensor memory (512 columns): S0 [0,128) S1 [128,256) O0 [256,320) O1 [320,384)
-// P0 [384,448) P1 [448,512).
+// Tensor memory (512 columns): scores S(t, b) 4 x 64 in [0, 256), accumulators O(t) 2 x 64
+// in [256, 384), probabilities P(t, b) 4 x 32 in [384, 512).
 //
 // Every mbarrier wait is bounded: a wait that runs out sets the device status word,
 // raises a CTA-wide abort flag, and every role falls through to the common teardown
@@ -37,6 +39,8 @@ constexpr int kTileBytes = kTile * kD * 2; // 16 KB
 constexpr int kStages = 3;
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kSub = 64;                    // keys per softmax / MMA step: half a key tile
+// Tensor-memory columns: S(t, b) at kColS + (2 t + b) * 64, O(t) at kColO + 64 t, P(t, b) at kColP + (2 t + b) * 32
 constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
@@ -56,7 +60,7 @@ struct TcParams {
 struct __align__(8) Barriers {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], p_full[2], o_full[2];
+  uint64_t s_full[2][2], p_full[2][2], pv_done[2][2], o_full[2];
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -135,7 +139,6 @@ __device__ __forceinline__ bool elect_one() {
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   if (elect_one())
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-  __syncwarp();
 }
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
@@ -301,7 +304,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 constexpr uint32_t idesc(uint32_t M, uint32_t N, uint32_t b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
-constexpr uint32_t kIdescQK = idesc(kTile, kTile, 0);
+constexpr uint32_t kIdescQK = idesc(kTile, kSub, 0);
 constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
 
 // ---- the kernel ------------------------------------------------------------------
@@ -313,7 +316,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
   const uint32_t sQ = smem_u32(smem), sK = sQ + 2 * kTileBytes, sV = sK + kStages * kTileBytes;
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // broadcast from lane 0: lets the compiler keep everything derived from the warp index uniform
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const int bh = blockIdx.z;
   const int wy = blockIdx.y / p.nwx, wx = blockIdx.y % p.nwx;
   const int x0 = wx * p.win_w, y0 = wy * p.win_h;
@@ -334,16 +338,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     mbar_init(&bar->q_full, 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
-      mbar_init(&bar->k_empty[s], 1);
+      mbar_init(&bar->k_empty[s], 2);     // one commit from each MMA issuer warp
       mbar_init(&bar->v_full[s], 1);
-      mbar_init(&bar->v_empty[s], 1);
+      mbar_init(&bar->v_empty[s], 2);
     }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&bar->s_full[t], 1);
-      mbar_init(&bar->p_full[t], 128);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(&bar->s_full[t][b], 1);
+        mbar_init(&bar->p_full[t][b], 128);
+        mbar_init(&bar->pv_done[t][b], 1);
+      }
       mbar_init(&bar->o_full[t], 1);
     }
-    mbar_init(&bar->drain, 1);
+    mbar_init(&bar->drain, 2);
     bar->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -357,7 +364,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = bar->tmem_base;
+  const uint32_t tmem = __shfl_sync(0xffffffffu, bar->tmem_base, 0);   // warp-uniform, and known to be
 
   // Warps 0 and 1 run their loops with all 32 lanes (waits included) so that stage counters,
   // addresses and descriptors stay warp-uniform; only the TMA / tcgen05 instructions themselves
@@ -399,47 +406,62 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int j = max(0, issued - kStages); j < issued; ++j)
         while (!mbar_try(&bar->v_full[j % kStages], (j / kStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
     }
-  } else if (warp == 1) {
-    // ================= MMA issuer =================
+  } else if (warp == 1 || warp == 2) {
+    // ================= MMA issuers: warp 1 serves query tile 0, warp 2 query tile 1 =================
+    // Per query tile t the work is a stream of 64-key steps u = 2 j + h (key tile j, half h):
+    //   S(t, u) = Q_t K_u^T  into score buffer h     (4 MMAs, M128 N64 K16, operands in smem)
+    //   O_t   += P(t, u) V_u                          (4 MMAs, M128 N64 K16, A = P in tensor memory)
+    // With two score buffers per query tile, S(t, u + 2) is issued as soon as P(t, u) has been
+    // published (its buffer is free then), so the softmax of step u + 1 never waits for the
+    // tensor pipe: S(t, u + 1) was issued one step earlier.  Each stream is a chain of
+    // wait -> issue -> commit latencies, so the two streams run in warps of their own.
+    // pv_done[t][h] (one phase per key tile) tells the softmax warps that P(t, h) may be
+    // overwritten and, on the rare rescale, that O is quiescent.
+    const int t = warp - 1;
     bool ok = warp_wait(&bar->q_full, 0, bar, p.status);
-    auto issue_qk = [&](int t, int stage) {
-      const uint32_t kb = sK + stage * kTileBytes, qb = sQ + t * kTileBytes;
+    auto issue_qk = [&](int stage, int h) {
+      const uint32_t kb = sK + stage * kTileBytes + h * (kSub * kD * 2), qb = sQ + t * kTileBytes;
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks)
-        mma_ss(tmem + kColS + t * kTile, smem_desc(qb + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
-      tc_commit(&bar->s_full[t]);
+        mma_ss(tmem + kColS + (2 * t + h) * kSub, smem_desc(qb + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
+      tc_commit(&bar->s_full[t][h]);
     };
     if (ok) ok = warp_wait(&bar->k_full[0], 0, bar, p.status);
     if (ok) {
       tc_fence_after();
       issue_qk(0, 0);
-      issue_qk(1, 0);
+      issue_qk(0, 1);
       tc_commit(&bar->k_empty[0]);
     }
     int s = 0, s1 = 1 % kStages;            // ring stage of key tile j and of key tile j + 1
     uint32_t ph = 0, ph1 = (kStages == 1);  // and their "full" parities
     for (int j = 0; j < ntiles && ok; ++j) {
-      ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
-      for (int t = 0; t < 2 && ok; ++t) {
-        ok = warp_wait(&bar->p_full[t], j & 1, bar, p.status);
+      const bool last = j + 1 == ntiles;
+      for (int h = 0; h < 2 && ok; ++h) {
+        ok = warp_wait(&bar->p_full[t][h], j & 1, bar, p.status);
         if (!ok) break;
-        tc_fence_after();
-        const uint32_t vb = sV + s * kTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < kTile / 16; ++ks)
-          mma_ts(tmem + kColO + t * kD, tmem + kColP + t * (kTile / 2) + ks * 8, smem_desc(vb + ks * 2048), kIdescPV,
-                 (j > 0 || ks > 0) ? 1u : 0u);
-        if (j + 1 < ntiles) {
-          if (t == 0) {
+        // Scores first: S(t, u + 2) is what the softmax warps will be waiting for next.
+        if (!last) {
+          if (h == 0) {
             ok = warp_wait(&bar->k_full[s1], ph1, bar, p.status);
             if (!ok) break;
-            tc_fence_after();
           }
-          issue_qk(t, s1);
-          if (t == 1) tc_commit(&bar->k_empty[s1]);
-        } else {
-          tc_commit(&bar->o_full[t]);
+          tc_fence_after();
+          issue_qk(s1, h);
+          if (h == 1) tc_commit(&bar->k_empty[s1]);
         }
+        if (h == 0) {
+          ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
+          if (!ok) break;
+        }
+        tc_fence_after();
+        const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
+#pragma unroll
+        for (int ks = 0; ks < kSub / 16; ++ks)
+          mma_ts(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, smem_desc(vb + ks * 2048),
+                 kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(&bar->pv_done[t][h]);
+        if (last && h == 1) tc_commit(&bar->o_full[t]);
       }
       if (ok) tc_commit(&bar->v_empty[s]);
       if (++s == kStages) { s = 0; ph ^= 1; }
@@ -457,127 +479,75 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const int t = (warp - 4) >> 2;                 // query tile of this warpgroup
     const int row = ((warp & 3) << 5) + lane;      // row of the tile == tensor-memory lane
     const uint32_t lane_base = (uint32_t)((warp & 3) << 5) << 16;
-    const uint32_t tS = tmem + lane_base + kColS + t * kTile;
+    const uint32_t tS = tmem + lane_base + kColS + 2 * t * kSub;          // + h * kSub
     const uint32_t tO = tmem + lane_base + kColO + t * kD;
-    const uint32_t tP = tmem + lane_base + kColP + t * (kTile / 2);
+    const uint32_t tP = tmem + lane_base + kColP + 2 * t * (kSub / 2);    // + h * kSub / 2
     const float sl2 = p.scale_log2;
-    const float kLazy = 8.f / sl2;                 // rescale only when the max grew by > 2^8
+    const float kLazy = 8.f / sl2;                 // the reference maximum moves only when it grew by > 2^8
     float m = -INFINITY, l = 0.f;
     bool ok = true;
 
     const uint64_t sl2x2 = pack2(sl2, sl2);
     const int lg_bw = 31 - __clz(p.box_w);          // box_w is a power of two
 
-    // One key tile: two passes over the 128 scores of this thread's row (maximum, then
-    // exponentials), reading tensor memory 32 columns at a time with the next read in flight.
-    auto tile = [&](int j) {
+    // o_scale: factor the accumulator O has to be multiplied by before this step's P V is added.
+    float o_scale = 1.f;
+
+    // One 64-key step in two passes over this thread's row: maximum first, then exponentials.
+    auto two_pass = [&](uint32_t tSb, uint32_t tPb) {
       uint32_t va[32], vb[32];
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      tmem_ld32(tS, va);
+      tmem_ld32(tSb, va);
       tmem_wait_ld(va);
-      tmem_ld32(tS + 32, vb);
+      tmem_ld32(tSb + 32, vb);
       max32(va, mx4);
       tmem_wait_ld(vb);
-      tmem_ld32(tS + 64, va);
       max32(vb, mx4);
-      tmem_wait_ld(va);
-      tmem_ld32(tS + 96, vb);
-      max32(va, mx4);
-      tmem_wait_ld(vb);
-      tmem_ld32(tS, va);                             // first read of pass 2
-      max32(vb, mx4);
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));   // finite: >= 1 valid key per tile
-
-      float alpha = 1.f;
-      bool rescale = false;
-      if (mx > m + kLazy) {          // always true on the first tile (m = -inf)
-        alpha = ex2((m - mx) * sl2); // first tile: exp2(-inf) = 0
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      if (mx > m + kLazy) {          // always true on the first step (m = -inf, mx finite)
+        const float alpha = ex2((m - mx) * sl2);   // first step: exp2(-inf) = 0
         l *= alpha;
+        o_scale *= alpha;
         m = mx;
-        rescale = j > 0;
-      }
-      tmem_wait_ld(va);
-      if (__any_sync(0xffffffffu, rescale)) {
-        // PV of the previous key tile has retired (its commit preceded this S tile's): O is ours
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          tmem_ld32(tO + 32 * c, vb);
-          tmem_wait_ld(vb);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * alpha);
-          tmem_st32(tO + 32 * c, vb);
-        }
       }
       const float mneg = -m * sl2;
       const uint64_t mnegx2 = pack2(mneg, mneg);
       uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
       uint32_t pk[16];
-      tmem_ld32(tS + 32, vb);
       exp32<false>(va, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP, pk);
-      tmem_wait_ld(vb);
-      tmem_ld32(tS + 64, va);
+      tmem_st16(tPb, pk);
       exp32<false>(vb, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP + 16, pk);
-      tmem_wait_ld(va);
-      tmem_ld32(tS + 96, vb);
-      exp32<false>(va, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP + 32, pk);
-      tmem_wait_ld(vb);
-      exp32<false>(vb, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP + 48, pk);
+      tmem_st16(tPb + 16, pk);
       float a0, a1, b0, b1;
       unpack2(add2(lsum[0], lsum[1]), a0, a1);
       unpack2(add2(lsum[2], lsum[3]), b0, b1);
       l += (a0 + a1) + (b0 + b1);
     };
 
-    // Later key tiles, one pass: the exponentials are taken against the maximum known so far
-    // while the tile's own maximum is tracked on the side.  Any reference value gives the same
-    // softmax as long as nothing overflows, so a larger maximum only matters for the tiles
-    // that follow: O and l are rescaled at the start of the next tile, once this tile's PV
-    // has retired.  A tile whose scores exceed the reference by more than 2^kSpecLimit is redone
-    // with the two-pass routine above (P has not been published yet).
+    // Later steps, one pass: the exponentials are taken against the maximum known so far while
+    // the step's own maximum is tracked on the side.  Any reference value gives the same
+    // softmax as long as nothing overflows, so a larger maximum only matters for the steps
+    // that follow: it becomes the reference of the next step, which rescales l and O.
+    // A step whose scores exceed the reference by more than 2^kSpecLimit is redone with the
+    // two-pass routine (P has not been published yet).
     constexpr float kSpecLimit = 64.f;
     float pend_alpha = 1.f, pend_m = 0.f;
     bool pending = false;
-    auto spec_tile = [&](int j) -> bool {
+    auto one_pass = [&](uint32_t tSb, uint32_t tPb) -> bool {
       uint32_t va[32], vb[32];
-      if (__any_sync(0xffffffffu, pending)) {
-        // the previous tile's PV has retired (its commit preceded this S tile's): O is ours
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          tmem_ld32(tO + 32 * c, vb);
-          tmem_wait_ld(vb);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) vb[i] = __float_as_uint(__uint_as_float(vb[i]) * pend_alpha);
-          tmem_st32(tO + 32 * c, vb);
-        }
-        if (pending) { l *= pend_alpha; m = pend_m; }
-        pending = false;
-        pend_alpha = 1.f;
-      }
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       const float mneg = -m * sl2;
       const uint64_t mnegx2 = pack2(mneg, mneg);
       uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
       uint32_t pk[16];
-      tmem_ld32(tS, va);
+      tmem_ld32(tSb, va);
       tmem_wait_ld(va);
-      tmem_ld32(tS + 32, vb);
+      tmem_ld32(tSb + 32, vb);
       exp32<true>(va, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP, pk);
-      tmem_wait_ld(vb);
-      tmem_ld32(tS + 64, va);
-      exp32<true>(vb, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP + 16, pk);
-      tmem_wait_ld(va);
-      tmem_ld32(tS + 96, vb);
-      exp32<true>(va, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP + 32, pk);
+      tmem_st16(tPb, pk);
       tmem_wait_ld(vb);
       exp32<true>(vb, sl2x2, mnegx2, lsum, pk, mx4);
-      tmem_st16(tP + 48, pk);
+      tmem_st16(tPb + 16, pk);
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       if (__any_sync(0xffffffffu, (mx - m) * sl2 > kSpecLimit)) return false;   // redo (whole warp)
       float a0, a1, b0, b1;
@@ -592,47 +562,76 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       return true;
     };
 
-    for (int j = 0; j < ntiles && ok; ++j) {
+    const int nsteps = 2 * ntiles;
+    for (int u = 0; u < nsteps && ok; ++u) {
+      const int j = u >> 1, h = u & 1;
       // warp-uniform outcome: the tensor-memory accesses below are warp-collective
-      ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t], j & 1, bar, p.status));
+      ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], j & 1, bar, p.status));
       if (!ok) break;
       tc_fence_after();
-      // which keys of this tile exist?  vx, vy: valid extent of the box along x and y
+      // P(t, h) is free again once P V of step u - 2 has read it (long done in steady state)
+      if (u >= 2) {
+        ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t][h], (j - 1) & 1, bar, p.status));
+        if (!ok) break;
+      }
+      const uint32_t tSb = tS + h * kSub, tPb = tP + h * (kSub / 2);
+      o_scale = 1.f;
+      if (pending) {                 // the previous step raised the maximum: new reference from here on
+        l *= pend_alpha;
+        o_scale = pend_alpha;
+        m = pend_m;
+        pending = false;
+      }
+      // which keys of this step exist?  vx, vy: valid extent of the key tile's box along x and y
       const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
       if (vx < p.box_w || vy < p.box_h) {
         // Edge tile: overwrite the scores of keys that do not exist (outside the grid or the
-        // window) with -inf in tensor memory, then treat the tile like any other.
+        // window) with -inf in tensor memory, then treat the step like any other.
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
+          const int k0 = 64 * h + 32 * c;            // first of the 32 keys, as an index into the box
           uint32_t bits = 0;
           if (p.box_w >= 32) {                       // the 32 keys lie in one box row
-            const int ly = (32 * c) >> lg_bw, lx0 = (32 * c) & (p.box_w - 1);
+            const int ly = k0 >> lg_bw, lx0 = k0 & (p.box_w - 1);
             const int n = min(32, vx - lx0);
             if (ly < vy && n > 0) bits = n >= 32 ? 0xffffffffu : ((1u << n) - 1u);
           } else {                                   // 32 / box_w whole box rows
             const uint32_t rowbits = (1u << min(vx, p.box_w)) - 1u;
-            const int ly0 = (32 * c) >> lg_bw;
+            const int ly0 = k0 >> lg_bw;
             for (int r = 0; r < (32 >> lg_bw); ++r)
               if (ly0 + r < vy) bits |= rowbits << (r << lg_bw);
           }
           if (bits != 0xffffffffu) {                 // warp-uniform: the mask depends on the tile only
             uint32_t v[32];
-            tmem_ld32(tS + 32 * c, v);
+            tmem_ld32(tSb + 32 * c, v);
             tmem_wait_ld(v);
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (!((bits >> i) & 1u)) v[i] = kNegInf;   // exp2(-inf) = 0 and -inf never wins the maximum
-            tmem_st32(tS + 32 * c, v);
+            tmem_st32(tSb + 32 * c, v);
           }
         }
         tmem_wait_st();
       }
-      if (j == 0 || !spec_tile(j)) {
-        tile(j);
+      if (u == 0 || !one_pass(tSb, tPb)) two_pass(tSb, tPb);
+      if (u > 0 && __any_sync(0xffffffffu, o_scale != 1.f)) {
+        // O may be touched once P V of step u - 1 has retired; the next P V waits for our P.
+        ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t][h ^ 1], ((u - 1) >> 1) & 1, bar, p.status));
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tO + 32 * c, v);
+          tmem_wait_ld(v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * o_scale);
+          tmem_st32(tO + 32 * c, v);
+        }
       }
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bar->p_full[t]);
+      mbar_arrive(&bar->p_full[t][h]);
     }
 
     ok = __all_sync(0xffffffffu, ok && mbar_wait(&bar->o_full[t], 0, bar, p.status));
