@@ -60,7 +60,7 @@ struct TcParams {
 struct __align__(8) Barriers {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2][2], p_full[2][2], pv_done[2][2], o_full[2];
+  uint64_t s_full[2][2], p_full[2][2], pv_done[2], o_full[2];
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -90,6 +90,17 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
   asm volatile(
       "{\n.reg .pred p;\n"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Non-blocking test of a phase: used to take a barrier's round trip off the critical path
+// (test early, consume the answer later, fall back to mbar_wait if it was not yet complete).
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
       "selp.u32 %0, 1, 0, p;\n}\n"
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
@@ -346,8 +357,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int b = 0; b < 2; ++b) {
         mbar_init(&bar->s_full[t][b], 1);
         mbar_init(&bar->p_full[t][b], 128);
-        mbar_init(&bar->pv_done[t][b], 1);
       }
+      mbar_init(&bar->pv_done[t], 1);
       mbar_init(&bar->o_full[t], 1);
     }
     mbar_init(&bar->drain, 2);
@@ -415,8 +426,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     // published (its buffer is free then), so the softmax of step u + 1 never waits for the
     // tensor pipe: S(t, u + 1) was issued one step earlier.  Each stream is a chain of
     // wait -> issue -> commit latencies, so the two streams run in warps of their own.
-    // pv_done[t][h] (one phase per key tile) tells the softmax warps that P(t, h) may be
-    // overwritten and, on the rare rescale, that O is quiescent.
+    // The commit of S(t, u + 2) follows the issue of P V (t, u): seeing those scores tells the
+    // softmax warps that P(t, h) may be overwritten; seeing S(t, u + 1) tells them that
+    // P V (t, u - 1) has retired and O is quiescent (pv_done does that on the last key tile).
     const int t = warp - 1;
     bool ok = warp_wait(&bar->q_full, 0, bar, p.status);
     auto issue_qk = [&](int stage, int h) {
@@ -437,31 +449,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     uint32_t ph = 0, ph1 = (kStages == 1);  // and their "full" parities
     for (int j = 0; j < ntiles && ok; ++j) {
       const bool last = j + 1 == ntiles;
+      ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
       for (int h = 0; h < 2 && ok; ++h) {
         ok = warp_wait(&bar->p_full[t][h], j & 1, bar, p.status);
         if (!ok) break;
-        // Scores first: S(t, u + 2) is what the softmax warps will be waiting for next.
-        if (!last) {
-          if (h == 0) {
-            ok = warp_wait(&bar->k_full[s1], ph1, bar, p.status);
-            if (!ok) break;
-          }
-          tc_fence_after();
-          issue_qk(s1, h);
-          if (h == 1) tc_commit(&bar->k_empty[s1]);
-        }
-        if (h == 0) {
-          ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
-          if (!ok) break;
-        }
         tc_fence_after();
         const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
 #pragma unroll
         for (int ks = 0; ks < kSub / 16; ++ks)
           mma_ts(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, smem_desc(vb + ks * 2048),
                  kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
-        tc_commit(&bar->pv_done[t][h]);
-        if (last && h == 1) tc_commit(&bar->o_full[t]);
+        if (!last) {
+          if (h == 0) {
+            ok = warp_wait(&bar->k_full[s1], ph1, bar, p.status);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          issue_qk(s1, h);          // its commit also covers the P V just issued
+          if (h == 1) tc_commit(&bar->k_empty[s1]);
+        } else {
+          tc_commit(&bar->pv_done[t]);
+          if (h == 1) tc_commit(&bar->o_full[t]);
+        }
       }
       if (ok) tc_commit(&bar->v_empty[s]);
       if (++s == kStages) { s = 0; ph ^= 1; }
@@ -492,6 +501,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
     // o_scale: factor the accumulator O has to be multiplied by before this step's P V is added.
     float o_scale = 1.f;
+    unsigned rescale_vote = 0;        // warp-uniform: some lane has o_scale != 1
 
     // One 64-key step in two passes over this thread's row: maximum first, then exponentials.
     auto two_pass = [&](uint32_t tSb, uint32_t tPb) {
@@ -533,7 +543,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     constexpr float kSpecLimit = 64.f;
     float pend_alpha = 1.f, pend_m = 0.f;
     bool pending = false;
-    auto one_pass = [&](uint32_t tSb, uint32_t tPb) -> bool {
+    bool next_ready = false;          // answer of the early test of the next step's score barrier
+    auto one_pass = [&](uint32_t tSb, uint32_t tPb, uint64_t* next_bar, uint32_t next_parity) -> bool {
       uint32_t va[32], vb[32];
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       const float mneg = -m * sl2;
@@ -545,35 +556,43 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tmem_ld32(tSb + 32, vb);
       exp32<true>(va, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tPb, pk);
+      next_ready = mbar_test(next_bar, next_parity);   // round trip hidden behind the second half
       tmem_wait_ld(vb);
       exp32<true>(vb, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tPb + 16, pk);
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      if (__any_sync(0xffffffffu, (mx - m) * sl2 > kSpecLimit)) return false;   // redo (whole warp)
       float a0, a1, b0, b1;
       unpack2(add2(lsum[0], lsum[1]), a0, a1);
       unpack2(add2(lsum[2], lsum[3]), b0, b1);
+      const float grow = (mx - m) * sl2;              // log2 of the largest p of this step
+      // one vote for both rare cases: bit 1 = redo this step, bit 0 = some O needs rescaling
+      const unsigned flags = __reduce_or_sync(0xffffffffu, (grow > kSpecLimit ? 2u : 0u) | (o_scale != 1.f ? 1u : 0u));
+      if (flags & 2u) return false;                    // redo (whole warp); l untouched
       l += (a0 + a1) + (b0 + b1);
-      if (mx > m + kLazy) {
+      if (grow > 8.f) {                                // new reference from the next step on
         pending = true;
-        pend_alpha = ex2((m - mx) * sl2);
+        pend_alpha = ex2(-grow);
         pend_m = mx;
       }
+      rescale_vote = flags & 1u;
       return true;
     };
 
     const int nsteps = 2 * ntiles;
+    // Which key tiles have keys that do not exist?  A window narrower than the box makes every
+    // tile an edge tile; otherwise only the last tile of the window / sequence can be one.
+    const bool edge_all = (x_end - x0) < p.box_w && p.step_x == 0;
+    const int last_vx = x_end - (x0 + (ntiles - 1) * p.step_x), last_vy = y_end - (y0 + (ntiles - 1) * p.step_y);
+    const bool edge_last = last_vx < p.box_w || last_vy < p.box_h;
+    next_ready = mbar_test(&bar->s_full[t][0], 0);
     for (int u = 0; u < nsteps && ok; ++u) {
       const int j = u >> 1, h = u & 1;
       // warp-uniform outcome: the tensor-memory accesses below are warp-collective
-      ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], j & 1, bar, p.status));
-      if (!ok) break;
-      tc_fence_after();
-      // P(t, h) is free again once P V of step u - 2 has read it (long done in steady state)
-      if (u >= 2) {
-        ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t][h], (j - 1) & 1, bar, p.status));
+      if (!__all_sync(0xffffffffu, next_ready)) {
+        ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], j & 1, bar, p.status));
         if (!ok) break;
       }
+      tc_fence_after();
       const uint32_t tSb = tS + h * kSub, tPb = tP + h * (kSub / 2);
       o_scale = 1.f;
       if (pending) {                 // the previous step raised the maximum: new reference from here on
@@ -582,11 +601,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         m = pend_m;
         pending = false;
       }
-      // which keys of this step exist?  vx, vy: valid extent of the key tile's box along x and y
-      const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
-      if (vx < p.box_w || vy < p.box_h) {
+      if (edge_all || (edge_last && j == ntiles - 1)) {
         // Edge tile: overwrite the scores of keys that do not exist (outside the grid or the
         // window) with -inf in tensor memory, then treat the step like any other.
+        // vx, vy: valid extent of the key tile's box along x and y
+        const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
 #pragma unroll 1
         for (int c = 0; c < 2; ++c) {
           const int k0 = 64 * h + 32 * c;            // first of the 32 keys, as an index into the box
@@ -613,10 +632,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         tmem_wait_st();
       }
-      if (u == 0 || !one_pass(tSb, tPb)) two_pass(tSb, tPb);
-      if (u > 0 && __any_sync(0xffffffffu, o_scale != 1.f)) {
+      uint64_t* next_bar = &bar->s_full[t][h ^ 1];
+      const uint32_t next_parity = ((u + 1) >> 1) & 1;
+      if (u == 0 || !one_pass(tSb, tPb, next_bar, next_parity)) {
+        two_pass(tSb, tPb);
+        next_ready = false;
+        rescale_vote = __any_sync(0xffffffffu, o_scale != 1.f);
+      }
+      if (u > 0 && rescale_vote) {
         // O may be touched once P V of step u - 1 has retired; the next P V waits for our P.
-        ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t][h ^ 1], ((u - 1) >> 1) & 1, bar, p.status));
+        // The issuer commits S(t, u + 1) after issuing P V (u - 1), so that barrier tells us;
+        // on the last step there is no further S, and pv_done (committed after each P V of
+        // the last key tile) does.
+        if (u + 1 < nsteps)
+          ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, bar, p.status));
+        else
+          ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, bar, p.status));
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
@@ -629,6 +660,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           tmem_st32(tO + 32 * c, v);
         }
       }
+      if (u + 1 == nsteps) next_ready = true;   // nothing to wait for after the last step
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bar->p_full[t][h]);
