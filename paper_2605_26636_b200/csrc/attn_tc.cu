@@ -8,8 +8,9 @@
 // the grid arrive as zeros from TMA's out-of-bounds fill and are masked to -inf before
 // the softmax; query rows outside the grid / window are never stored.
 //
-// Per CTA: two 128-row query tiles against all key tiles of their window.  Warp roles:
-//   warp 0        TMA producer: Q tiles once, then K and V tiles through 3-stage rings
+// Persistent CTAs (one per SM) loop over work items; an item is two 128-row query tiles
+// against all key tiles of their window.  Warp roles:
+//   warp 0        TMA producer: Q tiles (two buffers), K and V tiles through 4-stage rings
 //   warps 1, 2    MMA issuers (one elected lane each; warp 1 + t serves query tile t), in steps of 64 keys:
 //                 S_t = Q_t K^T (operands in smem, M128 N64 K64),
 //                 O_t += P_t V (A = P from tensor memory, B = V MN-major, M128 N64 K64)
@@ -36,7 +37,7 @@ namespace {
 constexpr int kD = 64;
 constexpr int kTile = 128;                 // tokens per tile (MMA M and key-tile N)
 constexpr int kTileBytes = kTile * kD * 2; // 16 KB
-constexpr int kStages = 3;
+constexpr int kStages = 4;                 // K and V ring depth
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSub = 64;                    // keys per softmax / MMA step: half a key tile
@@ -53,19 +54,43 @@ struct TcParams {
   int box_w, box_h;      // tile box: box_w * box_h == 128
   int step_x, step_y;    // origin step from one tile of a window to the next
   int nwx;               // windows per grid row
+  int nwin;              // windows per (batch, head)
+  int qpairs;            // pairs of query tiles per window (by the full window height)
+  int total_items;       // work items: (batch*head, window, query-tile pair), pair index fastest
   float scale_log2;      // softmax scale * log2(e)
 };
 
+// One work item of the persistent loop: two query tiles of one window of one (batch, head).
+struct Item {
+  int bh, x0, y0, x_end, y_end;   // window origin and valid end (exclusive) in the token grid
+  int ntiles;                     // key tiles of the window
+  int qt0;                        // first of the two query tiles
+};
+__device__ __forceinline__ Item decode_item(const TcParams& p, int i) {
+  Item it;
+  const int qp = i % p.qpairs, r = i / p.qpairs;
+  const int win = r % p.nwin;
+  it.bh = r / p.nwin;
+  const int wy = win / p.nwx, wx = win % p.nwx;
+  it.x0 = wx * p.win_w;
+  it.y0 = wy * p.win_h;
+  it.x_end = min(it.x0 + p.win_w, p.gridW);
+  it.y_end = min(it.y0 + p.win_h, p.gridH);
+  it.ntiles = p.step_x ? (it.x_end - it.x0 + kTile - 1) / kTile : (it.y_end - it.y0 + p.box_h - 1) / p.box_h;
+  it.qt0 = 2 * qp;                // an item with qt0 >= ntiles (short edge window) is empty: every role skips it
+  return it;
+}
+
 // ---- shared-memory layout -------------------------------------------------------
 struct __align__(8) Barriers {
-  uint64_t q_full;
+  uint64_t q_full[2], q_empty[2];                     // the two query buffers (items alternate)
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2][2], p_full[2][2], pv_done[2], o_full[2];
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
-constexpr size_t kSmemTiles = (2 + 2 * kStages) * (size_t)kTileBytes;          // Q0 Q1 K[3] V[3]
+constexpr size_t kSmemTiles = (4 + 2 * kStages) * (size_t)kTileBytes;          // Q[2][2] K[kStages] V[kStages]
 constexpr size_t kSmemBytes = kSmemTiles + sizeof(Barriers) + 1024;            // + alignment slack
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -319,24 +344,22 @@ constexpr uint32_t kIdescQK = idesc(kTile, kSub, 0);
 constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
 
 // ---- the kernel ------------------------------------------------------------------
+// Persistent: CTA c works on items c, c + gridDim.x, ...  Every role walks the same item
+// sequence on its own; ring stages and barrier parities follow running counters (key tiles
+// and items seen so far), so the pipeline runs straight through item boundaries: the next
+// item's Q, K and V are already in flight, and its first scores already issued, while the
+// current item is being finished and stored.
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                const __grid_constant__ CUtensorMap mapV, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
-  const uint32_t sQ = smem_u32(smem), sK = sQ + 2 * kTileBytes, sV = sK + kStages * kTileBytes;
+  // Q buffer b holds the two query tiles of an item at sQ + b * 2 tiles
+  const uint32_t sQ = smem_u32(smem), sK = sQ + 4 * kTileBytes, sV = sK + kStages * kTileBytes;
 
   // broadcast from lane 0: lets the compiler keep everything derived from the warp index uniform
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
-  const int bh = blockIdx.z;
-  const int wy = blockIdx.y / p.nwx, wx = blockIdx.y % p.nwx;
-  const int x0 = wx * p.win_w, y0 = wy * p.win_h;
-  const int x_end = min(x0 + p.win_w, p.gridW), y_end = min(y0 + p.win_h, p.gridH);
-  // key tiles of this window, and the two query tiles of this CTA
-  const int ntiles = p.step_x ? (x_end - x0 + kTile - 1) / kTile : (y_end - y0 + p.box_h - 1) / p.box_h;
-  const int qt0 = 2 * blockIdx.x;
-  if (qt0 >= ntiles) return;   // uniform: nothing of this window left for this CTA
 
   // Once any CTA has flagged a timeout the rest of the grid (and later launches, until the
   // host reads the status) leave at once instead of each running into the same limit.
@@ -346,10 +369,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   __syncthreads();
 
   if (threadIdx.x == 0) {
-    mbar_init(&bar->q_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&bar->q_full[b], 1);
+      mbar_init(&bar->q_empty[b], 2);     // one commit from each MMA issuer warp
+    }
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bar->k_full[s], 1);
-      mbar_init(&bar->k_empty[s], 2);     // one commit from each MMA issuer warp
+      mbar_init(&bar->k_empty[s], 2);
       mbar_init(&bar->v_full[s], 1);
       mbar_init(&bar->v_empty[s], 2);
     }
@@ -375,106 +401,145 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = __shfl_sync(0xffffffffu, bar->tmem_base, 0);   // warp-uniform, and known to be
+  const uint32_t tmem = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
 
-  // Warps 0 and 1 run their loops with all 32 lanes (waits included) so that stage counters,
+  const int item0 = blockIdx.x, item_step = gridDim.x;
+
+  // Warps 0, 1 and 2 run their loops with all 32 lanes (waits included) so that counters,
   // addresses and descriptors stay warp-uniform; only the TMA / tcgen05 instructions themselves
   // are issued by one elected lane (always the same one: the election is deterministic for a
   // full warp, and tcgen05.commit has to come from the thread that issued the MMAs).
   if (warp == 0) {
     // ================= TMA producer =================
-    if (elect_one()) {
-      mbar_expect_tx(&bar->q_full, 2 * kTileBytes);
-      for (int t = 0; t < 2; ++t)
-        tma_load_4d(sQ + t * kTileBytes, &mapQ, &bar->q_full, 0, x0 + (qt0 + t) * p.step_x,
-                    y0 + (qt0 + t) * p.step_y, bh);
-    }
-    __syncwarp();
     bool ok = true;
-    int issued = 0, s = 0;
-    uint32_t par = 1;                       // parity of the "empty" phase this pass over the ring waits for
-    for (int j = 0; j < ntiles; ++j) {
-      ok = warp_wait(&bar->k_empty[s], par, bar, p.status);
+    int n = 0;                 // items seen (non-empty ones): Q buffer n & 1
+    int s = 0;                 // ring stage of the next key tile
+    uint32_t par = 1;          // parity of the "empty" phase this pass over the ring waits for
+    int issued_v = 0;          // for the abort path: V copies issued so far
+    for (int i = item0; i < p.total_items && ok; i += item_step) {
+      const Item it = decode_item(p, i);
+      if (it.qt0 >= it.ntiles) continue;
+      const int qb = n & 1;
+      ok = warp_wait(&bar->q_empty[qb], ((n >> 1) & 1) ^ 1, bar, p.status);
       if (!ok) break;
       if (elect_one()) {
-        mbar_expect_tx(&bar->k_full[s], kTileBytes);
-        tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, x0 + j * p.step_x, y0 + j * p.step_y, bh);
+        mbar_expect_tx(&bar->q_full[qb], 2 * kTileBytes);
+        for (int t = 0; t < 2; ++t)
+          tma_load_4d(sQ + (2 * qb + t) * kTileBytes, &mapQ, &bar->q_full[qb], 0, it.x0 + (it.qt0 + t) * p.step_x,
+                      it.y0 + (it.qt0 + t) * p.step_y, it.bh);
       }
       __syncwarp();
-      ok = warp_wait(&bar->v_empty[s], par, bar, p.status);
-      if (!ok) break;
-      if (elect_one()) {
-        mbar_expect_tx(&bar->v_full[s], kTileBytes);
-        tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, x0 + j * p.step_x, y0 + j * p.step_y, bh);
+      for (int j = 0; j < it.ntiles; ++j) {
+        ok = warp_wait(&bar->k_empty[s], par, bar, p.status);
+        if (!ok) break;
+        if (elect_one()) {
+          mbar_expect_tx(&bar->k_full[s], kTileBytes);
+          tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
+        }
+        __syncwarp();
+        ok = warp_wait(&bar->v_empty[s], par, bar, p.status);
+        if (!ok) break;
+        if (elect_one()) {
+          mbar_expect_tx(&bar->v_full[s], kTileBytes);
+          tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
+        }
+        __syncwarp();
+        ++issued_v;
+        if (++s == kStages) { s = 0; par ^= 1; }
       }
-      __syncwarp();
-      issued = j + 1;
-      if (++s == kStages) { s = 0; par ^= 1; }
+      ++n;
     }
     if (!ok && lane == 0) {
       // let the copies still in flight land before the CTA leaves (bounded by the same limit)
       const unsigned long long t0 = globaltimer();
-      for (int j = max(0, issued - kStages); j < issued; ++j)
-        while (!mbar_try(&bar->v_full[j % kStages], (j / kStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
+      for (int g = max(0, issued_v - kStages); g < issued_v; ++g)
+        while (!mbar_try(&bar->v_full[g % kStages], (g / kStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
     }
   } else if (warp == 1 || warp == 2) {
     // ================= MMA issuers: warp 1 serves query tile 0, warp 2 query tile 1 =================
-    // Per query tile t the work is a stream of 64-key steps u = 2 j + h (key tile j, half h):
-    //   S(t, u) = Q_t K_u^T  into score buffer h     (4 MMAs, M128 N64 K16, operands in smem)
-    //   O_t   += P(t, u) V_u                          (4 MMAs, M128 N64 K16, A = P in tensor memory)
-    // With two score buffers per query tile, S(t, u + 2) is issued as soon as P(t, u) has been
-    // published (its buffer is free then), so the softmax of step u + 1 never waits for the
-    // tensor pipe: S(t, u + 1) was issued one step earlier.  Each stream is a chain of
-    // wait -> issue -> commit latencies, so the two streams run in warps of their own.
-    // The commit of S(t, u + 2) follows the issue of P V (t, u): seeing those scores tells the
-    // softmax warps that P(t, h) may be overwritten; seeing S(t, u + 1) tells them that
-    // P V (t, u - 1) has retired and O is quiescent (pv_done does that on the last key tile).
+    // Per query tile t the work is a stream of 64-key steps (key tile G of the CTA's whole run,
+    // half h), running on through item boundaries:
+    //   S(t, G, h) = Q_t K^T  into score buffer h     (4 MMAs, M128 N64 K16, operands in smem)
+    //   O_t      += P(t, G, h) V                       (4 MMAs, M128 N64 K16, A = P in tensor memory)
+    // With two score buffers per query tile, the scores of tile G + 1 (half h) are issued as soon
+    // as P(t, G, h) has been published (its buffer is free then), so the softmax of the step in
+    // between never waits for the tensor pipe.  Each stream is a chain of wait -> issue ->
+    // commit latencies, so the two streams run in warps of their own.
+    // The commit that publishes scores follows the issue of the preceding P V: seeing the
+    // scores of step u + 2 tells the softmax warps that P V (u) has read its probabilities, and
+    // seeing those of step u + 1 that P V (u - 1) has retired and O is quiescent (pv_done does
+    // that at the very end of the run, where no further scores are issued).
     const int t = warp - 1;
-    bool ok = warp_wait(&bar->q_full, 0, bar, p.status);
-    auto issue_qk = [&](int stage, int h) {
-      const uint32_t kb = sK + stage * kTileBytes + h * (kSub * kD * 2), qb = sQ + t * kTileBytes;
+    auto next_item = [&](int i) {           // next non-empty item after index i, or -1
+      for (i += item_step; i < p.total_items; i += item_step) {
+        const Item it = decode_item(p, i);
+        if (it.qt0 < it.ntiles) return i;
+      }
+      return -1;
+    };
+    int cur = item0 - item_step;
+    cur = next_item(cur);
+    bool ok = cur >= 0;
+    int n = 0;                              // items seen: Q buffer n & 1, parity (n >> 1) & 1
+    int s = 0, s1 = 0;                      // ring stage of the P V key tile and of the score key tile
+    uint32_t ph = 0, ph1 = 0;               // and their "full" parities
+    uint32_t g_par = 0;                     // parity of the global key-tile index of the P V tile
+
+    // scores of half h of local tile jq of the item in Q buffer qb (n_q-th item), key ring stage s1
+    auto issue_qk = [&](int h, int jq, int ntiles_q, int n_q) -> bool {
+      const int qb = n_q & 1;
+      if (h == 0) {
+        if (jq == 0 && !warp_wait(&bar->q_full[qb], (n_q >> 1) & 1, bar, p.status)) return false;
+        if (!warp_wait(&bar->k_full[s1], ph1, bar, p.status)) return false;
+        tc_fence_after();
+      }
+      const uint32_t kb = sK + s1 * kTileBytes + h * (kSub * kD * 2), qa = sQ + (2 * qb + t) * kTileBytes;
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks)
-        mma_ss(tmem + kColS + (2 * t + h) * kSub, smem_desc(qb + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
+        mma_ss(tmem + kColS + (2 * t + h) * kSub, smem_desc(qa + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
       tc_commit(&bar->s_full[t][h]);
-    };
-    if (ok) ok = warp_wait(&bar->k_full[0], 0, bar, p.status);
-    if (ok) {
-      tc_fence_after();
-      issue_qk(0, 0);
-      issue_qk(0, 1);
-      tc_commit(&bar->k_empty[0]);
-    }
-    int s = 0, s1 = 1 % kStages;            // ring stage of key tile j and of key tile j + 1
-    uint32_t ph = 0, ph1 = (kStages == 1);  // and their "full" parities
-    for (int j = 0; j < ntiles && ok; ++j) {
-      const bool last = j + 1 == ntiles;
-      ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
-      for (int h = 0; h < 2 && ok; ++h) {
-        ok = warp_wait(&bar->p_full[t][h], j & 1, bar, p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
-#pragma unroll
-        for (int ks = 0; ks < kSub / 16; ++ks)
-          mma_ts(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, smem_desc(vb + ks * 2048),
-                 kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
-        if (!last) {
-          if (h == 0) {
-            ok = warp_wait(&bar->k_full[s1], ph1, bar, p.status);
-            if (!ok) break;
-            tc_fence_after();
-          }
-          issue_qk(s1, h);          // its commit also covers the P V just issued
-          if (h == 1) tc_commit(&bar->k_empty[s1]);
-        } else {
-          tc_commit(&bar->pv_done[t]);
-          if (h == 1) tc_commit(&bar->o_full[t]);
-        }
+      if (h == 1) {
+        tc_commit(&bar->k_empty[s1]);
+        if (jq == ntiles_q - 1) tc_commit(&bar->q_empty[qb]);
+        if (++s1 == kStages) { s1 = 0; ph1 ^= 1; }
       }
-      if (ok) tc_commit(&bar->v_empty[s]);
-      if (++s == kStages) { s = 0; ph ^= 1; }
-      if (++s1 == kStages) { s1 = 0; ph1 ^= 1; }
+      return true;
+    };
+
+    Item it{};
+    if (ok) {
+      it = decode_item(p, cur);
+      ok = issue_qk(0, 0, it.ntiles, 0) && issue_qk(1, 0, it.ntiles, 0);
+    }
+    while (ok) {
+      const int nxt = next_item(cur);
+      Item itn{};
+      if (nxt >= 0) itn = decode_item(p, nxt);
+      for (int j = 0; j < it.ntiles && ok; ++j) {
+        ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
+        const bool last = j + 1 == it.ntiles;
+        for (int h = 0; h < 2 && ok; ++h) {
+          ok = warp_wait(&bar->p_full[t][h], g_par, bar, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
+#pragma unroll
+          for (int ks = 0; ks < kSub / 16; ++ks)
+            mma_ts(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, smem_desc(vb + ks * 2048),
+                   kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
+          if (last && h == 1) tc_commit(&bar->o_full[t]);
+          if (!last) ok = issue_qk(h, j + 1, it.ntiles, n);              // its commit also covers the P V just issued
+          else if (nxt >= 0) ok = issue_qk(h, 0, itn.ntiles, n + 1);     // first key tile of the next item
+          else tc_commit(&bar->pv_done[t]);
+        }
+        if (ok) tc_commit(&bar->v_empty[s]);
+        if (++s == kStages) { s = 0; ph ^= 1; }
+        g_par ^= 1;
+      }
+      if (nxt < 0) break;
+      cur = nxt;
+      it = itn;
+      ++n;
     }
     // Teardown: every MMA issued so far must have retired before tensor memory is released.
     tc_commit(&bar->drain);
@@ -578,119 +643,144 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       return true;
     };
 
-    const int nsteps = 2 * ntiles;
-    // Which key tiles have keys that do not exist?  A window narrower than the box makes every
-    // tile an edge tile; otherwise only the last tile of the window / sequence can be one.
-    const bool edge_all = (x_end - x0) < p.box_w && p.step_x == 0;
-    const int last_vx = x_end - (x0 + (ntiles - 1) * p.step_x), last_vy = y_end - (y0 + (ntiles - 1) * p.step_y);
-    const bool edge_last = last_vx < p.box_w || last_vy < p.box_h;
-    next_ready = mbar_test(&bar->s_full[t][0], 0);
-    for (int u = 0; u < nsteps && ok; ++u) {
-      const int j = u >> 1, h = u & 1;
-      // warp-uniform outcome: the tensor-memory accesses below are warp-collective
-      if (!__all_sync(0xffffffffu, next_ready)) {
-        ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], j & 1, bar, p.status));
-        if (!ok) break;
+    int n = 0;                        // items seen: parity of o_full
+    uint32_t g_par = 0;               // parity of the global key-tile index (phase of s_full / p_full)
+    auto next_item = [&](int i) {     // next non-empty item after index i, or -1
+      for (i += item_step; i < p.total_items; i += item_step) {
+        const Item itx = decode_item(p, i);
+        if (itx.qt0 < itx.ntiles) return i;
       }
-      tc_fence_after();
-      const uint32_t tSb = tS + h * kSub, tPb = tP + h * (kSub / 2);
-      o_scale = 1.f;
-      if (pending) {                 // the previous step raised the maximum: new reference from here on
-        l *= pend_alpha;
-        o_scale = pend_alpha;
-        m = pend_m;
-        pending = false;
-      }
-      if (edge_all || (edge_last && j == ntiles - 1)) {
-        // Edge tile: overwrite the scores of keys that do not exist (outside the grid or the
-        // window) with -inf in tensor memory, then treat the step like any other.
-        // vx, vy: valid extent of the key tile's box along x and y
-        const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
+      return -1;
+    };
+    int cur = next_item(item0 - item_step);
+    if (cur >= 0) next_ready = mbar_test(&bar->s_full[t][0], 0);
+    while (cur >= 0 && ok) {
+      const Item it = decode_item(p, cur);
+      const int nxt = next_item(cur);
+      const int ntiles = it.ntiles, nsteps = 2 * ntiles;
+      const int x0 = it.x0, y0 = it.y0, x_end = it.x_end, y_end = it.y_end;
+      // Which key tiles have keys that do not exist?  A window narrower than the box makes every
+      // tile an edge tile; otherwise only the last tile of the window / sequence can be one.
+      const bool edge_all = (x_end - x0) < p.box_w && p.step_x == 0;
+      const int last_vx = x_end - (x0 + (ntiles - 1) * p.step_x), last_vy = y_end - (y0 + (ntiles - 1) * p.step_y);
+      const bool edge_last = last_vx < p.box_w || last_vy < p.box_h;
+      m = -INFINITY;
+      l = 0.f;
+      pending = false;
+      for (int u = 0; u < nsteps && ok; ++u) {
+        const int j = u >> 1, h = u & 1;
+        // warp-uniform outcome: the tensor-memory accesses below are warp-collective
+        if (!__all_sync(0xffffffffu, next_ready)) {
+          ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], g_par, bar, p.status));
+          if (!ok) break;
+        }
+        tc_fence_after();
+        const uint32_t tSb = tS + h * kSub, tPb = tP + h * (kSub / 2);
+        o_scale = 1.f;
+        if (pending) {                 // the previous step raised the maximum: new reference from here on
+          l *= pend_alpha;
+          o_scale = pend_alpha;
+          m = pend_m;
+          pending = false;
+        }
+        if (edge_all || (edge_last && j == ntiles - 1)) {
+          // Edge tile: overwrite the scores of keys that do not exist (outside the grid or the
+          // window) with -inf in tensor memory, then treat the step like any other.
+          // vx, vy: valid extent of the key tile's box along x and y
+          const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-          const int k0 = 64 * h + 32 * c;            // first of the 32 keys, as an index into the box
-          uint32_t bits = 0;
-          if (p.box_w >= 32) {                       // the 32 keys lie in one box row
-            const int ly = k0 >> lg_bw, lx0 = k0 & (p.box_w - 1);
-            const int n = min(32, vx - lx0);
-            if (ly < vy && n > 0) bits = n >= 32 ? 0xffffffffu : ((1u << n) - 1u);
-          } else {                                   // 32 / box_w whole box rows
-            const uint32_t rowbits = (1u << min(vx, p.box_w)) - 1u;
-            const int ly0 = k0 >> lg_bw;
-            for (int r = 0; r < (32 >> lg_bw); ++r)
-              if (ly0 + r < vy) bits |= rowbits << (r << lg_bw);
+          for (int c = 0; c < 2; ++c) {
+            const int k0 = 64 * h + 32 * c;            // first of the 32 keys, as an index into the box
+            uint32_t bits = 0;
+            if (p.box_w >= 32) {                       // the 32 keys lie in one box row
+              const int ly = k0 >> lg_bw, lx0 = k0 & (p.box_w - 1);
+              const int nv = min(32, vx - lx0);
+              if (ly < vy && nv > 0) bits = nv >= 32 ? 0xffffffffu : ((1u << nv) - 1u);
+            } else {                                   // 32 / box_w whole box rows
+              const uint32_t rowbits = (1u << min(vx, p.box_w)) - 1u;
+              const int ly0 = k0 >> lg_bw;
+              for (int r = 0; r < (32 >> lg_bw); ++r)
+                if (ly0 + r < vy) bits |= rowbits << (r << lg_bw);
+            }
+            if (bits != 0xffffffffu) {                 // warp-uniform: the mask depends on the tile only
+              uint32_t v[32];
+              tmem_ld32(tSb + 32 * c, v);
+              tmem_wait_ld(v);
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (!((bits >> i) & 1u)) v[i] = kNegInf;   // exp2(-inf) = 0 and -inf never wins the maximum
+              tmem_st32(tSb + 32 * c, v);
+            }
           }
-          if (bits != 0xffffffffu) {                 // warp-uniform: the mask depends on the tile only
+          tmem_wait_st();
+        }
+        // the step after this one (possibly the first of the next item): its score barrier
+        const bool has_next = u + 1 < nsteps || nxt >= 0;
+        uint64_t* next_bar = &bar->s_full[t][h ^ 1];
+        const uint32_t next_parity = g_par ^ (uint32_t)h;      // same key tile after h = 0, the next one after h = 1
+        if (u == 0 || !one_pass(tSb, tPb, next_bar, next_parity)) {
+          two_pass(tSb, tPb);
+          next_ready = false;
+          rescale_vote = __any_sync(0xffffffffu, o_scale != 1.f);
+        }
+        if (!has_next) next_ready = false;
+        if (u > 0 && rescale_vote) {
+          // O may be touched once P V of step u - 1 has retired; the next P V waits for our P.
+          // The issuer commits the scores of step u + 1 after issuing P V (u - 1), so that barrier
+          // tells us; after the last step of the run there are no further scores, and pv_done
+          // (committed after each P V of the run's last key tile) does.
+          if (has_next)
+            ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, bar, p.status));
+          else
+            ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, bar, p.status));
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
             uint32_t v[32];
-            tmem_ld32(tSb + 32 * c, v);
+            tmem_ld32(tO + 32 * c, v);
             tmem_wait_ld(v);
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (!((bits >> i) & 1u)) v[i] = kNegInf;   // exp2(-inf) = 0 and -inf never wins the maximum
-            tmem_st32(tSb + 32 * c, v);
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * o_scale);
+            tmem_st32(tO + 32 * c, v);
           }
         }
         tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar->p_full[t][h]);
+        g_par ^= (uint32_t)h;
       }
-      uint64_t* next_bar = &bar->s_full[t][h ^ 1];
-      const uint32_t next_parity = ((u + 1) >> 1) & 1;
-      if (u == 0 || !one_pass(tSb, tPb, next_bar, next_parity)) {
-        two_pass(tSb, tPb);
-        next_ready = false;
-        rescale_vote = __any_sync(0xffffffffu, o_scale != 1.f);
-      }
-      if (u > 0 && rescale_vote) {
-        // O may be touched once P V of step u - 1 has retired; the next P V waits for our P.
-        // The issuer commits S(t, u + 1) after issuing P V (u - 1), so that barrier tells us;
-        // on the last step there is no further S, and pv_done (committed after each P V of
-        // the last key tile) does.
-        if (u + 1 < nsteps)
-          ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, bar, p.status));
-        else
-          ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, bar, p.status));
-        if (!ok) break;
-        tc_fence_after();
+
+      // ---- epilogue of the item: O / l -> bf16 -> global memory ----
+      ok = __all_sync(0xffffffffu, ok && mbar_wait(&bar->o_full[t], n & 1, bar, p.status));
+      if (!ok) break;
+      tc_fence_after();
+      {
+        // this row's token
+        const int qx = x0 + (it.qt0 + t) * p.step_x + row % p.box_w, qy = y0 + (it.qt0 + t) * p.step_y + row / p.box_w;
+        const bool row_ok = (it.qt0 + t < ntiles) && qx < x_end && qy < y_end;
+        const float inv = 1.f / l;
+        __nv_bfloat16* dst = p.o + ((size_t)it.bh * p.tokens_per_head + (size_t)qy * p.gridW + qx) * kD;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t v[32];
           tmem_ld32(tO + 32 * c, v);
           tmem_wait_ld(v);
+          if (row_ok) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * o_scale);
-          tmem_st32(tO + 32 * c, v);
-        }
-      }
-      if (u + 1 == nsteps) next_ready = true;   // nothing to wait for after the last step
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bar->p_full[t][h]);
-    }
-
-    ok = __all_sync(0xffffffffu, ok && mbar_wait(&bar->o_full[t], 0, bar, p.status));
-    if (ok) {
-      tc_fence_after();
-      // this row's token
-      const int qx = x0 + (qt0 + t) * p.step_x + row % p.box_w, qy = y0 + (qt0 + t) * p.step_y + row / p.box_w;
-      const bool row_ok = (qt0 + t < ntiles) && qx < x_end && qy < y_end;
-      const float inv = 1.f / l;
-      __nv_bfloat16* dst = p.o + ((size_t)bh * p.tokens_per_head + (size_t)qy * p.gridW + qx) * kD;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t v[32];
-        tmem_ld32(tO + 32 * c, v);
-        tmem_wait_ld(v);
-        if (row_ok) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + 32 * c + 8 * i) = w;
+            for (int i = 0; i < 4; ++i) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
+              *reinterpret_cast<uint4*>(dst + 32 * c + 8 * i) = w;
+            }
           }
         }
       }
+      cur = nxt;
+      ++n;
     }
   }
 
@@ -745,7 +835,7 @@ bool attn_tc_supported(const AttnArgs& a, bool full) {
   if (a.dtype != JV_BF16 || a.D != kD) return false;
   Geometry g;
   if (!geometry(a, full, &g)) return false;
-  if ((int64_t)g.nwx * g.nwy > 65535) return false;
+  if ((int64_t)g.nwx * g.nwy * ceil_div(g.tiles_per_window, 2) * a.BH > 0x7fffffffll) return false;
   // 128-byte rows keep every TMA stride a multiple of 16 bytes; the base must be 16-byte aligned (checked by the ABI)
   return encode_fn() != nullptr;
 }
@@ -787,8 +877,22 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   p.step_x = g.step_x;
   p.step_y = g.step_y;
   p.nwx = g.nwx;
+  p.nwin = g.nwx * g.nwy;
+  p.qpairs = ceil_div(g.tiles_per_window, 2);
+  p.total_items = p.qpairs * p.nwin * a.BH;
   p.scale_log2 = a.scale * 1.4426950408889634f;
-  dim3 grid(ceil_div(g.tiles_per_window, 2), g.nwx * g.nwy, a.BH);
+  // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no more)
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
+      num_sms = 0;
+      cudaGetLastError();
+      return cudaErrorUnknown;
+    }
+  }
+  const int grid = p.total_items < num_sms ? p.total_items : num_sms;
   attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], p);
   count_launch();
   return cudaGetLastError();
