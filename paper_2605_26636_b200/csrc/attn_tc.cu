@@ -29,6 +29,8 @@
 // (tensor memory is always released).
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace jv {
@@ -45,6 +47,18 @@ constexpr int kSub = 64;                    // keys per softmax / MMA step: half
 constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
+// Division by a run-time constant without a divide: q = (umulhi(n, mul) + n) >> shr, exact for
+// 0 <= n < 2^31 (mul = floor(2^32 (2^shr - d) / d) + 1, shr = ceil(log2 d)).
+struct FastDiv {
+  uint32_t mul, shr, d;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;
+  return FastDiv{(uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1), l, d};
+}
+__device__ __forceinline__ int fdiv(int n, const FastDiv& f) { return (int)((__umulhi((uint32_t)n, f.mul) + (uint32_t)n) >> f.shr); }
+
 struct TcParams {
   __nv_bfloat16* o;
   int* status;
@@ -57,6 +71,8 @@ struct TcParams {
   int nwin;              // windows per (batch, head)
   int qpairs;            // pairs of query tiles per window (by the full window height)
   int total_items;       // work items: (batch*head, window, query-tile pair), pair index fastest
+  int lg_box_h;          // log2(box_h)
+  FastDiv div_qpairs, div_nwin, div_nwx;
   float scale_log2;      // softmax scale * log2(e)
 };
 
@@ -68,15 +84,15 @@ struct Item {
 };
 __device__ __forceinline__ Item decode_item(const TcParams& p, int i) {
   Item it;
-  const int qp = i % p.qpairs, r = i / p.qpairs;
-  const int win = r % p.nwin;
-  it.bh = r / p.nwin;
-  const int wy = win / p.nwx, wx = win % p.nwx;
+  const int r = fdiv(i, p.div_qpairs), qp = i - r * p.qpairs;
+  it.bh = fdiv(r, p.div_nwin);
+  const int win = r - it.bh * p.nwin;
+  const int wy = fdiv(win, p.div_nwx), wx = win - wy * p.nwx;
   it.x0 = wx * p.win_w;
   it.y0 = wy * p.win_h;
   it.x_end = min(it.x0 + p.win_w, p.gridW);
   it.y_end = min(it.y0 + p.win_h, p.gridH);
-  it.ntiles = p.step_x ? (it.x_end - it.x0 + kTile - 1) / kTile : (it.y_end - it.y0 + p.box_h - 1) / p.box_h;
+  it.ntiles = p.step_x ? (it.x_end - it.x0 + kTile - 1) / kTile : (it.y_end - it.y0 + p.box_h - 1) >> p.lg_box_h;
   it.qt0 = 2 * qp;                // an item with qt0 >= ntiles (short edge window) is empty: every role skips it
   return it;
 }
@@ -86,11 +102,12 @@ struct __align__(8) Barriers {
   uint64_t q_full[2], q_empty[2];                     // the two query buffers (items alternate)
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2][2], p_full[2][2], pv_done[2], o_full[2];
+  uint64_t wg_sync[2];                                // the 128 threads of a softmax warpgroup among themselves
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
-constexpr size_t kSmemTiles = (4 + 2 * kStages) * (size_t)kTileBytes;          // Q[2][2] K[kStages] V[kStages]
+constexpr size_t kSmemTiles = (6 + 2 * kStages) * (size_t)kTileBytes;          // Q[2][2] K[kStages] V[kStages] O[2]
 constexpr size_t kSmemBytes = kSmemTiles + sizeof(Barriers) + 1024;            // + alignment slack
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -351,12 +368,14 @@ constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
 // current item is being finished and stored.
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-               const __grid_constant__ CUtensorMap mapV, const TcParams p) {
+               const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
+               const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
   // Q buffer b holds the two query tiles of an item at sQ + b * 2 tiles
   const uint32_t sQ = smem_u32(smem), sK = sQ + 4 * kTileBytes, sV = sK + kStages * kTileBytes;
+  const uint32_t sO = sV + kStages * kTileBytes;      // output staging, one tile per query tile
 
   // broadcast from lane 0: lets the compiler keep everything derived from the warp index uniform
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
@@ -386,6 +405,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       mbar_init(&bar->pv_done[t], 1);
       mbar_init(&bar->o_full[t], 1);
+      mbar_init(&bar->wg_sync[t], 128);
     }
     mbar_init(&bar->drain, 2);
     bar->abort_flag = 0;
@@ -652,6 +672,73 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       return -1;
     };
+
+    // ---- epilogue of an item, in two parts around the publication of the next item's first P ----
+    // Part 1 reads O (which the next item's first P V will overwrite) and scales it by 1 / l;
+    // part 2 writes the bf16 tile to global memory: through a swizzled staging tile and one TMA
+    // store when the tile's box, clipped to the grid, lies inside the window (the store clips at
+    // the grid edge by itself), row by row otherwise.
+    struct Done {
+      bool have, store, tma;
+      int bh, qx0, qy0, x_end, y_end, par;
+      float inv;
+    } done{};
+    done.have = false;
+    const uint32_t sOt = sO + t * kTileBytes;
+    unsigned char* sOt_ptr = smem + (size_t)(4 + 2 * kStages + t) * kTileBytes;
+    const bool store_leader = (threadIdx.x & 127) == 0;
+    auto epi_load = [&](uint32_t (&ob)[32]) -> bool {
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->o_full[t], done.par, bar, p.status))) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tO + 32 * c, v);
+        tmem_wait_ld(v);
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          ob[16 * c + i] = pack_bf16(__uint_as_float(v[2 * i]) * done.inv, __uint_as_float(v[2 * i + 1]) * done.inv);
+      }
+      return true;
+    };
+    uint32_t wg_par = 0;
+    // warpgroup-wide barrier with the same bounded wait as everything else (a plain bar.sync
+    // would wait for ever for a warp that has given up)
+    auto wg_barrier = [&]() -> bool {
+      mbar_arrive(&bar->wg_sync[t]);
+      const bool done_ok = mbar_wait(&bar->wg_sync[t], wg_par, bar, p.status);
+      wg_par ^= 1;
+      return __all_sync(0xffffffffu, done_ok);
+    };
+    auto epi_store = [&](const uint32_t (&ob)[32]) -> bool {
+      if (!done.store) return true;
+      if (done.tma) {
+        // the previous store must have finished reading the staging tile
+        if (store_leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        if (!wg_barrier()) return false;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)     // 16-byte chunk c of this row, at its 128-byte-swizzle position
+          *reinterpret_cast<uint4*>(sOt_ptr + row * 128 + ((c ^ (row & 7)) << 4)) =
+              make_uint4(ob[4 * c], ob[4 * c + 1], ob[4 * c + 2], ob[4 * c + 3]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (!wg_barrier()) return false;
+        if (store_leader) {
+          asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                       ::"l"(&mapO), "r"(sOt), "r"(0), "r"(done.qx0), "r"(done.qy0), "r"(done.bh) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      } else {
+        const int qx = done.qx0 + row % p.box_w, qy = done.qy0 + row / p.box_w;
+        if (qx < done.x_end && qy < done.y_end) {
+          __nv_bfloat16* dst = p.o + ((size_t)done.bh * p.tokens_per_head + (size_t)qy * p.gridW + qx) * kD;
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<uint4*>(dst + 8 * c) = make_uint4(ob[4 * c], ob[4 * c + 1], ob[4 * c + 2], ob[4 * c + 3]);
+        }
+      }
+      return true;
+    };
+
     int cur = next_item(item0 - item_step);
     if (cur >= 0) next_ready = mbar_test(&bar->s_full[t][0], 0);
     while (cur >= 0 && ok) {
@@ -667,12 +754,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       m = -INFINITY;
       l = 0.f;
       pending = false;
-      for (int u = 0; u < nsteps && ok; ++u) {
+      // one 64-key step up to (not including) the publication of its P; first_tag: first step of the item
+      auto compute_step = [&](auto first_tag, int u) -> bool {
+        constexpr bool kFirst = decltype(first_tag)::value;
         const int j = u >> 1, h = u & 1;
         // warp-uniform outcome: the tensor-memory accesses below are warp-collective
         if (!__all_sync(0xffffffffu, next_ready)) {
           ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], g_par, bar, p.status));
-          if (!ok) break;
+          if (!ok) return false;
         }
         tc_fence_after();
         const uint32_t tSb = tS + h * kSub, tPb = tP + h * (kSub / 2);
@@ -718,13 +807,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const bool has_next = u + 1 < nsteps || nxt >= 0;
         uint64_t* next_bar = &bar->s_full[t][h ^ 1];
         const uint32_t next_parity = g_par ^ (uint32_t)h;      // same key tile after h = 0, the next one after h = 1
-        if (u == 0 || !one_pass(tSb, tPb, next_bar, next_parity)) {
+        if (kFirst || !one_pass(tSb, tPb, next_bar, next_parity)) {
           two_pass(tSb, tPb);
           next_ready = false;
           rescale_vote = __any_sync(0xffffffffu, o_scale != 1.f);
         }
         if (!has_next) next_ready = false;
-        if (u > 0 && rescale_vote) {
+        if (!kFirst && rescale_vote) {
           // O may be touched once P V of step u - 1 has retired; the next P V waits for our P.
           // The issuer commits the scores of step u + 1 after issuing P V (u - 1), so that barrier
           // tells us; after the last step of the run there are no further scores, and pv_done
@@ -733,7 +822,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, bar, p.status));
           else
             ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, bar, p.status));
-          if (!ok) break;
+          if (!ok) return false;
           tc_fence_after();
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
@@ -745,43 +834,55 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             tmem_st32(tO + 32 * c, v);
           }
         }
+        return true;
+      };
+      auto publish = [&](int h) {
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar->p_full[t][h]);
         g_par ^= (uint32_t)h;
-      }
-
-      // ---- epilogue of the item: O / l -> bf16 -> global memory ----
-      ok = __all_sync(0xffffffffu, ok && mbar_wait(&bar->o_full[t], n & 1, bar, p.status));
+      };
+      // First step.  The previous item's O has to be read before this item's first P is published
+      // (its P V overwrites O); by now that item's last P V has long retired.
+      ok = compute_step(std::true_type{}, 0);
       if (!ok) break;
-      tc_fence_after();
-      {
-        // this row's token
-        const int qx = x0 + (it.qt0 + t) * p.step_x + row % p.box_w, qy = y0 + (it.qt0 + t) * p.step_y + row / p.box_w;
-        const bool row_ok = (it.qt0 + t < ntiles) && qx < x_end && qy < y_end;
-        const float inv = 1.f / l;
-        __nv_bfloat16* dst = p.o + ((size_t)it.bh * p.tokens_per_head + (size_t)qy * p.gridW + qx) * kD;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t v[32];
-          tmem_ld32(tO + 32 * c, v);
-          tmem_wait_ld(v);
-          if (row_ok) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint4 w;
-              w.x = pack_bf16(__uint_as_float(v[8 * i + 0]) * inv, __uint_as_float(v[8 * i + 1]) * inv);
-              w.y = pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv);
-              w.z = pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv);
-              w.w = pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv);
-              *reinterpret_cast<uint4*>(dst + 32 * c + 8 * i) = w;
-            }
-          }
-        }
+      if (done.have) {
+        uint32_t ob[32];
+        ok = epi_load(ob);
+        if (!ok) break;
+        publish(0);
+        ok = epi_store(ob);
+        done.have = false;
+      } else {
+        publish(0);
       }
+      for (int u = 1; u < nsteps && ok; ++u) {
+        ok = compute_step(std::false_type{}, u);
+        if (ok) publish(u & 1);
+      }
+      if (!ok) break;
+      // what the deferred epilogue of this item needs
+      done.have = true;
+      done.store = it.qt0 + t < ntiles;
+      done.bh = it.bh;
+      done.qx0 = x0 + (it.qt0 + t) * p.step_x;
+      done.qy0 = y0 + (it.qt0 + t) * p.step_y;
+      done.x_end = x_end;
+      done.y_end = y_end;
+      done.par = n & 1;
+      done.inv = 1.f / l;
+      // one TMA store is right when the box, clipped to the grid, holds tokens of this window only
+      done.tma = p.step_x != 0 || ((x0 + p.box_w <= x_end || x_end == p.gridW) &&
+                                   (done.qy0 + p.box_h <= y_end || y_end == p.gridH));
       cur = nxt;
       ++n;
     }
+    if (ok && done.have) {            // the run's last item
+      uint32_t ob[32];
+      if (epi_load(ob)) ok = epi_store(ob);
+    }
+    // the staging tile must outlive the last store's reads; wait for the writes as well
+    if (store_leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // ================= common teardown =================
@@ -846,13 +947,13 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   EncodeFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
   const int N = a.Hg * a.Wg;
-  CUtensorMap maps[3];
-  const void* ptrs[3] = {a.q, a.k, a.v};
+  CUtensorMap maps[4];
+  const void* ptrs[4] = {a.q, a.k, a.v, a.o};
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.gridW, (cuuint64_t)g.gridH, (cuuint64_t)a.BH};
   const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.gridW * kD * 2, (cuuint64_t)N * kD * 2};
   const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  for (int i = 0; i < 3; ++i) {
+  for (int i = 0; i < 4; ++i) {
     CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -880,6 +981,11 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   p.nwin = g.nwx * g.nwy;
   p.qpairs = ceil_div(g.tiles_per_window, 2);
   p.total_items = p.qpairs * p.nwin * a.BH;
+  p.lg_box_h = 0;
+  while ((1 << p.lg_box_h) < g.box_h) ++p.lg_box_h;
+  p.div_qpairs = make_fastdiv((uint32_t)p.qpairs);
+  p.div_nwin = make_fastdiv((uint32_t)p.nwin);
+  p.div_nwx = make_fastdiv((uint32_t)p.nwx);
   p.scale_log2 = a.scale * 1.4426950408889634f;
   // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no more)
   static int num_sms = 0;
@@ -893,7 +999,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
     }
   }
   const int grid = p.total_items < num_sms ? p.total_items : num_sms;
-  attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], p);
+  attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   count_launch();
   return cudaGetLastError();
 }
