@@ -1,21 +1,33 @@
 // bf16 tensor-core path of the linear-attention block (Sec. 3.2.1, Eq. 2
 // reordered, Eq. 4), head_dim 64.
 //
-// The block is bound by HBM traffic (read K, V, Q once, write O once), but only
-// if the two 64x64 contractions per token run on tensor cores: at ~32 flop per
-// byte they would otherwise exceed the fp32 ALU rate.  Both passes therefore
-// stream 64-token tiles through a cp.async ring into XOR-swizzled shared memory
-// and feed mma.sync m16n8k16 (bf16 in, fp32 accumulate) via ldmatrix.
+// The block is bound by HBM traffic (read K, V, Q once, write O once; V a second
+// time, mostly from L2, when the squeeze dynamic convolution is on), but only if the
+// two 64x64 contractions per token run on tensor cores: at ~32 flop per byte they
+// would otherwise exceed the fp32 ALU rate.  Two kernels, each a one-wave grid of
+// CTAs that stream 64-token tiles through a TMA + mbarrier ring (one producer warp,
+// four MMA warps; 128-byte-swizzled tiles feed ldmatrix without bank conflicts):
 //
-//   pass 1  lin_state_kernel   per (head, token chunk):  KV = relu(K)^T V, z = relu(K)^T 1,
-//                              (v-sum when the dynamic convolution is on) -> fp32 partials
-//   pass 2  launch_lin_reduce  fixed-order sum of the chunk partials (bit-reproducible)
-//   pass 3  lin_apply_kernel   o = relu(q) KV / (relu(q).z + eps): KV as bf16 MMA operand,
-//                              the denominator exactly in fp32 from the A fragments
-//   pass 4  dwc_add_kernel     (only with the dynamic convolution) o += DWC_w(V)
+//   lin_state_kernel   per (head, token chunk):  KV = relu(K)^T V, z = relu(K)^T 1,
+//                      (v-sum when the convolution is on) -> fp32 chunk partials
+//   lin_apply_kernel   sums the chunk partials of its head in a fixed order (the
+//                      deterministic second pass: no floating-point atomics), then
+//                      o = relu(q) KV / (relu(q).z + eps) [+ DWC_w(V)] per tile:
+//                      KV as bf16 MMA operand, the denominator exactly in fp32 from
+//                      the A fragments, output tiles written back by TMA stores.
 //
-// Fast-path partial / state layout per (batch, head), in floats:
+// The apply kernel is launched with programmatic stream serialisation: its set-up and
+// its first Q loads overlap the tail of the state kernel, and it waits for that grid
+// (griddepcontrol.wait) only before touching the partials.
+//
+// With the convolution on, two small kernels (the generator MLP) run in between, and
+// the apply kernel keeps a ring of V tiles covering the (k-1)/2 grid rows above and
+// below the tile it is working on.
+//
+// Partial layout per (batch, head, chunk), in floats:
 //   [0, 4096) KV[a][e], [4096, 4160) z[a], [4160, 4224) vsum[e]
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace jv {
@@ -24,19 +36,71 @@ namespace {
 constexpr int kD = 64;
 constexpr int kTileTok = 64;                  // tokens per shared-memory tile
 constexpr int kTileBytes = kTileTok * kD * 2; // 8 KB
-constexpr int kStateFloats = kD * kD + 2 * kD;
 constexpr int kOffZ = kD * kD, kOffVsum = kD * kD + kD;
-constexpr int kThreads = 128;
+constexpr int kConsumers = 128;               // 4 MMA warps
+constexpr int kThreads = kConsumers + 32;     // + 1 producer warp
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-  const int sz = valid ? 16 : 0;   // size 0: the 16 destination bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait of a whole (converged) warp with a warp-uniform outcome.  On expiry the
+// status word and the CTA's abort flag are set and every role leaves its loop.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status) {
+  bool ok = mbar_try(bar, parity);
+  if (!ok) {
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+      if (mbar_try(bar, parity)) { ok = true; break; }
+      if ((spin & 63u) == 63u) {
+        if (*abort_flag) break;
+        const unsigned long long now = globaltimer();
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitLimitNs) {
+          *abort_flag = 1;
+          atomicOr(status, kStatusTimeout);
+          break;
+        }
+      }
+    }
+  }
+  return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
+  return pred != 0;
+}
+// 64 tokens x 64 channels of a [B*H, N, 64] tensor -> shared memory (128-byte swizzle);
+// tokens past N arrive as zeros.
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int tok, int bh) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(tok), "r"(bh) : "memory");
+}
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -57,48 +121,79 @@ __device__ __forceinline__ uint32_t relu_bf16x2(uint32_t x) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 __device__ __forceinline__ float2 bf16x2_to_f2(uint32_t x) {
-  return __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&x));
+  return make_float2(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
 }
 
-// Byte offset of 16-byte chunk `ch` (0..7) of row `row` in a [rows][64 bf16] tile whose
-// chunks are XOR-swizzled by the row index, so that ldmatrix reads hit 8 distinct banks groups.
+// Byte offset of 16-byte chunk `ch` (0..7) of row `row` in a [rows][64 bf16] tile in the
+// 128-byte-swizzle layout (what TMA writes): chunks are XORed with the row index mod 8, so
+// ldmatrix reads of 8 rows hit 8 distinct bank groups.
 __device__ __forceinline__ uint32_t tile_off(int row, int ch) { return (uint32_t)(row * 128 + ((ch ^ (row & 7)) << 4)); }
 
-// One 64-token tile of a [.., 64] bf16 tensor -> shared memory; rows >= rows_valid are zero-filled.
-__device__ __forceinline__ void load_tile(uint32_t dst, const __nv_bfloat16* src, int rows_valid) {
-#pragma unroll
-  for (int i = 0; i < (kTileTok * 8) / kThreads; ++i) {
-    const int c = threadIdx.x + kThreads * i, row = c >> 3, ch = c & 7;
-    const bool ok = row < rows_valid;
-    cp_async16(dst + tile_off(row, ch), src + (ok ? (size_t)row * kD + ch * 8 : 0), ok);
-  }
-}
+struct __align__(8) Ring {
+  uint64_t full[8], empty[8];
+  volatile uint32_t abort_flag;
+};
 
 // ---- pass 1: partial state of one token chunk ------------------------------------
+constexpr int kStateStages = 6;               // 6 x (K tile + V tile) = 96 KB per CTA, two CTAs per SM
+constexpr size_t kStateSmem = (size_t)kStateStages * 2 * kTileBytes + 1024 + sizeof(Ring);
+
 template <bool kVsum>
 __global__ void __launch_bounds__(kThreads)
-lin_state_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
-                 float* __restrict__ partial, int N, int chunk_tokens, int state_elems) {
-  constexpr int kStages = 3;
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  const uint32_t smem = smem_u32(smem_raw);     // stage s: K tile at s*16K, V tile at s*16K + 8K
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
+                 float* __restrict__ partial, int* status, int N, int chunk_tokens, int state_elems) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t smem = smem_u32(smem_al);      // stage s: K tile at s * 16 KB, V tile at s * 16 KB + 8 KB
+  Ring* ring = reinterpret_cast<Ring*>(smem_al + (size_t)kStateStages * 2 * kTileBytes);
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const int bh = blockIdx.y, chunk = blockIdx.x;
   const int t_begin = chunk * chunk_tokens, t_end = min(N, t_begin + chunk_tokens);
   const int ntiles = (t_end - t_begin + kTileTok - 1) / kTileTok;
-  const __nv_bfloat16* kb = k + ((size_t)bh * N + t_begin) * kD;
-  const __nv_bfloat16* vb = v + ((size_t)bh * N + t_begin) * kD;
 
-  auto issue = [&](int tile) {
-    if (tile < ntiles) {
-      const uint32_t st = smem + (tile % kStages) * 2 * kTileBytes;
-      const int valid = min(kTileTok, t_end - t_begin - tile * kTileTok);
-      load_tile(st, kb + (size_t)tile * kTileTok * kD, valid);
-      load_tile(st + kTileBytes, vb + (size_t)tile * kTileTok * kD, valid);
+  // let the grid that depends on this one (the apply pass) start its set-up as SMs free up
+  griddep_launch_dependents();
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStateStages; ++s) {
+      mbar_init(&ring->full[s], 1);
+      mbar_init(&ring->empty[s], 4);          // one arrival per MMA warp
     }
-    cp_async_commit();
-  };
+    ring->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(status) != 0) return;   // an earlier kernel gave up: leave at once
 
+  if (warp == 4) {
+    // ================= TMA producer =================
+    int s = 0;
+    uint32_t par = 1;
+    int issued = 0;
+    bool ok = true;
+    for (int it = 0; it < ntiles; ++it) {
+      ok = warp_wait(&ring->empty[s], par, &ring->abort_flag, status);
+      if (!ok) break;
+      if (elect_one()) {
+        mbar_expect_tx(&ring->full[s], 2 * kTileBytes);
+        const int tok = t_begin + it * kTileTok;     // a chunk's last tile may run past t_end: only by whole
+        tma_load_tile(smem + s * 2 * kTileBytes, &mapK, &ring->full[s], tok, bh);              // zero rows past N
+        tma_load_tile(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], tok, bh);
+      }
+      __syncwarp();
+      ++issued;
+      if (++s == kStateStages) { s = 0; par ^= 1; }
+    }
+    if (!ok && lane == 0) {   // let the copies in flight land before the CTA leaves
+      const unsigned long long t0 = globaltimer();
+      for (int g = max(0, issued - kStateStages); g < issued; ++g)
+        while (!mbar_try(&ring->full[g % kStateStages], (g / kStateStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
+    }
+    return;
+  }
+
+  // ================= MMA warps: warp w owns rows 16 w .. 16 w + 15 of KV =================
   float acc[9][4];
 #pragma unroll
   for (int j = 0; j < 9; ++j)
@@ -108,14 +203,13 @@ lin_state_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __res
   // B fragment of the "ones" column: B[k][n] = 1 for n == 0 -> held by lanes 0..3
   const uint32_t ones = (lane < 4) ? 0x3F803F80u : 0u;
 
-#pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) issue(s);
-
+  int s = 0;
+  uint32_t par = 0;
+  bool ok = true;
   for (int it = 0; it < ntiles; ++it) {
-    cp_async_wait<kStages - 2>();
-    __syncthreads();
-    issue(it + kStages - 1);
-    const uint32_t ks = smem + (it % kStages) * 2 * kTileBytes, vsm = ks + kTileBytes;
+    ok = warp_wait(&ring->full[s], par, &ring->abort_flag, status);
+    if (!ok) break;
+    const uint32_t ks = smem + s * 2 * kTileBytes, vsm = ks + kTileBytes;
 #pragma unroll
     for (int kk = 0; kk < kTileTok / 16; ++kk) {
       uint32_t a[4];
@@ -141,8 +235,11 @@ lin_state_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __res
       }
       mma_bf16(acc[8], a, ones, ones);
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&ring->empty[s]);
+    if (++s == kStateStages) { s = 0; par ^= 1; }
   }
-  cp_async_wait<0>();
+  if (!ok) return;
 
   float* out = partial + ((size_t)bh * gridDim.x + chunk) * state_elems;
   const int g = lane >> 2, tq = lane & 3;
@@ -165,43 +262,89 @@ lin_state_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __res
       out[kOffVsum + 16 * warp + g] = vs0;
       out[kOffVsum + 16 * warp + 8 + g] = vs1;
     }
-  } else if (threadIdx.x < kD) {
-    out[kOffVsum + threadIdx.x] = 0.f;
   }
 }
 
-// ---- pass 3: streaming apply -----------------------------------------------------
+// ---- pass 2: deterministic sum of the chunk partials, then the streaming apply ----------
+constexpr int kApplyStages = 6;               // Q ring: 72 KB per CTA with KV and staging, three CTAs per SM
+struct __align__(8) ApplyBars {
+  uint64_t full[kApplyStages], empty[kApplyStages];
+  uint64_t state_ready;                       // the 128 MMA threads among themselves
+  volatile uint32_t abort_flag;
+};
+// shared memory: Q ring | KV (bf16, swizzled) | output staging 2 x 8 KB | z (fp32) | barriers
+constexpr size_t kApplySmem = (size_t)(kApplyStages + 1 + 2) * kTileBytes + 1024 + kD * sizeof(float) + sizeof(ApplyBars);
+
 __global__ void __launch_bounds__(kThreads)
-lin_apply_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ o,
-                 const float* __restrict__ state, int N, int cta_tokens, int state_elems, float eps) {
-  constexpr int kStages = 3;
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  const uint32_t smem = smem_u32(smem_raw);
-  const uint32_t kv_sm = smem + kStages * kTileBytes;            // bf16 KV[a][e], swizzled, 8 KB
-  float* z_sm = reinterpret_cast<float*>(smem_raw + (kStages + 1) * kTileBytes);   // 64 floats
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapO,
+                 const float* __restrict__ partial, int* status, int N, int span_tokens, int nchunk, int state_elems,
+                 float eps) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t smem = smem_u32(smem_al);
+  const uint32_t kv_sm = smem + kApplyStages * kTileBytes;                    // bf16 KV[a][e]
+  unsigned char* kv_ptr = smem_al + (size_t)kApplyStages * kTileBytes;
+  const uint32_t out_sm = kv_sm + kTileBytes;                                  // 2 staging tiles
+  unsigned char* out_ptr = kv_ptr + kTileBytes;
+  float* z_sm = reinterpret_cast<float*>(out_ptr + 2 * kTileBytes);
+  ApplyBars* bars = reinterpret_cast<ApplyBars*>(z_sm + kD);
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const int bh = blockIdx.y;
-  const int t_begin = blockIdx.x * cta_tokens, t_end = min(N, t_begin + cta_tokens);
+  const int t_begin = blockIdx.x * span_tokens, t_end = min(N, t_begin + span_tokens);
   const int ntiles = (t_end - t_begin + kTileTok - 1) / kTileTok;
-  const __nv_bfloat16* qb = q + ((size_t)bh * N + t_begin) * kD;
-  __nv_bfloat16* ob = o + ((size_t)bh * N + t_begin) * kD;
 
-  auto issue = [&](int tile) {
-    if (tile < ntiles)
-      load_tile(smem + (tile % kStages) * kTileBytes, qb + (size_t)tile * kTileTok * kD,
-                min(kTileTok, t_end - t_begin - tile * kTileTok));
-    cp_async_commit();
-  };
-#pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) issue(s);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kApplyStages; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 4);
+    }
+    mbar_init(&bars->state_ready, kConsumers);
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
 
-  {  // state -> shared memory: KV rounded to bf16 (MMA operand), z kept in fp32
-    const float* S = state + (size_t)bh * state_elems;
+  if (warp == 4) {
+    // ================= TMA producer: Q does not depend on the state pass, start at once =================
+    int s = 0;
+    uint32_t par = 1;
+    int issued = 0;
+    bool ok = true;
+    for (int it = 0; it < ntiles; ++it) {
+      ok = warp_wait(&bars->empty[s], par, &bars->abort_flag, status);
+      if (!ok) break;
+      if (elect_one()) {
+        mbar_expect_tx(&bars->full[s], kTileBytes);
+        tma_load_tile(smem + s * kTileBytes, &mapQ, &bars->full[s], t_begin + it * kTileTok, bh);
+      }
+      __syncwarp();
+      ++issued;
+      if (++s == kApplyStages) { s = 0; par ^= 1; }
+    }
+    if (!ok && lane == 0) {
+      const unsigned long long t0 = globaltimer();
+      for (int g = max(0, issued - kApplyStages); g < issued; ++g)
+        while (!mbar_try(&bars->full[g % kApplyStages], (g / kApplyStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
+    }
+    return;
+  }
+
+  // ================= MMA warps =================
+  griddep_wait();                                    // the state pass (and anything before it) has completed
+  bool ok = *reinterpret_cast<volatile int*>(status) == 0;
+  {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
+    const float* P = partial + (size_t)bh * nchunk * state_elems;
 #pragma unroll
-    for (int i = 0; i < (kD * 8) / kThreads; ++i) {
-      const int c = threadIdx.x + kThreads * i, row = c >> 3, ch = c & 7;
-      const float4 x = *reinterpret_cast<const float4*>(S + row * kD + ch * 8);
-      const float4 y = *reinterpret_cast<const float4*>(S + row * kD + ch * 8 + 4);
+    for (int i = 0; i < (kD * 8) / kConsumers; ++i) {
+      const int c = threadIdx.x + kConsumers * i, row = c >> 3, ch = c & 7;
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+      for (int k = 0; k < nchunk; ++k) {
+        const float4 xa = *reinterpret_cast<const float4*>(P + (size_t)k * state_elems + row * kD + ch * 8);
+        const float4 ya = *reinterpret_cast<const float4*>(P + (size_t)k * state_elems + row * kD + ch * 8 + 4);
+        x.x += xa.x; x.y += xa.y; x.z += xa.z; x.w += xa.w;
+        y.x += ya.x; y.y += ya.y; y.z += ya.z; y.w += ya.w;
+      }
       __nv_bfloat162 p0 = __floats2bfloat162_rn(x.x, x.y), p1 = __floats2bfloat162_rn(x.z, x.w);
       __nv_bfloat162 p2 = __floats2bfloat162_rn(y.x, y.y), p3 = __floats2bfloat162_rn(y.z, y.w);
       uint4 pk;
@@ -209,11 +352,17 @@ lin_apply_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict_
       pk.y = *reinterpret_cast<uint32_t*>(&p1);
       pk.z = *reinterpret_cast<uint32_t*>(&p2);
       pk.w = *reinterpret_cast<uint32_t*>(&p3);
-      *reinterpret_cast<uint4*>(smem_raw + kStages * kTileBytes + tile_off(row, ch)) = pk;
+      *reinterpret_cast<uint4*>(kv_ptr + tile_off(row, ch)) = pk;
     }
-    if (threadIdx.x < kD) z_sm[threadIdx.x] = S[kOffZ + threadIdx.x];
+    if (threadIdx.x < kD) {
+      float zs = 0.f;
+      for (int k = 0; k < nchunk; ++k) zs += P[(size_t)k * state_elems + kOffZ + threadIdx.x];
+      z_sm[threadIdx.x] = zs;
+    }
   }
-  __syncthreads();
+  mbar_arrive(&bars->state_ready);
+  ok = warp_wait(&bars->state_ready, 0, &bars->abort_flag, status) && ok;
+  if (!ok) return;
 
   const int g = lane >> 2, tq = lane & 3;
   float zr[16];   // z at the 16 k-indices this thread's A fragments cover
@@ -225,12 +374,12 @@ lin_apply_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict_
     zr[4 * kk + 3] = z_sm[16 * kk + 8 + 2 * tq + 1];
   }
 
+  int s = 0;
+  uint32_t par = 0;
   for (int it = 0; it < ntiles; ++it) {
-    cp_async_wait<kStages - 2>();
-    __syncthreads();
-    issue(it + kStages - 1);
-    const uint32_t qs = smem + (it % kStages) * kTileBytes;
-    unsigned char* qs_ptr = smem_raw + (it % kStages) * kTileBytes;
+    ok = warp_wait(&bars->full[s], par, &bars->abort_flag, status);
+    if (!ok) break;
+    const uint32_t qs = smem + s * kTileBytes;
 
     float acc[8][4];
 #pragma unroll
@@ -261,35 +410,45 @@ lin_apply_kernel(const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict_
         mma_bf16(acc[2 * jp + 1], a, b[2], b[3]);
       }
     }
+    // the Q tile has been read: hand the stage back to the producer
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&bars->empty[s]);
+    if (++s == kApplyStages) { s = 0; par ^= 1; }
+
     den_lo += __shfl_xor_sync(0xffffffffu, den_lo, 1);
     den_lo += __shfl_xor_sync(0xffffffffu, den_lo, 2);
     den_hi += __shfl_xor_sync(0xffffffffu, den_hi, 1);
     den_hi += __shfl_xor_sync(0xffffffffu, den_hi, 2);
     const float inv_lo = 1.f / (den_lo + eps), inv_hi = 1.f / (den_hi + eps);
 
-    // Stage the warp's 16 output rows over its own (now consumed) Q rows, then store 16 B per lane.
+    // This warp's 16 output rows -> its 2 KB of the staging tile (swizzled) -> one TMA store.
+    // The store issued from this staging tile two tiles ago must have finished reading it.
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
     __syncwarp();
+    unsigned char* st = out_ptr + (it & 1) * kTileBytes + warp * 2048;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       __nv_bfloat162 lo = __floats2bfloat162_rn(acc[j][0] * inv_lo, acc[j][1] * inv_lo);
       __nv_bfloat162 hi = __floats2bfloat162_rn(acc[j][2] * inv_hi, acc[j][3] * inv_hi);
-      *reinterpret_cast<__nv_bfloat162*>(qs_ptr + tile_off(16 * warp + g, j) + 4 * tq) = lo;
-      *reinterpret_cast<__nv_bfloat162*>(qs_ptr + tile_off(16 * warp + g + 8, j) + 4 * tq) = hi;
+      *reinterpret_cast<__nv_bfloat162*>(st + tile_off(g, j) + 4 * tq) = lo;
+      *reinterpret_cast<__nv_bfloat162*>(st + tile_off(g + 8, j) + 4 * tq) = hi;
     }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
-    const int rows_valid = t_end - t_begin - it * kTileTok;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int c = lane + 32 * i, row = 16 * warp + (c >> 3), ch = c & 7;
-      if (row < rows_valid)
-        *reinterpret_cast<uint4*>(ob + ((size_t)it * kTileTok + row) * kD + ch * 8) =
-            *reinterpret_cast<const uint4*>(qs_ptr + tile_off(row, ch));
+    if (lane == 0) {
+      const int tok = t_begin + it * kTileTok + 16 * warp;
+      if (tok < N) {      // rows past N inside the box are clipped by the store itself
+        asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                     ::"l"(&mapO), "r"(out_sm + (it & 1) * kTileBytes + warp * 2048), "r"(0), "r"(tok), "r"(bh) : "memory");
+      }
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     }
   }
-  cp_async_wait<0>();
+  // the staging tiles must outlive the reads of the last stores
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-// ---- pass 4: o += depth-wise k x k convolution of V with the sample's kernels ------
+// ---- o += depth-wise k x k convolution of V with the sample's kernels ------------------
 // One warp walks a run of consecutive tokens of one head; lane owns channels 2*lane, 2*lane+1.
 template <int K>
 __global__ void __launch_bounds__(256)
@@ -329,10 +488,39 @@ dwc_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ 
   }
 }
 
+// ---- host side ---------------------------------------------------------------------------
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn encode_fn() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = (EncodeFn)ptr;
+  }
+  return fn;
+}
+// [BH, N, 64] bf16 as a 3-D tensor (channel, token, batch*head); box = 64 channels x box_tok tokens
+bool make_map(CUtensorMap* m, const void* ptr, int BH, int N, int box_tok) {
+  EncodeFn enc = encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)BH};
+  const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)N * kD * 2};
+  const cuuint32_t box[3] = {(cuuint32_t)kD, (cuuint32_t)box_tok, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool linear_fast_supported(const LinArgs& a) {
-  return a.s.dtype == JV_BF16 && a.s.D == kD;
+  return a.s.dtype == JV_BF16 && a.s.D == kD && encode_fn() != nullptr;
 }
 
 cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t st) {
@@ -341,31 +529,58 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   char* ws = (char*)a.ws;
   float* partial = (float*)(ws + p.off_partial);
   float* state = (float*)(ws + p.off_state);
-  const __nv_bfloat16* q = (const __nv_bfloat16*)a.q;
-  const __nv_bfloat16* k = (const __nv_bfloat16*)a.k;
-  const __nv_bfloat16* v = (const __nv_bfloat16*)a.v;
-  __nv_bfloat16* o = (__nv_bfloat16*)a.o;
+  int* status = device_status_ptr();
+  if (!status) return cudaErrorUnknown;
+
+  CUtensorMap mq, mk, mv, mo;
+  if (!make_map(&mq, a.q, BH, N, kTileTok) || !make_map(&mk, a.k, BH, N, kTileTok) ||
+      !make_map(&mv, a.v, BH, N, kTileTok) || !make_map(&mo, a.o, BH, N, 16))
+    return cudaErrorInvalidValue;
 
   static bool attr_done = false;   // > 48 KB of dynamic shared memory needs the opt-in, once per process
-  const size_t smem1 = 3 * 2 * kTileBytes, smem3 = 4 * kTileBytes + kD * sizeof(float);
   if (!attr_done) {
-    cudaFuncSetAttribute(lin_state_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
-    cudaFuncSetAttribute(lin_state_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(lin_state_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStateSmem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(lin_state_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStateSmem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(lin_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApplySmem)) != cudaSuccess) return e;
     attr_done = true;
   }
   dim3 g1(p.nchunk, BH);
   if (a.dwc)
-    lin_state_kernel<true><<<g1, kThreads, smem1, st>>>(k, v, partial, N, p.chunk_tokens, p.state_elems);
+    lin_state_kernel<true><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems);
   else
-    lin_state_kernel<false><<<g1, kThreads, smem1, st>>>(k, v, partial, N, p.chunk_tokens, p.state_elems);
+    lin_state_kernel<false><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems);
   count_launch();
-  cudaError_t e = launch_lin_reduce(partial, state, p.nchunk, p.state_elems, (size_t)BH * p.state_elems, st);
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int cta_tokens = 512;
-  dim3 g3(ceil_div(N, cta_tokens), BH);
-  lin_apply_kernel<<<g3, kThreads, smem3, st>>>(q, o, state, N, cta_tokens, p.state_elems, a.eps);
+
+  // apply pass: one wave of three CTAs per SM, spans of whole tiles; launched so that its set-up
+  // overlaps the tail of the state pass
+  int nspan = (3 * 148) / BH;
+  if (nspan < 1) nspan = 1;
+  int span = ceil_div(ceil_div(N, nspan), kTileTok) * kTileTok;
+  if (span < 4 * kTileTok) span = 4 * kTileTok;
+  nspan = ceil_div(N, span);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(nspan, BH);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kApplySmem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, lin_apply_kernel, mq, mo, (const float*)partial, status, N, span, p.nchunk,
+                         p.state_elems, a.eps);
   count_launch();
+  if (e != cudaSuccess) return e;
+
   if (a.dwc) {
+    const __nv_bfloat16* v = (const __nv_bfloat16*)a.v;
+    __nv_bfloat16* o = (__nv_bfloat16*)a.o;
+    e = launch_lin_reduce(partial, state, p.nchunk, p.state_elems, (size_t)BH * p.state_elems, st);
+    if (e != cudaSuccess) return e;
     e = launch_dwc_generator(a, p, state + kOffVsum, p.state_elems, st);
     if (e != cudaSuccess) return e;
     const float* w = (const float*)(ws + p.off_kernel);

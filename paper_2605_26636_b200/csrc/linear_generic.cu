@@ -15,9 +15,11 @@ LinPlan lin_plan(const jv_shape& s, const jv_dwc* dwc) {
   const int N = s.Hg * s.Wg, BH = s.B * s.H;
   p.D1 = s.D + 1;
   p.state_elems = (p.D1 * p.D1 + 3) / 4 * 4;
-  // Enough chunks to give every SM a few CTAs, chunks a multiple of 128 tokens
-  // and at least 512 tokens long so that the partials stay small next to K and V.
-  int want = ceil_div(4 * 148, BH);
+  // Chunks: as many as fit one wave of two CTAs per SM over all (batch, head) pairs, each a
+  // multiple of 128 tokens and at least 512 tokens long so that the partials stay small next
+  // to K and V.  One wave means no tail, and chunks of equal length finish together.
+  int want = (2 * 148) / BH;
+  if (want < 1) want = 1;
   int chunk = ceil_div(ceil_div(N, want), 128) * 128;
   if (chunk < 512) chunk = 512;
   p.chunk_tokens = chunk;
