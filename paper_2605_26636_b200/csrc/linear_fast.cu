@@ -488,6 +488,159 @@ dwc_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ 
   }
 }
 
+// ---- o += depth-wise 3 x 3 convolution of V: the tuned kernel ----------------------------------
+// CTA = 8 warps = a patch of 8 grid rows x 16 grid columns of one (batch, head); warp w owns row
+// y0 + w.  A lane owns 4 channels (8 bytes: 16 lanes cover the 128-byte token row, so every
+// access is a full line) and 8 consecutive tokens, and slides a 3 x 3 window of V along x: each
+// V element is unpacked once and used for three taps.  All loads of the thread are issued
+// before the arithmetic; rows y +- 1 come from L1 / L2 (neighbouring warps read them too).
+constexpr int kDwcCols = 16, kDwcRows = 8, kDwcRun = 8;
+__device__ __forceinline__ uint64_t pack2f(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2f(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__global__ void __launch_bounds__(256, 2)
+dwc3_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ o, const float* __restrict__ w,
+                int H, int Hg, int Wg, int ncol_blocks) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int c4 = lane & 15, half = lane >> 4;              // channels 4 c4 .. 4 c4 + 3; tokens 8 half .. 8 half + 7
+  const int N = Hg * Wg, bh = blockIdx.y, b = bh / H, h = bh % H;
+  const int rb = blockIdx.x / ncol_blocks, cb = blockIdx.x % ncol_blocks;
+  const int y = rb * kDwcRows + warp, x0 = cb * kDwcCols + half * kDwcRun;
+  if (y >= Hg || x0 >= Wg) return;
+  const uint2* vb = reinterpret_cast<const uint2*>(v + (size_t)bh * N * kD) + c4;     // + token * 16
+  uint2* ob = reinterpret_cast<uint2*>(o + (size_t)bh * N * kD) + c4;
+
+  // weights of this thread's 4 channels: w[ch][tap] -> per tap two fp32 pairs
+  uint64_t w01[9], w23[9];
+  {
+    const float4* wp = reinterpret_cast<const float4*>(w + ((size_t)b * H * kD + (size_t)h * kD + 4 * c4) * 9);
+    float wf[36];
+#pragma unroll
+    for (int i = 0; i < 9; ++i) {
+      const float4 t = __ldg(wp + i);
+      wf[4 * i] = t.x; wf[4 * i + 1] = t.y; wf[4 * i + 2] = t.z; wf[4 * i + 3] = t.w;
+    }
+#pragma unroll
+    for (int tap = 0; tap < 9; ++tap) {
+      w01[tap] = pack2f(wf[tap], wf[9 + tap]);
+      w23[tap] = pack2f(wf[18 + tap], wf[27 + tap]);
+    }
+  }
+  // all loads first: 3 rows x 10 columns of V (zeros outside the grid), 8 tokens of o
+  uint2 vr[3][kDwcRun + 2], cur[kDwcRun];
+#pragma unroll
+  for (int dy = 0; dy < 3; ++dy) {
+    const int yy = y + dy - 1;
+    const bool row_ok = yy >= 0 && yy < Hg;
+#pragma unroll
+    for (int i = 0; i < kDwcRun + 2; ++i) {
+      const int xx = x0 + i - 1;
+      vr[dy][i] = (row_ok && xx >= 0 && xx < Wg) ? __ldg(vb + (size_t)(yy * Wg + xx) * 16) : make_uint2(0u, 0u);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kDwcRun; ++i)
+    cur[i] = (x0 + i < Wg) ? ob[(size_t)(y * Wg + x0 + i) * 16] : make_uint2(0u, 0u);
+
+#pragma unroll
+  for (int i = 0; i < kDwcRun; ++i) {
+    uint64_t a01 = pack2f(__uint_as_float(cur[i].x << 16), __uint_as_float(cur[i].x & 0xffff0000u));
+    uint64_t a23 = pack2f(__uint_as_float(cur[i].y << 16), __uint_as_float(cur[i].y & 0xffff0000u));
+#pragma unroll
+    for (int dy = 0; dy < 3; ++dy)
+#pragma unroll
+      for (int dx = 0; dx < 3; ++dx) {
+        const uint2 t = vr[dy][i + dx];
+        a01 = fma2f(w01[3 * dy + dx], pack2f(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u)), a01);
+        a23 = fma2f(w23[3 * dy + dx], pack2f(__uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u)), a23);
+      }
+    if (x0 + i < Wg) {
+      float r0, r1, r2, r3;
+      asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(a01));
+      asm("mov.b64 {%0, %1}, %2;" : "=f"(r2), "=f"(r3) : "l"(a23));
+      __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+      uint2 out;
+      out.x = *reinterpret_cast<uint32_t*>(&lo);
+      out.y = *reinterpret_cast<uint32_t*>(&hi);
+      ob[(size_t)(y * Wg + x0 + i) * 16] = out;
+    }
+  }
+}
+
+// ---- kernel generator of the squeeze dynamic convolution (Sec. 3.2.1), tuned for latency ------
+// hidden[b][r] = SiLU(b1[r] + sum_c W1[r][c] * mean_v[b][c]); one block per (r, b).  mean_v comes
+// straight from the chunk partials' v-sums (summed in a fixed order).
+__global__ void __launch_bounds__(128)
+gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W1, const float* __restrict__ b1,
+                  float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n) {
+  __shared__ float red[4];
+  const int r = blockIdx.x, b = blockIdx.y, C = H * kD;
+  float s = 0.f;
+  for (int c = threadIdx.x; c < C; c += 128) {
+    const int h = c / kD, e = c % kD;
+    const float* pv = partial + (size_t)(b * H + h) * nchunk * state_elems + kOffVsum + e;
+    float m = 0.f;
+    for (int k = 0; k < nchunk; ++k) m += pv[(size_t)k * state_elems];
+    s = fmaf(__ldg(&W1[(size_t)r * C + c]), m * inv_n, s);
+  }
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const float x = ((red[0] + red[1]) + (red[2] + red[3])) + (b1 ? b1[r] : 0.f);
+    hidden[(size_t)b * R + r] = x / (1.f + expf(-x));
+  }
+}
+// w[b][t] = b2[t] + sum_r W2[t][r] * hidden[b][r]; 8 lanes per output t, 32 outputs per block, all
+// samples.  A lane's W2 values (r = part, part + 8, ...) are fetched 16 at a time, all loads in
+// flight together, and reused for up to 8 samples.
+__global__ void __launch_bounds__(256)
+gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, const float* __restrict__ b2,
+               float* __restrict__ w, int B, int T, int R) {
+  const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
+  const bool t_ok = t < T;
+  const float* wrow = W2 + (size_t)(t_ok ? t : 0) * R;
+  for (int b0 = 0; b0 < B; b0 += 8) {
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int r0 = 0; r0 < R; r0 += 128) {
+      float wv[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int r = r0 + part + 8 * i;
+        wv[i] = r < R ? __ldg(wrow + r) : 0.f;
+      }
+#pragma unroll
+      for (int bb = 0; bb < 8; ++bb) {
+        if (b0 + bb < B) {
+          const float* hp = hidden + (size_t)(b0 + bb) * R;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int r = r0 + part + 8 * i;
+            if (r < R) acc[bb] = fmaf(wv[i], __ldg(hp + r), acc[bb]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int bb = 0; bb < 8; ++bb) {
+      float sres = acc[bb];
+      sres += __shfl_xor_sync(0xffffffffu, sres, 1);
+      sres += __shfl_xor_sync(0xffffffffu, sres, 2);
+      sres += __shfl_xor_sync(0xffffffffu, sres, 4);
+      if (t_ok && part == 0 && b0 + bb < B) w[(size_t)(b0 + bb) * T + t] = sres + (b2 ? b2[t] : 0.f);
+    }
+  }
+}
+
 // ---- host side ---------------------------------------------------------------------------
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -579,16 +732,22 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   if (a.dwc) {
     const __nv_bfloat16* v = (const __nv_bfloat16*)a.v;
     __nv_bfloat16* o = (__nv_bfloat16*)a.o;
-    e = launch_lin_reduce(partial, state, p.nchunk, p.state_elems, (size_t)BH * p.state_elems, st);
-    if (e != cudaSuccess) return e;
-    e = launch_dwc_generator(a, p, state + kOffVsum, p.state_elems, st);
-    if (e != cudaSuccess) return e;
+    const jv_dwc& d = *a.dwc;
+    float* hidden = (float*)(ws + p.off_hidden);
+    float* wk = (float*)(ws + p.off_kernel);
+    gen_hidden_kernel<<<dim3(d.R, s.B), 128, 0, st>>>(partial, d.W1, d.b1, hidden, s.H, d.R, p.nchunk, p.state_elems,
+                                                      1.f / (float)N);
+    count_launch();
+    const int T = s.H * kD * d.k * d.k;
+    gen_out_kernel<<<ceil_div(T, 32), 256, 0, st>>>(hidden, d.W2, d.b2, wk, s.B, T, d.R);
+    count_launch();
     const float* w = (const float*)(ws + p.off_kernel);
     const int run = 32;
     dim3 g4(ceil_div(ceil_div(N, run), 8), BH);
-    if (a.dwc->k == 3)
-      dwc_add_kernel<3><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
-    else
+    if (a.dwc->k == 3) {
+      const int ncb = ceil_div(s.Wg, kDwcCols);
+      dwc3_add_kernel<<<dim3(ncb * ceil_div(s.Hg, kDwcRows), BH), 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, ncb);
+    } else
       dwc_add_kernel<5><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
     count_launch();
   }
