@@ -40,6 +40,9 @@ METRIC = "mixer tokens/sec (L+W+F stack at ViT-L shapes)"
 UNIT = "tokens/s"
 STEP_SCHEDULE = "LWF"
 WIN = 16
+# DRAM bytes of one attn_tc_kernel launch running F at the DINOv3-L shape, from the ncu capture
+# summarised in profiles/ (None when the kernel has changed since the capture)
+ATTN_F_DRAM_BYTES = None
 
 
 def load_peaks():
@@ -80,7 +83,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -140,6 +143,22 @@ def dist_env():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     return rank, world, local
+
+
+def max_over_ranks(x: float, world: int, device=None) -> float:
+    """MAX all-reduce of a per-rank time (the step time of a multi-GPU run is the slowest rank's)."""
+    if world <= 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_layer_ids(rank: int, n_layers: int):
+    """Layer indices that seed rank `rank`'s inputs: every rank draws its own shard (the path shards
+    over independent (batch, head) units, so ranks share nothing but the timing barrier)."""
+    return [100 * rank + l for l in range(n_layers)]
 
 
 # ----------------------------------------------------------------------------- oracle legs
@@ -218,7 +237,7 @@ def run_cuda(args):
     C = w.H * w.D
 
     # ---- inputs: three layers of Q/K/V in pinned host memory and on the device
-    host = [[t.pin_memory() for t in inputs.qkv(w, layer=100 * rank + l)] for l in range(nL)]
+    host = [[t.pin_memory() for t in inputs.qkv(w, layer=lid)] for lid in rank_layer_ids(rank, nL)]
     dq, dk, dv = ([host[l][i].to(dev, non_blocking=True) for l in range(nL)] for i in range(3))
     outs = [torch.empty_like(t) for t in dq]
     host_out = [torch.empty(w.shape, dtype=torch.bfloat16).pin_memory() for _ in range(nL)]
@@ -229,8 +248,16 @@ def run_cuda(args):
     ws = jv.alloc_workspace("S", shape, jv.make_dwc(dwc_dev, dev), dev)
     torch.cuda.synchronize()
 
-    def step(_i=0):
-        jv.hybrid_mixers(STEP_SCHEDULE, dq, dk, dv, w.Hg, w.Wg, WIN, WIN, dwc=dwcs, out=outs, ws=ws)
+    # One step = the schedule driver over the three layers.  It is issued as one jv_hybrid_mixers
+    # call per layer so that events between the calls give each mixer's time inside the timed region.
+    def step(_i=0, ev=None):
+        for l, m in enumerate(STEP_SCHEDULE):
+            if ev is not None:
+                ev[l].record(stream)
+            jv.hybrid_mixers(m, dq[l:l + 1], dk[l:l + 1], dv[l:l + 1], w.Hg, w.Wg, WIN, WIN, dwc=dwcs[l:l + 1],
+                             out=outs[l:l + 1], ws=ws)
+        if ev is not None:
+            ev[nL].record(stream)
 
     def barrier():
         if world > 1:
@@ -244,19 +271,18 @@ def run_cuda(args):
     barrier()
     l0 = jv.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_ev = min(args.steps, 64)            # steps whose per-layer events are kept
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nL + 1)] for _ in range(n_ev)]
     with ClockSampler(local) as clk:
         e0.record(stream)
         for i in range(args.steps):
-            step()
+            step(i, evs[i] if i < n_ev else None)
         e1.record(stream)
         barrier()
     launches = jv.launch_count() - l0
     ms = e0.elapsed_time(e1) / args.steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    layer_ms = [float(np.mean([evs[i][l].elapsed_time(evs[i][l + 1]) for i in range(n_ev)])) for l in range(nL)]
+    ms = max_over_ranks(ms, world, dev)
     assert jv.device_status() == jv.JV_OK, "a kernel reported a timeout"
     step_tokens = nL * w.tokens
     value = world * step_tokens / (ms * 1e-3)
@@ -279,11 +305,7 @@ def run_cuda(args):
     e1.record(stream)
     barrier()
     ms_e2e = e0.elapsed_time(e1) / n_e2e
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    ms_e2e = max_over_ranks(ms_e2e, world, dev)
     tensor_bytes = int(np.prod(w.shape)) * 2
     e2e = {"value": world * step_tokens / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
            "h2d_bytes_per_step": 3 * nL * tensor_bytes, "d2h_bytes_per_step": nL * tensor_bytes}
@@ -297,7 +319,7 @@ def run_cuda(args):
 
     # ---- per-mixer timings (rank 0; rotating over the three layers' tensors: 805 MB > L2)
     per = {}
-    K, W = max(args.steps, 10), max(args.warmup, 3)
+    K, W = min(max(args.steps, 10), 100), max(min(args.warmup, 10), 3)
     hbm, tf = peaks["hbm_gbs"], peaks["bf16_tflops"]
 
     def add(name, fn, bytes_, flops, bound):
@@ -353,13 +375,20 @@ def run_cuda(args):
     del q5, lo, base
     assert jv.device_status() == jv.JV_OK, "a kernel reported a timeout"
 
-    # ---- roofline of the dominant kernel of the step (full attention)
-    dom = per["F"]
-    roofline = {"kernel": "full attention (jv_full_attn)", "bound": "tensor", "achieved": dom["TFLOPs"],
-                "peak": tf, "unit": "TFLOP/s", "frac": dom["TFLOPs"] / tf, "traffic": None,
-                "peak_source": peaks["source"] + " bf16 burst",
+    # ---- roofline of the dominant kernel of the step: the attention kernel running F, timed inside
+    # the timed region (events around the F layer of every step)
+    f_ms = layer_ms[STEP_SCHEDULE.index("F")]
+    f_tf = f_flops / f_ms / 1e9
+    roofline = {"kernel": "attn_tc_kernel as jv_full_attn (one launch per step)", "bound": "tensor", "achieved": f_tf,
+                "peak": tf, "unit": "TFLOP/s", "frac": f_tf / tf, "traffic": ATTN_F_DRAM_BYTES,
+                "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
+                "peak_source": peaks["source"] + " bf16 burst", "ms_per_launch": f_ms,
+                "flops_per_launch": f_flops, "alg_bytes_per_launch": alg_bytes(*w.shape),
+                "step_layers_ms": dict(zip(["L+dwc", "W", "F"], layer_ms)),
                 "linear": {"bound": "hbm", "achieved": per["L"]["GBps"], "peak": hbm, "unit": "GB/s",
                            "frac": per["L"]["GBps"] / hbm},
+                "linear_dwc": {"bound": "hbm", "achieved": per["L+dwc"]["GBps"], "peak": hbm, "unit": "GB/s",
+                               "frac": per["L+dwc"]["GBps"] / hbm},
                 "window": {"bound": "hbm", "achieved": per["W"]["GBps"], "peak": hbm, "unit": "GB/s",
                            "frac": per["W"]["GBps"] / hbm, "tensor_frac": per["W"]["TFLOPs"] / tf}}
 
@@ -421,8 +450,8 @@ def run_single(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--single", choices=["L", "L+dwc", "W", "F"], default=None,
