@@ -163,9 +163,9 @@ def rank_layer_ids(rank: int, n_layers: int):
 
 # ----------------------------------------------------------------------------- oracle legs
 def oracle_sample_step(w, scale=1.0):
-    """A bounded sample of one step for the CPU oracle (about 10 s on 8 cores at
-    scale 1): L with the dynamic convolution and W on ceil(scale * B) batch samples,
-    F on all query rows of round(32 * scale) of the B*H (batch, head) pairs; each
+    """A bounded sample of one step for the CPU oracle (about 10 s on 16 cores, 30 s on 8,
+    at scale 1): L with the dynamic convolution and W on ceil(scale * B) batch samples,
+    F on all query rows of round(scale * B * H) of the B*H (batch, head) pairs; each
     mixer's time is extrapolated to the whole step by its sampled fraction.
     Returns (seconds spent, extrapolated seconds of a whole step, description,
     threads used)."""
@@ -181,7 +181,7 @@ def oracle_sample_step(w, scale=1.0):
     t0 = time.perf_counter()
     jv_oracle.window_attn(q, k, v, w.Hg, w.Wg, WIN, WIN)
     tW = time.perf_counter() - t0
-    nF = max(1, min(w.B * w.H, int(round(32 * scale))))
+    nF = max(1, min(w.B * w.H, int(round(w.B * w.H * scale))))
     q, k, v = inputs.qkv(w, layer=2, shape=(1, nF, w.N, w.D))
     t0 = time.perf_counter()
     jv_oracle.full_attn(q, k, v)
@@ -200,7 +200,7 @@ def run_reference(args):
     step_tokens = len(STEP_SCHEDULE) * w.tokens
     # size the per-step sample so that the whole run stays near two minutes
     n_warm = min(args.warmup, 1)
-    scale = min(1.0, 120.0 / (10.5 * (args.steps + n_warm)))
+    scale = min(1.0, 120.0 / (30.0 * (args.steps + n_warm)))
     for _ in range(n_warm):
         oracle_sample_step(w, scale)
     spent, full = [], []
