@@ -5,16 +5,17 @@
 // time, mostly from L2, when the squeeze dynamic convolution is on), but only if the
 // two 64x64 contractions per token run on tensor cores: at ~32 flop per byte they
 // would otherwise exceed the fp32 ALU rate.  Two kernels, each a one-wave grid of
-// CTAs that stream 64-token tiles through a TMA + mbarrier ring (one producer warp,
-// four MMA warps; 128-byte-swizzled tiles feed ldmatrix without bank conflicts):
+// CTAs that stream token tiles through a TMA + mbarrier ring (one producer warp, four
+// worker warps; 128-byte-swizzled tiles feed ldmatrix / the tensor core without bank conflicts):
 //
 //   lin_state_kernel   per (head, token chunk):  KV = relu(K)^T V, z = relu(K)^T 1,
 //                      (v-sum when the convolution is on) -> fp32 chunk partials
 //   lin_apply_kernel   sums the chunk partials of its head in a fixed order (the
 //                      deterministic second pass: no floating-point atomics), then
-//                      o = relu(q) KV / (relu(q).z + eps) [+ DWC_w(V)] per tile:
-//                      KV as bf16 MMA operand, the denominator exactly in fp32 from
-//                      the A fragments, output tiles written back by TMA stores.
+//                      o = relu(q) KV / (relu(q).z + eps) per 128-token tile: ReLU in
+//                      place in shared memory, relu(Q) KV as tcgen05.mma with the
+//                      accumulator in tensor memory (KV as bf16 operand), the
+//                      denominator exactly in fp32, output written back by TMA stores.
 //
 // The apply kernel is launched with programmatic stream serialisation: its set-up and
 // its first Q loads overlap the tail of the state kernel, and it waits for that grid
@@ -266,14 +267,58 @@ lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant
 }
 
 // ---- pass 2: deterministic sum of the chunk partials, then the streaming apply ----------
-constexpr int kApplyStages = 6;               // Q ring: 72 KB per CTA with KV and staging, three CTAs per SM
+// 128-token tiles.  Per tile: TMA brings Q in; the four worker warps apply ReLU in place (one
+// thread per token row, which also gives that row's denominator relu(q).z exactly in fp32);
+// one elected thread issues O_tile = relu(Q) KV as four tcgen05.mma (M128 N64 K16, A = Q tile
+// K-major, B = bf16 KV MN-major, accumulator in tensor memory); the same thread-per-row
+// mapping reads the accumulator back, divides, rounds to bf16 and stages its row; each warp
+// writes its 32 rows with one TMA store.  Accumulators and staging are double-buffered so the
+// MMA of tile i + 1 runs under the epilogue of tile i.
+constexpr int kApplyTok = 128;                          // tokens per apply tile
+constexpr int kApplyTileBytes = kApplyTok * kD * 2;     // 16 KB
+constexpr int kApplyStages = 4;                         // Q ring
+constexpr uint32_t kApplyTmemCols = 128;                // two 64-column fp32 accumulators
 struct __align__(8) ApplyBars {
   uint64_t full[kApplyStages], empty[kApplyStages];
-  uint64_t state_ready;                       // the 128 MMA threads among themselves
+  uint64_t d_full[2];                         // accumulator of tile i ready (tcgen05.commit)
+  uint64_t workers;                           // the 128 worker threads among themselves (once, after the state is in place)
+  uint64_t relu_done[2];                      // 128 arrivals per tile (tiles alternate): Q tile rectified, accumulator buffer free
+  uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
-// shared memory: Q ring | KV (bf16, swizzled) | output staging 2 x 8 KB | z (fp32) | barriers
-constexpr size_t kApplySmem = (size_t)(kApplyStages + 1 + 2) * kTileBytes + 1024 + kD * sizeof(float) + sizeof(ApplyBars);
+// shared memory: Q ring | KV (bf16, swizzled) | output staging 2 x 16 KB | z (fp32) | barriers
+constexpr size_t kApplySmem =
+    (size_t)(kApplyStages + 2) * kApplyTileBytes + kTileBytes + 1024 + kD * sizeof(float) + sizeof(ApplyBars);
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, B MN-major, M = 128, N = 64.
+constexpr uint32_t kIdescApply = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+// Waits for this thread's outstanding tensor-memory loads; the registers are threaded through
+// the statement so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :: "memory");
+}
 
 __global__ void __launch_bounds__(kThreads)
 lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapO,
@@ -281,171 +326,258 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  float eps) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const uint32_t smem = smem_u32(smem_al);
-  const uint32_t kv_sm = smem + kApplyStages * kTileBytes;                    // bf16 KV[a][e]
-  unsigned char* kv_ptr = smem_al + (size_t)kApplyStages * kTileBytes;
-  const uint32_t out_sm = kv_sm + kTileBytes;                                  // 2 staging tiles
-  unsigned char* out_ptr = kv_ptr + kTileBytes;
-  float* z_sm = reinterpret_cast<float*>(out_ptr + 2 * kTileBytes);
+  const uint32_t smem = smem_u32(smem_al);                                       // Q ring
+  unsigned char* out_ptr = smem_al + (size_t)kApplyStages * kApplyTileBytes;     // 2 staging tiles
+  const uint32_t out_sm = smem + kApplyStages * kApplyTileBytes;
+  unsigned char* kv_ptr = out_ptr + 2 * kApplyTileBytes;                         // bf16 KV[a][e], swizzled
+  const uint32_t kv_sm = out_sm + 2 * kApplyTileBytes;
+  float* z_sm = reinterpret_cast<float*>(kv_ptr + kTileBytes);
   ApplyBars* bars = reinterpret_cast<ApplyBars*>(z_sm + kD);
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const int bh = blockIdx.y;
   const int t_begin = blockIdx.x * span_tokens, t_end = min(N, t_begin + span_tokens);
-  const int ntiles = (t_end - t_begin + kTileTok - 1) / kTileTok;
+  const int ntiles = (t_end - t_begin + kApplyTok - 1) / kApplyTok;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kApplyStages; ++s) {
       mbar_init(&bars->full[s], 1);
-      mbar_init(&bars->empty[s], 4);
+      mbar_init(&bars->empty[s], 1);          // released by the commit that follows the tile's MMAs
     }
-    mbar_init(&bars->state_ready, kConsumers);
+    mbar_init(&bars->d_full[0], 1);
+    mbar_init(&bars->d_full[1], 1);
+    mbar_init(&bars->workers, kConsumers);
+    mbar_init(&bars->relu_done[0], kConsumers);
+    mbar_init(&bars->relu_done[1], kConsumers);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)),
+                 "r"(kApplyTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
   __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
 
   if (warp == 4) {
-    // ================= TMA producer: Q does not depend on the state pass, start at once =================
-    int s = 0;
-    uint32_t par = 1;
-    int issued = 0;
+    // ================= TMA producer and MMA issuer (one elected lane) =================
+    // Q does not depend on the state pass: the first loads start at once.  Per tile: refill the
+    // ring slot freed by the previous tile's MMAs, wait until the workers have rectified the tile
+    // (and are done with the accumulator buffer it will overwrite), issue its four MMAs.
     bool ok = true;
-    for (int it = 0; it < ntiles; ++it) {
-      ok = warp_wait(&bars->empty[s], par, &bars->abort_flag, status);
-      if (!ok) break;
+    int issued = 0;
+    auto load_tile = [&](int it) {
       if (elect_one()) {
-        mbar_expect_tx(&bars->full[s], kTileBytes);
-        tma_load_tile(smem + s * kTileBytes, &mapQ, &bars->full[s], t_begin + it * kTileTok, bh);
+        const int s = it % kApplyStages;
+        mbar_expect_tx(&bars->full[s], kApplyTileBytes);
+        tma_load_tile(smem + s * kApplyTileBytes, &mapQ, &bars->full[s], t_begin + it * kApplyTok, bh);
       }
       __syncwarp();
       ++issued;
-      if (++s == kApplyStages) { s = 0; par ^= 1; }
+    };
+    for (int it = 0; it < kApplyStages - 1 && it < ntiles; ++it) load_tile(it);
+    for (int it = 0; it < ntiles; ++it) {
+      const int nx = it + kApplyStages - 1;            // goes into the slot of tile it - 1
+      if (nx < ntiles) {
+        if (it > 0) {
+          ok = warp_wait(&bars->empty[nx % kApplyStages], ((it - 1) / kApplyStages) & 1, &bars->abort_flag, status);
+          if (!ok) break;
+        }
+        load_tile(nx);
+      }
+      ok = warp_wait(&bars->relu_done[it & 1], (it >> 1) & 1, &bars->abort_flag, status);
+      if (!ok) break;
+      tc_fence_after();
+      const int s = it % kApplyStages, b = it & 1;
+      const uint32_t qa = smem + s * kApplyTileBytes;
+#pragma unroll
+      for (int ks = 0; ks < kD / 16; ++ks) {
+        if (elect_one())
+          asm volatile(
+              "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+              "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+              ::"r"(tmem + b * kD), "l"(smem_desc(qa + ks * 32)), "l"(smem_desc(kv_sm + ks * 2048)), "r"(kIdescApply),
+                "r"(ks > 0 ? 1u : 0u) : "memory");
+      }
+      if (elect_one()) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&bars->d_full[b])) : "memory");
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&bars->empty[s])) : "memory");
+      }
+      __syncwarp();
     }
     if (!ok && lane == 0) {
       const unsigned long long t0 = globaltimer();
       for (int g = max(0, issued - kApplyStages); g < issued; ++g)
         while (!mbar_try(&bars->full[g % kApplyStages], (g / kApplyStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
     }
-    return;
-  }
-
-  // ================= MMA warps =================
-  griddep_wait();                                    // the state pass (and anything before it) has completed
-  bool ok = *reinterpret_cast<volatile int*>(status) == 0;
-  {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
-    const float* P = partial + (size_t)bh * nchunk * state_elems;
+  } else {
+    // ================= worker warps: thread r = 32 warp + lane owns token row r of every tile =================
+    griddep_wait();                                    // the state pass (and anything before it) has completed
+    bool ok = *reinterpret_cast<volatile int*>(status) == 0;
+    {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
+      const float* P = partial + (size_t)bh * nchunk * state_elems;
 #pragma unroll
-    for (int i = 0; i < (kD * 8) / kConsumers; ++i) {
-      const int c = threadIdx.x + kConsumers * i, row = c >> 3, ch = c & 7;
-      float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
-      for (int k = 0; k < nchunk; ++k) {
-        const float4 xa = *reinterpret_cast<const float4*>(P + (size_t)k * state_elems + row * kD + ch * 8);
-        const float4 ya = *reinterpret_cast<const float4*>(P + (size_t)k * state_elems + row * kD + ch * 8 + 4);
-        x.x += xa.x; x.y += xa.y; x.z += xa.z; x.w += xa.w;
-        y.x += ya.x; y.y += ya.y; y.z += ya.z; y.w += ya.w;
+      for (int i = 0; i < (kD * 8) / kConsumers; ++i) {
+        const int c = threadIdx.x + kConsumers * i, row = c >> 3, ch = c & 7;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f), y = x;
+        for (int k0 = 0; k0 < nchunk; k0 += 4) {       // four chunks' loads in flight, summed in chunk order
+          float4 xa[4], ya[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const bool in = k0 + k < nchunk;
+            const float* src = P + (size_t)(in ? k0 + k : 0) * state_elems + row * kD + ch * 8;
+            xa[k] = in ? *reinterpret_cast<const float4*>(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+            ya[k] = in ? *reinterpret_cast<const float4*>(src + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            x.x += xa[k].x; x.y += xa[k].y; x.z += xa[k].z; x.w += xa[k].w;
+            y.x += ya[k].x; y.y += ya[k].y; y.z += ya[k].z; y.w += ya[k].w;
+          }
+        }
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(x.x, x.y), p1 = __floats2bfloat162_rn(x.z, x.w);
+        __nv_bfloat162 p2 = __floats2bfloat162_rn(y.x, y.y), p3 = __floats2bfloat162_rn(y.z, y.w);
+        uint4 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&p0);
+        pk.y = *reinterpret_cast<uint32_t*>(&p1);
+        pk.z = *reinterpret_cast<uint32_t*>(&p2);
+        pk.w = *reinterpret_cast<uint32_t*>(&p3);
+        *reinterpret_cast<uint4*>(kv_ptr + tile_off(row, ch)) = pk;
       }
-      __nv_bfloat162 p0 = __floats2bfloat162_rn(x.x, x.y), p1 = __floats2bfloat162_rn(x.z, x.w);
-      __nv_bfloat162 p2 = __floats2bfloat162_rn(y.x, y.y), p3 = __floats2bfloat162_rn(y.z, y.w);
-      uint4 pk;
-      pk.x = *reinterpret_cast<uint32_t*>(&p0);
-      pk.y = *reinterpret_cast<uint32_t*>(&p1);
-      pk.z = *reinterpret_cast<uint32_t*>(&p2);
-      pk.w = *reinterpret_cast<uint32_t*>(&p3);
-      *reinterpret_cast<uint4*>(kv_ptr + tile_off(row, ch)) = pk;
-    }
-    if (threadIdx.x < kD) {
-      float zs = 0.f;
-      for (int k = 0; k < nchunk; ++k) zs += P[(size_t)k * state_elems + kOffZ + threadIdx.x];
-      z_sm[threadIdx.x] = zs;
-    }
-  }
-  mbar_arrive(&bars->state_ready);
-  ok = warp_wait(&bars->state_ready, 0, &bars->abort_flag, status) && ok;
-  if (!ok) return;
-
-  const int g = lane >> 2, tq = lane & 3;
-  float zr[16];   // z at the 16 k-indices this thread's A fragments cover
-#pragma unroll
-  for (int kk = 0; kk < 4; ++kk) {
-    zr[4 * kk + 0] = z_sm[16 * kk + 2 * tq];
-    zr[4 * kk + 1] = z_sm[16 * kk + 2 * tq + 1];
-    zr[4 * kk + 2] = z_sm[16 * kk + 8 + 2 * tq];
-    zr[4 * kk + 3] = z_sm[16 * kk + 8 + 2 * tq + 1];
-  }
-
-  int s = 0;
-  uint32_t par = 0;
-  for (int it = 0; it < ntiles; ++it) {
-    ok = warp_wait(&bars->full[s], par, &bars->abort_flag, status);
-    if (!ok) break;
-    const uint32_t qs = smem + s * kTileBytes;
-
-    float acc[8][4];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
-    float den_lo = 0.f, den_hi = 0.f;
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      uint32_t a[4];   // A = relu(Q): rows = tokens 16*warp.., cols = a
-      ldmatrix_x4(a, qs + tile_off(16 * warp + (lane & 7) + ((lane >> 3) & 1) * 8, 2 * kk + (lane >> 4)));
-#pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = relu_bf16x2(a[i]);
-      {  // denominator relu(q).z in fp32, from the same fragments
-        const float2 f0 = bf16x2_to_f2(a[0]), f1 = bf16x2_to_f2(a[1]);
-        const float2 f2 = bf16x2_to_f2(a[2]), f3 = bf16x2_to_f2(a[3]);
-        den_lo = fmaf(f0.x, zr[4 * kk], fmaf(f0.y, zr[4 * kk + 1], den_lo));
-        den_lo = fmaf(f2.x, zr[4 * kk + 2], fmaf(f2.y, zr[4 * kk + 3], den_lo));
-        den_hi = fmaf(f1.x, zr[4 * kk], fmaf(f1.y, zr[4 * kk + 1], den_hi));
-        den_hi = fmaf(f3.x, zr[4 * kk + 2], fmaf(f3.y, zr[4 * kk + 3], den_hi));
-      }
-      const int ab = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-#pragma unroll
-      for (int jp = 0; jp < 4; ++jp) {
-        uint32_t b[4];   // KV stored [a][e]: B[k = a][n = e] -> .trans
-        ldmatrix_x4_trans(b, kv_sm + tile_off(ab, 2 * jp + (lane >> 4)));
-        mma_bf16(acc[2 * jp], a, b[0], b[1]);
-        mma_bf16(acc[2 * jp + 1], a, b[2], b[3]);
+      if (threadIdx.x < kD) {
+        float zs = 0.f;
+        for (int k = 0; k < nchunk; ++k) zs += P[(size_t)k * state_elems + kOffZ + threadIdx.x];
+        z_sm[threadIdx.x] = zs;
       }
     }
-    // the Q tile has been read: hand the stage back to the producer
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&bars->empty[s]);
-    if (++s == kApplyStages) { s = 0; par ^= 1; }
+    uint32_t wpar = 0;
+    // all 128 worker threads; makes their shared-memory writes visible to the tensor core / TMA
+    auto workers_sync = [&]() -> bool {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(&bars->workers);
+      const bool w_ok = warp_wait(&bars->workers, wpar, &bars->abort_flag, status);
+      wpar ^= 1;
+      tc_fence_after();
+      return w_ok;
+    };
+    const int row = threadIdx.x;                       // 0..127: token row of the tile and tensor-memory lane
+    const uint32_t lane_base = (uint32_t)(warp << 5) << 16;
+    float den = 0.f;
 
-    den_lo += __shfl_xor_sync(0xffffffffu, den_lo, 1);
-    den_lo += __shfl_xor_sync(0xffffffffu, den_lo, 2);
-    den_hi += __shfl_xor_sync(0xffffffffu, den_hi, 1);
-    den_hi += __shfl_xor_sync(0xffffffffu, den_hi, 2);
-    const float inv_lo = 1.f / (den_lo + eps), inv_hi = 1.f / (den_hi + eps);
-
-    // This warp's 16 output rows -> its 2 KB of the staging tile (swizzled) -> one TMA store.
-    // The store issued from this staging tile two tiles ago must have finished reading it.
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-    __syncwarp();
-    unsigned char* st = out_ptr + (it & 1) * kTileBytes + warp * 2048;
+    // ReLU of this thread's row of the Q tile in stage s, in place; returns relu(q).z.
+    // All loads come before the stores (the compiler cannot tell that they do not alias).
+    auto relu_row = [&](int s) -> float {
+      unsigned char* q = smem_al + (size_t)s * kApplyTileBytes + row * 128;
+      uint4 v[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      __nv_bfloat162 lo = __floats2bfloat162_rn(acc[j][0] * inv_lo, acc[j][1] * inv_lo);
-      __nv_bfloat162 hi = __floats2bfloat162_rn(acc[j][2] * inv_hi, acc[j][3] * inv_hi);
-      *reinterpret_cast<__nv_bfloat162*>(st + tile_off(g, j) + 4 * tq) = lo;
-      *reinterpret_cast<__nv_bfloat162*>(st + tile_off(g + 8, j) + 4 * tq) = hi;
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    if (lane == 0) {
-      const int tok = t_begin + it * kTileTok + 16 * warp;
-      if (tok < N) {      // rows past N inside the box are clipped by the store itself
-        asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-                     ::"l"(&mapO), "r"(out_sm + (it & 1) * kTileBytes + warp * 2048), "r"(0), "r"(tok), "r"(bh) : "memory");
+      for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const uint4*>(q + ((c ^ (row & 7)) << 4));
+      float4 zz[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) zz[c] = *reinterpret_cast<const float4*>(z_sm + 4 * c);
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        v[c].x = relu_bf16x2(v[c].x); v[c].y = relu_bf16x2(v[c].y); v[c].z = relu_bf16x2(v[c].z); v[c].w = relu_bf16x2(v[c].w);
+        *reinterpret_cast<uint4*>(q + ((c ^ (row & 7)) << 4)) = v[c];
+        const float2 f0 = bf16x2_to_f2(v[c].x), f1 = bf16x2_to_f2(v[c].y), f2 = bf16x2_to_f2(v[c].z), f3 = bf16x2_to_f2(v[c].w);
+        acc[0] = fmaf(f0.x, zz[2 * c].x, fmaf(f0.y, zz[2 * c].y, acc[0]));
+        acc[1] = fmaf(f1.x, zz[2 * c].z, fmaf(f1.y, zz[2 * c].w, acc[1]));
+        acc[2] = fmaf(f2.x, zz[2 * c + 1].x, fmaf(f2.y, zz[2 * c + 1].y, acc[2]));
+        acc[3] = fmaf(f3.x, zz[2 * c + 1].z, fmaf(f3.y, zz[2 * c + 1].w, acc[3]));
       }
-      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    };
+    // this thread's row of tile `it` is rectified, and it has finished reading the accumulator
+    // buffer that tile's MMAs will overwrite (tile it - 2's)
+    auto publish_relu = [&](int it) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      mbar_arrive(&bars->relu_done[it & 1]);
+    };
+
+    // prologue: state in place, first tile rectified
+    ok = workers_sync() && ok;                         // KV and z written by all
+    int s = 0;
+    uint32_t par = 0;
+    float den_next = 0.f;
+    if (ok && ntiles > 0) {
+      ok = warp_wait(&bars->full[0], 0, &bars->abort_flag, status);
+      if (ok) {
+        den_next = relu_row(0);
+        publish_relu(0);
+      }
+    }
+    for (int it = 0; it < ntiles && ok; ++it) {
+      den = den_next;
+      // tile it + 1 through ReLU first, so that the tensor core works under this tile's epilogue
+      if (it + 1 < ntiles) {
+        int s1 = s + 1;
+        uint32_t par1 = par;
+        if (s1 == kApplyStages) { s1 = 0; par1 ^= 1; }
+        ok = warp_wait(&bars->full[s1], par1, &bars->abort_flag, status);
+        if (!ok) break;
+        den_next = relu_row(s1);
+        publish_relu(it + 1);
+      }
+      // epilogue of tile it
+      ok = warp_wait(&bars->d_full[it & 1], (it >> 1) & 1, &bars->abort_flag, status);
+      if (!ok) break;
+      tc_fence_after();
+      const float inv = 1.f / (den + eps);
+      // this warp's staging region (32 rows, 4 KB) of buffer it & 1: its last store must have been read
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      __syncwarp();
+      unsigned char* st = out_ptr + (it & 1) * kApplyTileBytes + row * 128;
+#pragma unroll
+      for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_base + (it & 1) * kD + 32 * c2, v);
+        tmem_wait_ld(v);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint4 w;
+          __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 0]) * inv, __uint_as_float(v[8 * c + 1]) * inv);
+          __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv);
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv);
+          __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv);
+          w.x = *reinterpret_cast<uint32_t*>(&h0);
+          w.y = *reinterpret_cast<uint32_t*>(&h1);
+          w.z = *reinterpret_cast<uint32_t*>(&h2);
+          w.w = *reinterpret_cast<uint32_t*>(&h3);
+          *reinterpret_cast<uint4*>(st + (((4 * c2 + c) ^ (row & 7)) << 4)) = w;
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        const int tok = t_begin + it * kApplyTok + 32 * warp;
+        if (tok < N)        // rows past N inside the box are clipped by the store itself
+          asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                       ::"l"(&mapO), "r"(out_sm + (it & 1) * kApplyTileBytes + warp * 4096), "r"(0), "r"(tok), "r"(bh) : "memory");
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+      if (++s == kApplyStages) { s = 0; par ^= 1; }
+    }
+    // the staging tiles must outlive the reads of the last stores
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    // every MMA issued has been waited for (d_full) unless a wait gave up; in that case give the
+    // tensor core the same bounded time before tensor memory is released
+    if (!ok && warp == 0 && lane == 0) {
+      const unsigned long long t0 = globaltimer();
+      while (globaltimer() - t0 < 1000000ull) {}
     }
   }
-  // the staging tiles must outlive the reads of the last stores
-  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kApplyTmemCols) : "memory");
 }
 
 // ---- o += depth-wise k x k convolution of V with the sample's kernels ------------------
@@ -686,8 +818,8 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   if (!status) return cudaErrorUnknown;
 
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map(&mq, a.q, BH, N, kTileTok) || !make_map(&mk, a.k, BH, N, kTileTok) ||
-      !make_map(&mv, a.v, BH, N, kTileTok) || !make_map(&mo, a.o, BH, N, 16))
+  if (!make_map(&mq, a.q, BH, N, kApplyTok) || !make_map(&mk, a.k, BH, N, kTileTok) ||
+      !make_map(&mv, a.v, BH, N, kTileTok) || !make_map(&mo, a.o, BH, N, 32))
     return cudaErrorInvalidValue;
 
   static bool attr_done = false;   // > 48 KB of dynamic shared memory needs the opt-in, once per process
@@ -707,12 +839,12 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
-  // apply pass: one wave of three CTAs per SM, spans of whole tiles; launched so that its set-up
-  // overlaps the tail of the state pass
-  int nspan = (3 * 148) / BH;
+  // apply pass: one wave of two CTAs per SM, spans of whole 128-token tiles; launched so that its
+  // set-up overlaps the tail of the state pass
+  int nspan = (2 * 148) / BH;
   if (nspan < 1) nspan = 1;
-  int span = ceil_div(ceil_div(N, nspan), kTileTok) * kTileTok;
-  if (span < 4 * kTileTok) span = 4 * kTileTok;
+  int span = ceil_div(ceil_div(N, nspan), kApplyTok) * kApplyTok;
+  if (span < 4 * kApplyTok) span = 4 * kApplyTok;
   nspan = ceil_div(N, span);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(nspan, BH);
