@@ -282,13 +282,16 @@ struct __align__(8) ApplyBars {
   uint64_t full[kApplyStages], empty[kApplyStages];
   uint64_t d_full[2];                         // accumulator of tile i ready (tcgen05.commit)
   uint64_t workers;                           // the 128 worker threads among themselves (once, after the state is in place)
-  uint64_t relu_done[2];                      // 128 arrivals per tile (tiles alternate): Q tile rectified, accumulator buffer free
+  uint64_t relu_done[kApplyStages];           // 128 arrivals: the Q tile in this ring slot is rectified, its denominators stored
+  uint64_t d_empty[2];                        // 128 arrivals: the epilogue has read this accumulator buffer
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
-// shared memory: Q ring | KV (bf16, swizzled) | output staging 2 x 16 KB | z (fp32) | barriers
-constexpr size_t kApplySmem =
-    (size_t)(kApplyStages + 2) * kApplyTileBytes + kTileBytes + 1024 + kD * sizeof(float) + sizeof(ApplyBars);
+constexpr int kApplyThreads = 288;                      // 4 rectifier warps, 1 producer / issuer warp, 4 epilogue warps
+constexpr int kDenRing = 8;                             // denominators of the tiles between ReLU and epilogue
+// shared memory: Q ring | output staging 2 x 16 KB | KV (bf16, swizzled) | z (fp32) | denominators | barriers
+constexpr size_t kApplySmem = (size_t)(kApplyStages + 2) * kApplyTileBytes + kTileBytes + 1024 + kD * sizeof(float) +
+                              (size_t)kDenRing * kApplyTok * sizeof(float) + sizeof(ApplyBars);
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -320,7 +323,7 @@ __device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
                :: "memory");
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kApplyThreads, 2)
 lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapO,
                  const float* __restrict__ partial, int* status, int N, int span_tokens, int nchunk, int state_elems,
                  float eps) {
@@ -332,7 +335,8 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   unsigned char* kv_ptr = out_ptr + 2 * kApplyTileBytes;                         // bf16 KV[a][e], swizzled
   const uint32_t kv_sm = out_sm + 2 * kApplyTileBytes;
   float* z_sm = reinterpret_cast<float*>(kv_ptr + kTileBytes);
-  ApplyBars* bars = reinterpret_cast<ApplyBars*>(z_sm + kD);
+  float* den_sm = z_sm + kD;                                                     // [kDenRing][128]
+  ApplyBars* bars = reinterpret_cast<ApplyBars*>(den_sm + kDenRing * kApplyTok);
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const int bh = blockIdx.y;
   const int t_begin = blockIdx.x * span_tokens, t_end = min(N, t_begin + span_tokens);
@@ -346,8 +350,9 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     mbar_init(&bars->d_full[0], 1);
     mbar_init(&bars->d_full[1], 1);
     mbar_init(&bars->workers, kConsumers);
-    mbar_init(&bars->relu_done[0], kConsumers);
-    mbar_init(&bars->relu_done[1], kConsumers);
+    for (int s = 0; s < kApplyStages; ++s) mbar_init(&bars->relu_done[s], kConsumers);
+    mbar_init(&bars->d_empty[0], kConsumers);
+    mbar_init(&bars->d_empty[1], kConsumers);
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -389,10 +394,11 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         }
         load_tile(nx);
       }
-      ok = warp_wait(&bars->relu_done[it & 1], (it >> 1) & 1, &bars->abort_flag, status);
+      const int s = it % kApplyStages, b = it & 1;
+      ok = warp_wait(&bars->relu_done[s], (it / kApplyStages) & 1, &bars->abort_flag, status);
+      if (ok && it >= 2) ok = warp_wait(&bars->d_empty[b], ((it >> 1) - 1) & 1, &bars->abort_flag, status);
       if (!ok) break;
       tc_fence_after();
-      const int s = it % kApplyStages, b = it & 1;
       const uint32_t qa = smem + s * kApplyTileBytes;
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks) {
@@ -414,8 +420,8 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       for (int g = max(0, issued - kApplyStages); g < issued; ++g)
         while (!mbar_try(&bars->full[g % kApplyStages], (g / kApplyStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
     }
-  } else {
-    // ================= worker warps: thread r = 32 warp + lane owns token row r of every tile =================
+  } else if (warp < 4) {
+    // ================= rectifier warps: thread r = 32 warp + lane owns token row r of every tile =================
     griddep_wait();                                    // the state pass (and anything before it) has completed
     bool ok = *reinterpret_cast<volatile int*>(status) == 0;
     {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
@@ -465,9 +471,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       tc_fence_after();
       return w_ok;
     };
-    const int row = threadIdx.x;                       // 0..127: token row of the tile and tensor-memory lane
-    const uint32_t lane_base = (uint32_t)(warp << 5) << 16;
-    float den = 0.f;
+    const int row = threadIdx.x;                       // 0..127: token row of the tile
 
     // ReLU of this thread's row of the Q tile in stage s, in place; returns relu(q).z.
     // All loads come before the stores (the compiler cannot tell that they do not alias).
@@ -476,98 +480,90 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       uint4 v[8];
 #pragma unroll
       for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const uint4*>(q + ((c ^ (row & 7)) << 4));
-      float4 zz[16];
-#pragma unroll
-      for (int c = 0; c < 16; ++c) zz[c] = *reinterpret_cast<const float4*>(z_sm + 4 * c);
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
         v[c].x = relu_bf16x2(v[c].x); v[c].y = relu_bf16x2(v[c].y); v[c].z = relu_bf16x2(v[c].z); v[c].w = relu_bf16x2(v[c].w);
-        *reinterpret_cast<uint4*>(q + ((c ^ (row & 7)) << 4)) = v[c];
+        const float4 za = *reinterpret_cast<const float4*>(z_sm + 8 * c), zb = *reinterpret_cast<const float4*>(z_sm + 8 * c + 4);
         const float2 f0 = bf16x2_to_f2(v[c].x), f1 = bf16x2_to_f2(v[c].y), f2 = bf16x2_to_f2(v[c].z), f3 = bf16x2_to_f2(v[c].w);
-        acc[0] = fmaf(f0.x, zz[2 * c].x, fmaf(f0.y, zz[2 * c].y, acc[0]));
-        acc[1] = fmaf(f1.x, zz[2 * c].z, fmaf(f1.y, zz[2 * c].w, acc[1]));
-        acc[2] = fmaf(f2.x, zz[2 * c + 1].x, fmaf(f2.y, zz[2 * c + 1].y, acc[2]));
-        acc[3] = fmaf(f3.x, zz[2 * c + 1].z, fmaf(f3.y, zz[2 * c + 1].w, acc[3]));
+        acc[0] = fmaf(f0.x, za.x, fmaf(f0.y, za.y, acc[0]));
+        acc[1] = fmaf(f1.x, za.z, fmaf(f1.y, za.w, acc[1]));
+        acc[2] = fmaf(f2.x, zb.x, fmaf(f2.y, zb.y, acc[2]));
+        acc[3] = fmaf(f3.x, zb.z, fmaf(f3.y, zb.w, acc[3]));
       }
+#pragma unroll
+      for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(q + ((c ^ (row & 7)) << 4)) = v[c];
       return (acc[0] + acc[1]) + (acc[2] + acc[3]);
     };
-    // this thread's row of tile `it` is rectified, and it has finished reading the accumulator
-    // buffer that tile's MMAs will overwrite (tile it - 2's)
-    auto publish_relu = [&](int it) {
+    // this thread's row of the tile in ring slot s is rectified and its denominator stored
+    auto publish_relu = [&](int s) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      tc_fence_before();
-      mbar_arrive(&bars->relu_done[it & 1]);
+      mbar_arrive(&bars->relu_done[s]);
     };
 
-    // prologue: state in place, first tile rectified
     ok = workers_sync() && ok;                         // KV and z written by all
     int s = 0;
     uint32_t par = 0;
-    float den_next = 0.f;
-    if (ok && ntiles > 0) {
-      ok = warp_wait(&bars->full[0], 0, &bars->abort_flag, status);
-      if (ok) {
-        den_next = relu_row(0);
-        publish_relu(0);
-      }
-    }
     for (int it = 0; it < ntiles && ok; ++it) {
-      den = den_next;
-      // tile it + 1 through ReLU first, so that the tensor core works under this tile's epilogue
-      if (it + 1 < ntiles) {
-        int s1 = s + 1;
-        uint32_t par1 = par;
-        if (s1 == kApplyStages) { s1 = 0; par1 ^= 1; }
-        ok = warp_wait(&bars->full[s1], par1, &bars->abort_flag, status);
-        if (!ok) break;
-        den_next = relu_row(s1);
-        publish_relu(it + 1);
-      }
-      // epilogue of tile it
-      ok = warp_wait(&bars->d_full[it & 1], (it >> 1) & 1, &bars->abort_flag, status);
+      ok = warp_wait(&bars->full[s], par, &bars->abort_flag, status);
+      if (!ok) break;
+      den_sm[(it & (kDenRing - 1)) * kApplyTok + row] = relu_row(s);
+      publish_relu(s);
+      if (++s == kApplyStages) { s = 0; par ^= 1; }
+    }
+  } else {
+    // ================= epilogue warps: thread (quadrant q = warp % 4, lane) owns row 32 q + lane =================
+    const int q4 = warp & 3, row = 32 * q4 + lane;
+    const uint32_t lane_base = (uint32_t)(q4 << 5) << 16;
+    bool ok = true;
+    for (int it = 0; it < ntiles && ok; ++it) {
+      const int b = it & 1;
+      // The tile's MMAs were issued after all 128 rectifier threads had published its rows and
+      // denominators, so the accumulator being complete means the denominators are in place.
+      ok = warp_wait(&bars->d_full[b], (it >> 1) & 1, &bars->abort_flag, status);
       if (!ok) break;
       tc_fence_after();
-      const float inv = 1.f / (den + eps);
-      // this warp's staging region (32 rows, 4 KB) of buffer it & 1: its last store must have been read
+      const float inv = 1.f / (den_sm[(it & (kDenRing - 1)) * kApplyTok + row] + eps);
+      uint32_t v0[32], v1[32];
+      tmem_ld32(tmem + lane_base + b * kD, v0);
+      tmem_ld32(tmem + lane_base + b * kD + 32, v1);
+      tmem_wait_ld(v0);
+      tmem_wait_ld(v1);
+      tc_fence_before();
+      mbar_arrive(&bars->d_empty[b]);                  // the accumulator buffer may be overwritten
+      // this warp's staging region (32 rows, 4 KB) of buffer b: its last store must have been read
       if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
       __syncwarp();
-      unsigned char* st = out_ptr + (it & 1) * kApplyTileBytes + row * 128;
+      unsigned char* st = out_ptr + b * kApplyTileBytes + row * 128;
 #pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + (it & 1) * kD + 32 * c2, v);
-        tmem_wait_ld(v);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint4 w;
-          __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 0]) * inv, __uint_as_float(v[8 * c + 1]) * inv);
-          __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv);
-          __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv);
-          __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv);
-          w.x = *reinterpret_cast<uint32_t*>(&h0);
-          w.y = *reinterpret_cast<uint32_t*>(&h1);
-          w.z = *reinterpret_cast<uint32_t*>(&h2);
-          w.w = *reinterpret_cast<uint32_t*>(&h3);
-          *reinterpret_cast<uint4*>(st + (((4 * c2 + c) ^ (row & 7)) << 4)) = w;
-        }
+      for (int c = 0; c < 8; ++c) {
+        const uint32_t* v = c < 4 ? v0 + 8 * c : v1 + 8 * (c - 4);
+        uint4 w;
+        __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[0]) * inv, __uint_as_float(v[1]) * inv);
+        __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[2]) * inv, __uint_as_float(v[3]) * inv);
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[4]) * inv, __uint_as_float(v[5]) * inv);
+        __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[6]) * inv, __uint_as_float(v[7]) * inv);
+        w.x = *reinterpret_cast<uint32_t*>(&h0);
+        w.y = *reinterpret_cast<uint32_t*>(&h1);
+        w.z = *reinterpret_cast<uint32_t*>(&h2);
+        w.w = *reinterpret_cast<uint32_t*>(&h3);
+        *reinterpret_cast<uint4*>(st + ((c ^ (row & 7)) << 4)) = w;
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) {
-        const int tok = t_begin + it * kApplyTok + 32 * warp;
+        const int tok = t_begin + it * kApplyTok + 32 * q4;
         if (tok < N)        // rows past N inside the box are clipped by the store itself
           asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-                       ::"l"(&mapO), "r"(out_sm + (it & 1) * kApplyTileBytes + warp * 4096), "r"(0), "r"(tok), "r"(bh) : "memory");
+                       ::"l"(&mapO), "r"(out_sm + b * kApplyTileBytes + q4 * 4096), "r"(0), "r"(tok), "r"(bh) : "memory");
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
-      if (++s == kApplyStages) { s = 0; par ^= 1; }
     }
     // the staging tiles must outlive the reads of the last stores
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     // every MMA issued has been waited for (d_full) unless a wait gave up; in that case give the
-    // tensor core the same bounded time before tensor memory is released
-    if (!ok && warp == 0 && lane == 0) {
+    // tensor core a bounded time before tensor memory is released
+    if (!ok && lane == 0) {
       const unsigned long long t0 = globaltimer();
       while (globaltimer() - t0 < 1000000ull) {}
     }
@@ -848,7 +844,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   nspan = ceil_div(N, span);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(nspan, BH);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(kApplyThreads);
   cfg.dynamicSmemBytes = kApplySmem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
