@@ -102,7 +102,6 @@ struct __align__(8) Barriers {
   uint64_t q_full[2], q_empty[2];                     // the two query buffers (items alternate)
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2][2], p_full[2][2], pv_done[2], o_full[2];
-  uint64_t wg_sync[2];                                // the 128 threads of a softmax warpgroup among themselves
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -405,7 +404,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       mbar_init(&bar->pv_done[t], 1);
       mbar_init(&bar->o_full[t], 1);
-      mbar_init(&bar->wg_sync[t], 128);
     }
     mbar_init(&bar->drain, 2);
     bar->abort_flag = 0;
@@ -679,14 +677,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     // store when the tile's box, clipped to the grid, lies inside the window (the store clips at
     // the grid edge by itself), row by row otherwise.
     struct Done {
-      bool have, store, tma;
+      bool have, store;
       int bh, qx0, qy0, x_end, y_end, par;
       float inv;
     } done{};
     done.have = false;
     const uint32_t sOt = sO + t * kTileBytes;
     unsigned char* sOt_ptr = smem + (size_t)(4 + 2 * kStages + t) * kTileBytes;
-    const bool store_leader = (threadIdx.x & 127) == 0;
     auto epi_load = [&](uint32_t (&ob)[32]) -> bool {
       if (!__all_sync(0xffffffffu, mbar_wait(&bar->o_full[t], done.par, bar, p.status))) return false;
       tc_fence_after();
@@ -701,30 +698,33 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       return true;
     };
-    uint32_t wg_par = 0;
-    // warpgroup-wide barrier with the same bounded wait as everything else (a plain bar.sync
-    // would wait for ever for a warp that has given up)
-    auto wg_barrier = [&]() -> bool {
-      mbar_arrive(&bar->wg_sync[t]);
-      const bool done_ok = mbar_wait(&bar->wg_sync[t], wg_par, bar, p.status);
-      wg_par ^= 1;
-      return __all_sync(0xffffffffu, done_ok);
-    };
+    // Each warp writes its own quarter of the tile (32 rows = a sub-box of the tile's box): no
+    // synchronisation beyond the warp.  One TMA store when the sub-box, clipped to the grid, holds
+    // tokens of this window only (the store clips at the grid edge by itself); row by row otherwise.
+    const int q4 = warp & 3;
+    int sub_x, sub_y;                                   // origin of this warp's sub-box inside the tile's box
+    if (p.box_h >= 4) { sub_x = 0; sub_y = q4 * (p.box_h >> 2); }
+    else { sub_x = (32 * q4) & (p.box_w - 1); sub_y = (32 * q4) >> lg_bw; }
+    const int sub_w = p.box_h >= 4 ? p.box_w : 32, sub_h = p.box_h >= 4 ? (p.box_h >> 2) : 1;
     auto epi_store = [&](const uint32_t (&ob)[32]) -> bool {
       if (!done.store) return true;
-      if (done.tma) {
-        // the previous store must have finished reading the staging tile
-        if (store_leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        if (!wg_barrier()) return false;
+      const int wx0 = done.qx0 + sub_x, wy0 = done.qy0 + sub_y;
+      if (wx0 >= done.x_end || wy0 >= done.y_end) return true;       // none of this warp's rows exists
+      const bool tma = p.step_x != 0 || ((wx0 + sub_w <= done.x_end || done.x_end == p.gridW) &&
+                                         (wy0 + sub_h <= done.y_end || done.y_end == p.gridH));
+      if (tma) {
+        // this warp's previous store must have finished reading its staging quarter
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
 #pragma unroll
         for (int c = 0; c < 8; ++c)     // 16-byte chunk c of this row, at its 128-byte-swizzle position
           *reinterpret_cast<uint4*>(sOt_ptr + row * 128 + ((c ^ (row & 7)) << 4)) =
               make_uint4(ob[4 * c], ob[4 * c + 1], ob[4 * c + 2], ob[4 * c + 3]);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (!wg_barrier()) return false;
-        if (store_leader) {
+        __syncwarp();
+        if (lane == 0) {
           asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-                       ::"l"(&mapO), "r"(sOt), "r"(0), "r"(done.qx0), "r"(done.qy0), "r"(done.bh) : "memory");
+                       ::"l"(&mapO), "r"(sOt + q4 * 4096), "r"(0), "r"(wx0), "r"(wy0), "r"(done.bh) : "memory");
           asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       } else {
@@ -871,9 +871,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       done.y_end = y_end;
       done.par = n & 1;
       done.inv = 1.f / l;
-      // one TMA store is right when the box, clipped to the grid, holds tokens of this window only
-      done.tma = p.step_x != 0 || ((x0 + p.box_w <= x_end || x_end == p.gridW) &&
-                                   (done.qy0 + p.box_h <= y_end || y_end == p.gridH));
       cur = nxt;
       ++n;
     }
@@ -882,7 +879,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (epi_load(ob)) ok = epi_store(ob);
     }
     // the staging tile must outlive the last store's reads; wait for the writes as well
-    if (store_leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // ================= common teardown =================
@@ -953,8 +950,12 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.gridW * kD * 2, (cuuint64_t)N * kD * 2};
   const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
+  // the output is stored per warp: a quarter of the tile's box (32 tokens)
+  const cuuint32_t qbox[4] = {(cuuint32_t)kD, (cuuint32_t)(g.box_h >= 4 ? g.box_w : 32),
+                              (cuuint32_t)(g.box_h >= 4 ? g.box_h / 4 : 1), 1};
   for (int i = 0; i < 4; ++i) {
-    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides, box, estr,
+    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides,
+                     i == 3 ? qbox : box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
