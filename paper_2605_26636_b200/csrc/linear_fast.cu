@@ -21,9 +21,8 @@
 // its first Q loads overlap the tail of the state kernel, and it waits for that grid
 // (griddepcontrol.wait) only before touching the partials.
 //
-// With the convolution on, two small kernels (the generator MLP) run in between, and
-// the apply kernel keeps a ring of V tiles covering the (k-1)/2 grid rows above and
-// below the tile it is working on.
+// With the convolution on, two small kernels (the generator MLP) and a TMA-staged
+// depth-wise convolution pass over V and o follow.
 //
 // Partial layout per (batch, head, chunk), in floats:
 //   [0, 4096) KV[a][e], [4096, 4160) z[a], [4160, 4224) vsum[e]
@@ -103,10 +102,6 @@ __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* m
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -616,13 +611,7 @@ dwc_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ 
   }
 }
 
-// ---- o += depth-wise 3 x 3 convolution of V: the tuned kernel ----------------------------------
-// CTA = 8 warps = a patch of 8 grid rows x 16 grid columns of one (batch, head); warp w owns row
-// y0 + w.  A lane owns 4 channels (8 bytes: 16 lanes cover the 128-byte token row, so every
-// access is a full line) and 8 consecutive tokens, and slides a 3 x 3 window of V along x: each
-// V element is unpacked once and used for three taps.  All loads of the thread are issued
-// before the arithmetic; rows y +- 1 come from L1 / L2 (neighbouring warps read them too).
-constexpr int kDwcCols = 16, kDwcRows = 8, kDwcRun = 8;
+// packed fp32x2 helpers of the convolution kernel
 __device__ __forceinline__ uint64_t pack2f(float lo, float hi) {
   uint64_t r;
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
@@ -633,73 +622,156 @@ __device__ __forceinline__ uint64_t fma2f(uint64_t a, uint64_t b, uint64_t c) {
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
   return d;
 }
-__global__ void __launch_bounds__(256, 2)
-dwc3_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ o, const float* __restrict__ w,
-                int H, int Hg, int Wg, int ncol_blocks) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int c4 = lane & 15, half = lane >> 4;              // channels 4 c4 .. 4 c4 + 3; tokens 8 half .. 8 half + 7
-  const int N = Hg * Wg, bh = blockIdx.y, b = bh / H, h = bh % H;
-  const int rb = blockIdx.x / ncol_blocks, cb = blockIdx.x % ncol_blocks;
-  const int y = rb * kDwcRows + warp, x0 = cb * kDwcCols + half * kDwcRun;
-  if (y >= Hg || x0 >= Wg) return;
-  const uint2* vb = reinterpret_cast<const uint2*>(v + (size_t)bh * N * kD) + c4;     // + token * 16
-  uint2* ob = reinterpret_cast<uint2*>(o + (size_t)bh * N * kD) + c4;
+// ---- o += depth-wise 3 x 3 convolution of V, staged through shared memory by TMA ----------------
+// Persistent CTAs loop over patches of 8 grid rows x 16 grid columns of one (batch, head).  Per
+// patch the producer warp brings in the 10 x 18 halo of V (out-of-grid taps arrive as the zeros
+// of the padding) and the 8 x 16 patch of o; warp w owns patch row w: a lane owns 4 channels
+// (8 bytes) and 8 consecutive tokens and slides the 3 x 3 window along x, adds the result to o in
+// place, and the warp writes its row back with one TMA store (clipped at the grid edge).
+constexpr int kDwStages = 2;
+constexpr int kDwVBytes = 10 * 18 * 128;            // 23040
+constexpr int kDwOBytes = 8 * 16 * 128;             // 16384
+constexpr int kDwStageBytes = 23552 + kDwOBytes;    // V halo (padded to a multiple of 512) + o patch
+constexpr int kDwThreads = 288;                     // 8 row warps + 1 producer warp
+struct __align__(8) DwBars {
+  uint64_t full[kDwStages], empty[kDwStages];
+  volatile uint32_t abort_flag;
+};
+constexpr size_t kDwSmem = (size_t)kDwStages * kDwStageBytes + 1024 + sizeof(DwBars);
 
-  // weights of this thread's 4 channels: w[ch][tap] -> per tap two fp32 pairs
-  uint64_t w01[9], w23[9];
-  {
-    const float4* wp = reinterpret_cast<const float4*>(w + ((size_t)b * H * kD + (size_t)h * kD + 4 * c4) * 9);
-    float wf[36];
-#pragma unroll
-    for (int i = 0; i < 9; ++i) {
-      const float4 t = __ldg(wp + i);
-      wf[4 * i] = t.x; wf[4 * i + 1] = t.y; wf[4 * i + 2] = t.z; wf[4 * i + 3] = t.w;
-    }
-#pragma unroll
-    for (int tap = 0; tap < 9; ++tap) {
-      w01[tap] = pack2f(wf[tap], wf[9 + tap]);
-      w23[tap] = pack2f(wf[18 + tap], wf[27 + tap]);
-    }
-  }
-  // all loads first: 3 rows x 10 columns of V (zeros outside the grid), 8 tokens of o
-  uint2 vr[3][kDwcRun + 2], cur[kDwcRun];
-#pragma unroll
-  for (int dy = 0; dy < 3; ++dy) {
-    const int yy = y + dy - 1;
-    const bool row_ok = yy >= 0 && yy < Hg;
-#pragma unroll
-    for (int i = 0; i < kDwcRun + 2; ++i) {
-      const int xx = x0 + i - 1;
-      vr[dy][i] = (row_ok && xx >= 0 && xx < Wg) ? __ldg(vb + (size_t)(yy * Wg + xx) * 16) : make_uint2(0u, 0u);
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < kDwcRun; ++i)
-    cur[i] = (x0 + i < Wg) ? ob[(size_t)(y * Wg + x0 + i) * 16] : make_uint2(0u, 0u);
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
 
-#pragma unroll
-  for (int i = 0; i < kDwcRun; ++i) {
-    uint64_t a01 = pack2f(__uint_as_float(cur[i].x << 16), __uint_as_float(cur[i].x & 0xffff0000u));
-    uint64_t a23 = pack2f(__uint_as_float(cur[i].y << 16), __uint_as_float(cur[i].y & 0xffff0000u));
-#pragma unroll
-    for (int dy = 0; dy < 3; ++dy)
-#pragma unroll
-      for (int dx = 0; dx < 3; ++dx) {
-        const uint2 t = vr[dy][i + dx];
-        a01 = fma2f(w01[3 * dy + dx], pack2f(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u)), a01);
-        a23 = fma2f(w23[3 * dy + dx], pack2f(__uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u)), a23);
+__global__ void __launch_bounds__(kDwThreads, 2)
+dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapOld,
+                const __grid_constant__ CUtensorMap mapOst, const float* __restrict__ w, int* status, int H,
+                int Hg, int ncol_blocks, int npatch, int total_items) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t smem = smem_u32(smem_al);
+  DwBars* bars = reinterpret_cast<DwBars*>(smem_al + (size_t)kDwStages * kDwStageBytes);
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kDwStages; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 8);            // one arrival per row warp
+    }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  if (*reinterpret_cast<volatile int*>(status) != 0) return;
+
+  if (warp == 8) {
+    // ================= TMA producer =================
+    int s = 0, issued = 0;
+    uint32_t par = 1;
+    bool ok = true;
+    for (int i = blockIdx.x; i < total_items; i += gridDim.x) {
+      ok = warp_wait(&bars->empty[s], par, &bars->abort_flag, status);
+      if (!ok) break;
+      if (elect_one()) {
+        const int bh = i / npatch, pt = i - bh * npatch;
+        const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
+        mbar_expect_tx(&bars->full[s], kDwVBytes + kDwOBytes);
+        tma_load_4d(smem + s * kDwStageBytes, &mapV, &bars->full[s], x0 - 1, y0 - 1, bh);
+        tma_load_4d(smem + s * kDwStageBytes + 23552, &mapOld, &bars->full[s], x0, y0, bh);
       }
-    if (x0 + i < Wg) {
-      float r0, r1, r2, r3;
-      asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(a01));
-      asm("mov.b64 {%0, %1}, %2;" : "=f"(r2), "=f"(r3) : "l"(a23));
-      __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
-      uint2 out;
-      out.x = *reinterpret_cast<uint32_t*>(&lo);
-      out.y = *reinterpret_cast<uint32_t*>(&hi);
-      ob[(size_t)(y * Wg + x0 + i) * 16] = out;
+      __syncwarp();
+      ++issued;
+      if (++s == kDwStages) { s = 0; par ^= 1; }
     }
+    if (!ok && lane == 0) {
+      const unsigned long long t0 = globaltimer();
+      for (int g = max(0, issued - kDwStages); g < issued; ++g)
+        while (!mbar_try(&bars->full[g % kDwStages], (g / kDwStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
+    }
+    return;
   }
+
+  // ================= row warps =================
+  const int c4 = lane & 15, half = lane >> 4;              // channels 4 c4 .. 4 c4 + 3; tokens 8 half .. 8 half + 7
+  uint64_t w01[9], w23[9];
+  int cur_bh = -1;
+  int s = 0;
+  uint32_t par = 0;
+  bool ok = true;
+  for (int i = blockIdx.x; i < total_items && ok; i += gridDim.x) {
+    const int bh = i / npatch, pt = i - bh * npatch;
+    const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
+    if (bh != cur_bh) {      // weights of this thread's 4 channels: w[ch][tap] -> per tap two fp32 pairs
+      cur_bh = bh;
+      const int b = bh / H, h = bh - b * H;
+      const float4* wp = reinterpret_cast<const float4*>(w + ((size_t)b * H * kD + (size_t)h * kD + 4 * c4) * 9);
+      float wf[36];
+#pragma unroll
+      for (int k = 0; k < 9; ++k) {
+        const float4 t4 = __ldg(wp + k);
+        wf[4 * k] = t4.x; wf[4 * k + 1] = t4.y; wf[4 * k + 2] = t4.z; wf[4 * k + 3] = t4.w;
+      }
+#pragma unroll
+      for (int tap = 0; tap < 9; ++tap) {
+        w01[tap] = pack2f(wf[tap], wf[9 + tap]);
+        w23[tap] = pack2f(wf[18 + tap], wf[27 + tap]);
+      }
+    }
+    ok = warp_wait(&bars->full[s], par, &bars->abort_flag, status);
+    if (!ok) break;
+    const unsigned char* vs = smem_al + (size_t)s * kDwStageBytes + c4 * 8;            // halo: [10][18][128 B]
+    unsigned char* os = smem_al + (size_t)s * kDwStageBytes + 23552 + (warp * 16 + half * 8) * 128 + c4 * 8;
+#pragma unroll
+    for (int hk = 0; hk < 2; ++hk) {                       // two runs of four tokens: keeps the window in registers
+      uint2 vr[3][6], cur[4];
+#pragma unroll
+      for (int dy = 0; dy < 3; ++dy)
+#pragma unroll
+        for (int k = 0; k < 6; ++k)
+          vr[dy][k] = *reinterpret_cast<const uint2*>(vs + ((warp + dy) * 18 + half * 8 + 4 * hk + k) * 128);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) cur[k] = *reinterpret_cast<const uint2*>(os + (4 * hk + k) * 128);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint64_t a01 = pack2f(__uint_as_float(cur[k].x << 16), __uint_as_float(cur[k].x & 0xffff0000u));
+        uint64_t a23 = pack2f(__uint_as_float(cur[k].y << 16), __uint_as_float(cur[k].y & 0xffff0000u));
+#pragma unroll
+        for (int dy = 0; dy < 3; ++dy)
+#pragma unroll
+          for (int dx = 0; dx < 3; ++dx) {
+            const uint2 t2 = vr[dy][k + dx];
+            a01 = fma2f(w01[3 * dy + dx], pack2f(__uint_as_float(t2.x << 16), __uint_as_float(t2.x & 0xffff0000u)), a01);
+            a23 = fma2f(w23[3 * dy + dx], pack2f(__uint_as_float(t2.y << 16), __uint_as_float(t2.y & 0xffff0000u)), a23);
+          }
+        float r0, r1, r2, r3;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(a01));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(r2), "=f"(r3) : "l"(a23));
+        __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+        uint2 out;
+        out.x = *reinterpret_cast<uint32_t*>(&lo);
+        out.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(os + (4 * hk + k) * 128) = out;
+      }
+    }
+    // this warp's row (16 tokens, 2 KB) back to global memory; the stage is free once the store has read it
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (lane == 0) {
+      if (y0 + warp < Hg)      // a row below the grid is not stored at all; columns past the edge are clipped by the store
+        asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                   ::"l"(&mapOst), "r"(smem + s * kDwStageBytes + 23552 + warp * 2048), "r"(0), "r"(x0), "r"(y0 + warp), "r"(bh)
+                   : "memory");
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+      mbar_arrive(&bars->empty[s]);
+    }
+    __syncwarp();
+    if (++s == kDwStages) { s = 0; par ^= 1; }
+  }
+  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 // ---- kernel generator of the squeeze dynamic convolution (Sec. 3.2.1), tuned for latency ------
@@ -798,6 +870,19 @@ bool make_map(CUtensorMap* m, const void* ptr, int BH, int N, int box_tok) {
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// [BH, Hg, Wg, 64] bf16 as a 4-D tensor (channel, x, y, batch*head), no swizzle
+bool make_map_grid(CUtensorMap* m, const void* ptr, int BH, int Hg, int Wg, int box_x, int box_y) {
+  EncodeFn enc = encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)Wg, (cuuint64_t)Hg, (cuuint64_t)BH};
+  const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)Wg * kD * 2, (cuuint64_t)Hg * Wg * kD * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)box_x, (cuuint32_t)box_y, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool linear_fast_supported(const LinArgs& a) {
@@ -809,7 +894,6 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   const int N = s.Hg * s.Wg, BH = s.B * s.H;
   char* ws = (char*)a.ws;
   float* partial = (float*)(ws + p.off_partial);
-  float* state = (float*)(ws + p.off_state);
   int* status = device_status_ptr();
   if (!status) return cudaErrorUnknown;
 
@@ -873,8 +957,20 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     const int run = 32;
     dim3 g4(ceil_div(ceil_div(N, run), 8), BH);
     if (a.dwc->k == 3) {
-      const int ncb = ceil_div(s.Wg, kDwcCols);
-      dwc3_add_kernel<<<dim3(ncb * ceil_div(s.Hg, kDwcRows), BH), 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, ncb);
+      CUtensorMap mvg, mol, mos;
+      if (!make_map_grid(&mvg, a.v, BH, s.Hg, s.Wg, 18, 10) || !make_map_grid(&mol, a.o, BH, s.Hg, s.Wg, 16, 8) ||
+          !make_map_grid(&mos, a.o, BH, s.Hg, s.Wg, 16, 1))
+        return cudaErrorInvalidValue;
+      static bool dw_attr = false;
+      if (!dw_attr) {
+        if ((e = cudaFuncSetAttribute(dwc3_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDwSmem)) != cudaSuccess) return e;
+        dw_attr = true;
+      }
+      const int ncb = ceil_div(s.Wg, 16), npatch = ncb * ceil_div(s.Hg, 8);
+      const long long items = (long long)npatch * BH;
+      if (items > 0x7fffffffll) return cudaErrorInvalidValue;
+      const int grid = (int)(items < 2 * 148 ? items : 2 * 148);
+      dwc3_tma_kernel<<<grid, kDwThreads, kDwSmem, st>>>(mvg, mol, mos, w, status, s.H, s.Hg, ncb, npatch, (int)items);
     } else
       dwc_add_kernel<5><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
     count_launch();
