@@ -363,6 +363,11 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
 
+  // A grid launched behind this one with programmatic serialisation (the convolution's generator)
+  // may start once every thread here has passed this point; the rectifier warps pass it only
+  // after the state pass is complete, which is all the generator depends on.
+  if (warp >= 4) griddep_launch_dependents();
+
   if (warp == 4) {
     // ================= TMA producer and MMA issuer (one elected lane) =================
     // Q does not depend on the state pass: the first loads start at once.  Per tile: refill the
@@ -418,6 +423,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   } else if (warp < 4) {
     // ================= rectifier warps: thread r = 32 warp + lane owns token row r of every tile =================
     griddep_wait();                                    // the state pass (and anything before it) has completed
+    griddep_launch_dependents();
     bool ok = *reinterpret_cast<volatile int*>(status) == 0;
     {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
       const float* P = partial + (size_t)bh * nchunk * state_elems;
@@ -781,6 +787,7 @@ __global__ void __launch_bounds__(128)
 gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W1, const float* __restrict__ b1,
                   float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n) {
   __shared__ float red[4];
+  griddep_launch_dependents();
   const int r = blockIdx.x, b = blockIdx.y, C = H * kD;
   float s = 0.f;
   for (int c = threadIdx.x; c < C; c += 128) {
@@ -804,6 +811,7 @@ gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W
 __global__ void __launch_bounds__(256)
 gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, const float* __restrict__ b2,
                float* __restrict__ w, int B, int T, int R) {
+  griddep_wait();                                      // the hidden layer (launched just before) is complete
   const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
   const bool t_ok = t < T;
   const float* wrow = W2 + (size_t)(t_ok ? t : 0) * R;
@@ -947,12 +955,26 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     const jv_dwc& d = *a.dwc;
     float* hidden = (float*)(ws + p.off_hidden);
     float* wk = (float*)(ws + p.off_kernel);
-    gen_hidden_kernel<<<dim3(d.R, s.B), 128, 0, st>>>(partial, d.W1, d.b1, hidden, s.H, d.R, p.nchunk, p.state_elems,
-                                                      1.f / (float)N);
-    count_launch();
+    // Both generator kernels run beside the apply pass: they are launched with programmatic
+    // serialisation, the first one does not wait for the apply grid (it needs the state pass only,
+    // which the apply grid has waited for before it lets its dependents start), the second one
+    // waits for the first.
     const int T = s.H * kD * d.k * d.k;
-    gen_out_kernel<<<ceil_div(T, 32), 256, 0, st>>>(hidden, d.W2, d.b2, wk, s.B, T, d.R);
+    cudaLaunchConfig_t gcfg = {};
+    gcfg.stream = st;
+    gcfg.attrs = attr;
+    gcfg.numAttrs = 1;
+    gcfg.gridDim = dim3(d.R, s.B);
+    gcfg.blockDim = dim3(128);
+    e = cudaLaunchKernelEx(&gcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
+                           p.nchunk, p.state_elems, 1.f / (float)N);
     count_launch();
+    if (e != cudaSuccess) return e;
+    gcfg.gridDim = dim3(ceil_div(T, 32));
+    gcfg.blockDim = dim3(256);
+    e = cudaLaunchKernelEx(&gcfg, gen_out_kernel, (const float*)hidden, d.W2, d.b2, wk, (int)s.B, T, (int)d.R);
+    count_launch();
+    if (e != cudaSuccess) return e;
     const float* w = (const float*)(ws + p.off_kernel);
     const int run = 32;
     dim3 g4(ceil_div(ceil_div(N, run), 8), BH);
