@@ -64,10 +64,15 @@ typedef struct {
  * Kernel generator of the squeeze dynamic depth-wise convolution (Sec. 3.2.1):
  * a two-layer MLP with SiLU fed by the average-pooled V.  All pointers are
  * DEVICE pointers to fp32, row-major; C = H * D, channel c = h * D + e.
+ *
+ * R = 0 selects the static depth-wise convolution the paper compares against
+ * (Sec. 3.2.1, Table 1 "DWC"): no generator, b2 holds the kernels themselves
+ * ([C, k, k], shared by every sample and required); W1, b1 and W2 are ignored
+ * and may be NULL.
  */
 typedef struct {
   int32_t k;       /* odd kernel edge: 3 or 5 */
-  int32_t R;       /* hidden width of the generator, 1..1024 */
+  int32_t R;       /* hidden width of the generator, 1..1024; 0 = static kernels in b2 */
   const float* W1; /* [R, C] */
   const float* b1; /* [R] or NULL */
   const float* W2; /* [C*k*k, R] */

@@ -119,11 +119,16 @@ def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None) -> np.ndarray:
                                 0, 0, None, None, None, None)
         return o
     kk, R = int(dwc["k"]), int(dwc["R"])
-    W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
+    C = H * D
     b1 = None if dwc.get("b1") is None else _f64(dwc["b1"])
     b2 = None if dwc.get("b2") is None else _f64(dwc["b2"])
-    C = H * D
-    assert kk % 2 == 1 and W1.shape == (R, C) and W2.shape == (C * kk * kk, R)
+    if R == 0:      # static depth-wise convolution (Table 1 "DWC"): the kernels are b2, no generator
+        assert b2 is not None and b2.size == C * kk * kk
+        W1 = W2 = None
+    else:
+        W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
+        assert W1.shape == (R, C) and W2.shape == (C * kk * kk, R)
+    assert kk % 2 == 1
     _load().jvo_linear_attn(_p(q), _p(k), _p(v), _p(o), B, H, Hg, Wg, D, float(eps),
                             kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
     return o

@@ -964,12 +964,14 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     gcfg.stream = st;
     gcfg.attrs = attr;
     gcfg.numAttrs = 1;
-    gcfg.gridDim = dim3(d.R, s.B);
-    gcfg.blockDim = dim3(128);
-    e = cudaLaunchKernelEx(&gcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
-                           p.nchunk, p.state_elems, 1.f / (float)N);
-    count_launch();
-    if (e != cudaSuccess) return e;
+    if (d.R > 0) {           // R == 0: static kernels, the output layer below just broadcasts b2
+      gcfg.gridDim = dim3(d.R, s.B);
+      gcfg.blockDim = dim3(128);
+      e = cudaLaunchKernelEx(&gcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
+                             p.nchunk, p.state_elems, 1.f / (float)N);
+      count_launch();
+      if (e != cudaSuccess) return e;
+    }
     gcfg.gridDim = dim3(ceil_div(T, 32));
     gcfg.blockDim = dim3(256);
     e = cudaLaunchKernelEx(&gcfg, gen_out_kernel, (const float*)hidden, d.W2, d.b2, wk, (int)s.B, T, (int)d.R);

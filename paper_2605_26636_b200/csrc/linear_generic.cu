@@ -231,9 +231,11 @@ cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float
   float* hidden = (float*)(ws + p.off_hidden);
   float* w = (float*)(ws + p.off_kernel);
   const int N = s.Hg * s.Wg;
-  dim3 g1(ceil_div(d.R * 32, 256), s.B);
-  dwc_hidden_kernel<<<g1, 256, 0, st>>>(vsum, d.W1, d.b1, hidden, s.H, s.D, d.R, bh_stride, 1.f / (float)N);
-  count_launch();
+  if (d.R > 0) {   // R == 0: static kernels, the output layer just broadcasts b2
+    dim3 g1(ceil_div(d.R * 32, 256), s.B);
+    dwc_hidden_kernel<<<g1, 256, 0, st>>>(vsum, d.W1, d.b1, hidden, s.H, s.D, d.R, bh_stride, 1.f / (float)N);
+    count_launch();
+  }
   const int T = s.H * s.D * d.k * d.k;
   dwc_out_kernel<<<ceil_div(T * 32, 256), 256, 0, st>>>(hidden, d.W2, d.b2, w, s.B, T, d.R);
   count_launch();

@@ -116,12 +116,13 @@ def make_dwc(d: Optional[dict], device) -> Optional[JvDwc]:
     alive until the call has been enqueued."""
     if d is None:
         return None
-    for key in ("W1", "W2"):
-        t = d[key]
-        if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+    static = int(d["R"]) == 0          # static kernels in b2: no generator weights
+    for key in (("b2",) if static else ("W1", "W2")):
+        t = d.get(key)
+        if t is None or not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
             raise ValueError(f"dwc[{key!r}] must be a contiguous fp32 CUDA tensor")
     ptr = lambda t: None if t is None else t.data_ptr()
-    return JvDwc(int(d["k"]), int(d["R"]), ptr(d["W1"]), ptr(d.get("b1")), ptr(d["W2"]), ptr(d.get("b2")))
+    return JvDwc(int(d["k"]), int(d["R"]), ptr(d.get("W1")), ptr(d.get("b1")), ptr(d.get("W2")), ptr(d.get("b2")))
 
 
 def _stream(stream) -> int:

@@ -67,6 +67,11 @@ def test_argument_errors_are_found_before_any_launch(L):
     assert _call_linear(L, shp, ws_bytes=16) == jv.JV_ERR_WORKSPACE
     bad = jv.JvDwc(4, 8, 1, None, 1, None)
     assert _call_linear(L, shp, dwc=ctypes.byref(bad)) == jv.JV_ERR_INVALID_ARG
+    static_ok = jv.JvDwc(3, 0, None, None, None, 4096)          # R = 0: static kernels in b2
+    static_bad = jv.JvDwc(3, 0, None, None, None, None)
+    assert _call_linear(L, shp, dwc=ctypes.byref(static_bad)) == jv.JV_ERR_INVALID_ARG
+    if not torch.cuda.is_available():   # with fake addresses a call that passes validation may only run where nothing can launch
+        assert _call_linear(L, shp, dwc=ctypes.byref(static_ok)) in (jv.JV_ERR_CUDA, jv.JV_ERR_UNSUPPORTED)
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 64, 7)) == jv.JV_ERR_INVALID_ARG
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 0, jv.JV_F32)) == jv.JV_ERR_INVALID_ARG
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 512, jv.JV_F32)) == jv.JV_ERR_UNSUPPORTED

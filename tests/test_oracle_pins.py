@@ -297,6 +297,23 @@ def test_dwc_static_equals_library_depthwise_conv(oracle, ksz):
     np.testing.assert_allclose(o - la, _from_image(conv.numpy(), H, D), rtol=0, atol=1e-12)
 
 
+@pytest.mark.parametrize("ksz", [3, 5])
+def test_dwc_static_variant_r0_equals_library_depthwise_conv(oracle, ksz):
+    """R = 0 (static kernels passed in b2, no generator: the "DWC" row of Table 1) against a
+    float64 library depth-wise conv2d, and against the generator forced to the same constants."""
+    r = _rng(33)
+    B, H, Hg, Wg, D = 2, 2, 5, 9, 4
+    C = H * D
+    q, k, v = (r.standard_normal((B, H, Hg * Wg, D)) for _ in range(3))
+    kernel = r.standard_normal((C, ksz, ksz))
+    la = oracle.linear_attn(q, k, v, Hg, Wg)
+    o = oracle.linear_attn(q, k, v, Hg, Wg, dwc={"k": ksz, "R": 0, "b2": kernel.reshape(-1)})
+    conv = torch.nn.functional.conv2d(torch.from_numpy(_to_image(v, Hg, Wg)),
+                                      torch.from_numpy(kernel)[:, None], padding=ksz // 2, groups=C)
+    np.testing.assert_allclose(o - la, _from_image(conv.numpy(), H, D), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(o, oracle.linear_attn(q, k, v, Hg, Wg, dwc=_static_dwc(C, ksz, kernel)), rtol=0, atol=1e-12)
+
+
 def test_dwc_delta_kernel_adds_v_and_constant_v_shows_padding(oracle):
     r = _rng(31)
     B, H, Hg, Wg, D = 1, 2, 5, 6, 4

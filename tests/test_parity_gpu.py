@@ -111,6 +111,20 @@ def test_sweep_linear_dwc_ragged(jv, oracle, both_paths, dtype):
     assert rel_err(out, oracle.linear_attn(q, k, v, Hg, Wg, dwc=d)) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("ksz", [3, 5])
+def test_linear_with_static_dwc(jv, oracle, both_paths, dtype, ksz):
+    """R = 0: the static depth-wise convolution of Table 1 (kernels passed directly in b2)."""
+    B, H, Hg, Wg, D = 2, 2, 21, 18, 64
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, D, dtype, seed=40 + ksz)
+    kern = inputs.normal((H * D * ksz * ksz,), inputs.SEED_BASE + 777 + ksz) * 0.2
+    d = {"k": ksz, "R": 0, "b2": kern}
+    out, check = guarded_empty(q.shape, _dev((q,))[0].dtype, DEV)
+    jv.linear_attn(*_dev((q, k, v)), Hg, Wg, dwc={"k": ksz, "R": 0, "b2": kern.to(DEV)}, out=out)
+    check()
+    assert rel_err(out, oracle.linear_attn(q, k, v, Hg, Wg, dwc=d)) <= TOL[dtype]
+
+
 def test_explicit_scale_and_eps(jv, oracle, both_paths):
     q, k, v = inputs.custom_qkv(1, 2, 16 * 16, 64, "bf16", seed=8)
     dq, dk, dv = _dev((q, k, v))
