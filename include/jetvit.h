@@ -171,6 +171,30 @@ jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* c
                            const jv_dwc* const* dwc, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The projections either side of a mixer (the W_Q, W_K, W_V and W_O that a searched model
+ * inherits from its base model for every block, Sec. 3.3), as tensor-core GEMMs that write
+ * and read the mixers' [B, H, N, D] layout directly: no transpose pass between projection
+ * and mixer.  bf16 only, D = 64 only (JV_ERR_UNSUPPORTED otherwise); C = H * D.
+ *
+ * jv_qkv_proj:  x [B, N, C] (token-major activations), w [3C, C] row-major (output feature
+ *   by input feature, the rows ordered q | k | v and, inside each, head-major: row
+ *   which*C + h*D + e), bias fp32 [3C] or NULL.
+ *     q[b, h, n, e] = sum_c x[b, n, c] * w[0*C + h*D + e, c] + bias[0*C + h*D + e]
+ *   and likewise k (which = 1) and v (which = 2).
+ * jv_out_proj:  o [B, H, N, D] (a mixer's output), w [C, C] row-major, bias fp32 [C] or NULL.
+ *     y[b, n, f] = sum_{h, e} o[b, h, n, e] * w[f, h*D + e] + bias[f]          y: [B, N, C]
+ *
+ * Products in bf16 on the tensor cores with fp32 accumulation; the bias is added in fp32
+ * and the result rounded to bf16 once (round to nearest even).  All pointers are DEVICE
+ * pointers, 16-byte aligned; outputs must not alias inputs.  No scratch.  Errors as for the
+ * mixers: argument errors are found on the host before anything is launched.
+ */
+jv_status jv_qkv_proj(const void* x, const void* w, const float* bias, void* q, void* k, void* v,
+                      const jv_shape* shape, void* cuda_stream);
+jv_status jv_out_proj(const void* o, const void* w, const float* bias, void* y, const jv_shape* shape,
+                      void* cuda_stream);
+
+/*
  * Synchronises the stream, then returns and clears the sticky device status:
  * JV_OK, JV_ERR_TIMEOUT if a kernel abandoned a bounded wait since the last
  * call, or JV_ERR_CUDA if the stream reports a CUDA error.

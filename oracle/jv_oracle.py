@@ -150,3 +150,41 @@ def hybrid_mixers(schedule, q, k, v, Hg, Wg, win_h, win_w, scale=None, eps=1e-6,
         else:
             raise ValueError(f"schedule[{l}] = {m!r}: expected one of L, W, F")
     return out
+
+
+def qkv_proj(x, w, bias, H):
+    """The block's input projection W_Q | W_K | W_V (Sec. 3.3: inherited linear layers),
+    written out as the definition: x [B, N, C], w [3C, C] (row = output feature
+    which*C + h*D + e), bias [3C] or None -> q, k, v, each [B, H, N, D] with D = C / H:
+    q[b, h, n, e] = sum_c x[b, n, c] w[h*D + e, c] + bias[h*D + e], and k, v from the
+    next two row blocks of w."""
+    x, w = _f64(x), _f64(w)
+    B, N, C = x.shape
+    assert C % H == 0 and w.shape == (3 * C, C)
+    D = C // H
+    y = x @ w.T                                    # [B, N, 3C]
+    if bias is not None:
+        y = y + _f64(bias).reshape(1, 1, 3 * C)
+    out = []
+    for which in range(3):
+        t = np.empty((B, H, N, D), dtype=np.float64)
+        for h in range(H):
+            t[:, h] = y[:, :, which * C + h * D: which * C + (h + 1) * D]
+        out.append(t)
+    return tuple(out)
+
+
+def out_proj(o, w, bias):
+    """The block's output projection W_O (Sec. 3.3): o [B, H, N, D], w [C, C] with C = H*D
+    (column = input feature h*D + e), bias [C] or None -> y [B, N, C]:
+    y[b, n, f] = sum_{h, e} o[b, h, n, e] w[f, h*D + e] + bias[f]."""
+    o, w = _f64(o), _f64(w)
+    B, H, N, D = o.shape
+    C = H * D
+    assert w.shape == (C, C)
+    y = np.zeros((B, N, C), dtype=np.float64)
+    for h in range(H):
+        y += o[:, h] @ w[:, h * D:(h + 1) * D].T
+    if bias is not None:
+        y = y + _f64(bias).reshape(1, 1, C)
+    return y

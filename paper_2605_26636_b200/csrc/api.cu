@@ -69,6 +69,18 @@ jv_status check_device() {
   return major == 10 ? JV_OK : JV_ERR_UNSUPPORTED;
 }
 
+jv_status check_proj(const jv_shape* s, const void* const* ptrs, int nptr, int nin) {
+  jv_status st = check_shape(s);
+  if (st != JV_OK) return st;
+  for (int i = 0; i < nptr; ++i)
+    if (!ptrs[i] || !aligned(ptrs[i], 16)) return JV_ERR_INVALID_ARG;
+  for (int i = nin; i < nptr; ++i)           // outputs alias neither an input nor each other
+    for (int j = 0; j < i; ++j)
+      if (ptrs[i] == ptrs[j]) return JV_ERR_INVALID_ARG;
+  if (s->dtype != JV_BF16 || s->D != 64) return JV_ERR_UNSUPPORTED;
+  return JV_OK;
+}
+
 jv_status from_cuda(cudaError_t e) { return e == cudaSuccess ? JV_OK : JV_ERR_CUDA; }
 
 float pick_scale(float scale, int D) { return scale > 0.f ? scale : 1.f / sqrtf((float)D); }
@@ -199,6 +211,32 @@ jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* c
     if (st != JV_OK) return st;
   }
   return JV_OK;
+}
+
+jv_status jv_qkv_proj(const void* x, const void* w, const float* bias, void* q, void* k, void* v,
+                      const jv_shape* shape, void* cuda_stream) {
+  const void* ptrs[5] = {x, w, q, k, v};
+  jv_status st = check_proj(shape, ptrs, 5, 2);
+  if (st != JV_OK) return st;
+  if (bias && !aligned(bias, 16)) return JV_ERR_INVALID_ARG;
+  if ((st = check_device()) != JV_OK) return st;
+  if (!proj_tc_available()) return JV_ERR_CUDA;
+  int* status = device_status_ptr();
+  if (!status) return JV_ERR_CUDA;
+  return from_cuda(launch_proj_tc(true, x, w, bias, q, k, v, *shape, status, (cudaStream_t)cuda_stream));
+}
+
+jv_status jv_out_proj(const void* o, const void* w, const float* bias, void* y, const jv_shape* shape,
+                      void* cuda_stream) {
+  const void* ptrs[3] = {o, w, y};
+  jv_status st = check_proj(shape, ptrs, 3, 2);
+  if (st != JV_OK) return st;
+  if (bias && !aligned(bias, 16)) return JV_ERR_INVALID_ARG;
+  if ((st = check_device()) != JV_OK) return st;
+  if (!proj_tc_available()) return JV_ERR_CUDA;
+  int* status = device_status_ptr();
+  if (!status) return JV_ERR_CUDA;
+  return from_cuda(launch_proj_tc(false, o, w, bias, y, nullptr, nullptr, *shape, status, (cudaStream_t)cuda_stream));
 }
 
 jv_status jv_device_status(void* cuda_stream) {

@@ -83,4 +83,10 @@ cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float
 cudaError_t launch_lin_reduce(const float* partial, float* state, int nchunk, int state_elems, size_t total,
                               cudaStream_t st);
 
+// Projections either side of a mixer (bf16, D == 64): qkv = true computes q, k, v (d0, d1, d2)
+// from x [B, N, C]; qkv = false computes y (d0) [B, N, C] from x = o [B, H, N, 64].
+bool proj_tc_available();
+cudaError_t launch_proj_tc(bool qkv, const void* x, const void* w, const float* bias, void* d0, void* d1, void* d2,
+                           const jv_shape& s, int* status, cudaStream_t st);
+
 }  // namespace jv

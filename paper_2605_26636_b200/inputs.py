@@ -93,3 +93,12 @@ def dwc_weights(C: int, R: int, k: int, seed: int):
     b2[:, k // 2, k // 2] = 0.1
     return {"k": k, "R": R, "W1": torch.from_numpy(W1), "b1": torch.from_numpy(b1),
             "W2": torch.from_numpy(W2), "b2": torch.from_numpy(b2.reshape(-1))}
+
+
+def proj_weights(rows: int, C: int, seed: int, with_bias: bool = True):
+    """Weights of a linear projection as a trained layer would hold them: w ~ N(0, 1/C)
+    [rows, C] rounded to bf16, bias ~ 0.1 N(0, 1) fp32 [rows] (or None)."""
+    rng = np.random.default_rng(seed)
+    w = (rng.standard_normal((rows, C), dtype=np.float32) / np.sqrt(C)).astype(np.float32)
+    b = (0.1 * rng.standard_normal((rows,), dtype=np.float32)).astype(np.float32) if with_bias else None
+    return torch.from_numpy(w).to(torch.bfloat16), (None if b is None else torch.from_numpy(b))

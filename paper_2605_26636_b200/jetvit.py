@@ -59,7 +59,10 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(vp), ctypes.POINTER(vp), shp, i32, i32, f32, f32,
                                        ctypes.POINTER(dwc), vp, sz, vp]
         L.jv_device_status.argtypes = [vp]
-        for f in (L.jv_linear_attn, L.jv_window_attn, L.jv_full_attn, L.jv_hybrid_mixers, L.jv_device_status):
+        L.jv_qkv_proj.argtypes = [vp, vp, vp, vp, vp, vp, shp, vp]
+        L.jv_out_proj.argtypes = [vp, vp, vp, vp, shp, vp]
+        for f in (L.jv_linear_attn, L.jv_window_attn, L.jv_full_attn, L.jv_hybrid_mixers, L.jv_device_status,
+                  L.jv_qkv_proj, L.jv_out_proj):
             f.restype = ctypes.c_int
         L.jv_set_force_generic.argtypes = [i32]
         L.jv_set_force_generic.restype = i32
@@ -245,6 +248,56 @@ def hybrid_mixers(schedule: str, q: Sequence[torch.Tensor], k, v, Hg: int, Wg: i
                                     int(win_h), int(win_w), float(scale), float(eps), dptr, wp, wn, _stream(stream))
     _raise(st, "jv_hybrid_mixers")
     return out
+
+
+def _check_proj(x, w, bias, H: int, rows: int):
+    C = 64 * H
+    for t in (x, w):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()):
+            raise ValueError("projection operands must be contiguous bf16 CUDA tensors")
+    if tuple(w.shape) != (rows, C):
+        raise ValueError(f"w must be [{rows}, {C}]")
+    if bias is not None and not (bias.is_cuda and bias.dtype == torch.float32 and bias.is_contiguous()
+                                 and tuple(bias.shape) == (rows,)):
+        raise ValueError(f"bias must be a contiguous fp32 CUDA tensor of [{rows}]")
+
+
+def qkv_proj(x, w, bias, H: int, Hg: int, Wg: int, out=None, stream=None):
+    """jv_qkv_proj: x [B, N, C] bf16, w [3C, C] bf16, bias fp32 [3C] or None -> (q, k, v), each
+    [B, H, N, 64] in the mixers' layout.  ``out`` is an optional (q, k, v) triple to write into."""
+    B, N, C = x.shape
+    if C != 64 * H or N != Hg * Wg:
+        raise ValueError("x must be [B, Hg*Wg, 64*H]")
+    _check_proj(x, w, bias, H, 3 * C)
+    q, k, v = out if out is not None else (torch.empty((B, H, N, 64), dtype=x.dtype, device=x.device) for _ in range(3))
+    _check_tensors(q, k, v)
+    if tuple(q.shape) != (B, H, N, 64) or q.dtype != x.dtype:
+        raise ValueError("q, k, v must be [B, H, N, 64] bf16")
+    shape = JvShape(B, H, Hg, Wg, 64, JV_BF16)
+    with torch.cuda.device(x.device):
+        st = lib().jv_qkv_proj(x.data_ptr(), w.data_ptr(), None if bias is None else bias.data_ptr(), q.data_ptr(),
+                               k.data_ptr(), v.data_ptr(), ctypes.byref(shape), _stream(stream))
+    _raise(st, "jv_qkv_proj")
+    return q, k, v
+
+
+def out_proj(o, w, bias, Hg: int, Wg: int, out=None, stream=None) -> torch.Tensor:
+    """jv_out_proj: o [B, H, N, 64] bf16 (a mixer's output), w [C, C] bf16, bias fp32 [C] or None
+    -> y [B, N, C]."""
+    B, H, N, D = o.shape
+    if D != 64 or N != Hg * Wg:
+        raise ValueError("o must be [B, H, Hg*Wg, 64]")
+    C = 64 * H
+    _check_proj(o, w, bias, H, C)
+    y = torch.empty((B, N, C), dtype=o.dtype, device=o.device) if out is None else out
+    if not (y.is_cuda and y.is_contiguous() and tuple(y.shape) == (B, N, C) and y.dtype == o.dtype):
+        raise ValueError("y must be a contiguous [B, N, C] bf16 CUDA tensor")
+    shape = JvShape(B, H, Hg, Wg, 64, JV_BF16)
+    with torch.cuda.device(o.device):
+        st = lib().jv_out_proj(o.data_ptr(), w.data_ptr(), None if bias is None else bias.data_ptr(), y.data_ptr(),
+                               ctypes.byref(shape), _stream(stream))
+    _raise(st, "jv_out_proj")
+    return y
 
 
 def device_status(stream=None) -> int:
