@@ -368,6 +368,19 @@ def run_cuda(args):
     add("F", lambda i: jv.full_attn(dq[r(i)], dk[r(i)], dv[r(i)], out=outs[r(i)]),
         alg_bytes(*w.shape), f_flops, "tensor")
 
+    # the projections either side of a mixer (outside the step: the metric counts mixers only)
+    Cm = w.H * w.D
+    px = inputs.normal((w.B, w.N, Cm), inputs.seed_for(w.cfg, 0, 5), "bf16").to(dev)
+    pw, pb = (t.to(dev) for t in inputs.proj_weights(3 * Cm, Cm, inputs.seed_for(w.cfg, 0, 6)))
+    pwo, pbo = (t.to(dev) for t in inputs.proj_weights(Cm, Cm, inputs.seed_for(w.cfg, 0, 7)))
+    py = torch.empty_like(px)
+    tok = w.B * w.N
+    add("qkv_proj", lambda i: jv.qkv_proj(px, pw, pb, w.H, w.Hg, w.Wg, out=tuple(outs)),
+        2 * (tok * Cm + 3 * Cm * Cm + 3 * tok * Cm), 2.0 * tok * 3 * Cm * Cm, "tensor")
+    add("out_proj", lambda i: jv.out_proj(outs[r(i)], pwo, pbo, w.Hg, w.Wg, out=py),
+        2 * (2 * tok * Cm + Cm * Cm), 2.0 * tok * Cm * Cm, "tensor")
+    del px, py
+
     # ragged DepthAnythingV2-L grid (73x73, B=4): F and W with masked edge windows
     w4 = inputs.WORKLOADS["dav2_l"]
     q4 = [[t.to(dev) for t in inputs.qkv(w4, layer=l)] for l in range(3)]
@@ -456,6 +469,23 @@ def run_single(args):
     outs = [torch.empty_like(s[0]) for s in sets]
     C = w.H * w.D
     dwc = None
+    if args.single in ("qkv_proj", "out_proj"):
+        x = inputs.normal((w.B, w.N, C), inputs.seed_for(w.cfg, 0, 5), "bf16").to(dev)
+        rows = 3 * C if args.single == "qkv_proj" else C
+        pw, pb = (t.to(dev) for t in inputs.proj_weights(rows, C, inputs.seed_for(w.cfg, 0, 6)))
+        y = torch.empty_like(x)
+
+        def pfn(i):
+            q, k, v = sets[i % 3]
+            if args.single == "qkv_proj":
+                jv.qkv_proj(x, pw, pb, w.H, w.Hg, w.Wg, out=(q, k, v))
+            else:
+                jv.out_proj(q, pw, pb, w.Hg, w.Wg, out=y)
+        ms = time_calls(pfn, args.steps, args.warmup, stream)
+        assert jv.device_status() == jv.JV_OK
+        print(json.dumps({"single": args.single, "workload": args.workload, "ms": ms,
+                          "TFLOPs": 2.0 * w.tokens * rows * C / ms / 1e9}))
+        return
     if args.single == "L+dwc":
         d = inputs.dwc_weights(C, C // 8, 3, inputs.seed_for(w.cfg, 0, 3))
         dwc = {k: (v.to(dev) if hasattr(v, "to") else v) for k, v in d.items()}
@@ -483,7 +513,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--single", choices=["L", "L+dwc", "W", "F"], default=None,
+    ap.add_argument("--single", choices=["L", "L+dwc", "W", "F", "qkv_proj", "out_proj"], default=None,
                     help="time one mixer alone (used for profiler captures)")
     ap.add_argument("--workload", default="dinov3_l", choices=sorted(inputs.WORKLOADS))
     args = ap.parse_args()

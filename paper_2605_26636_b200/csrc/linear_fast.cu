@@ -21,8 +21,9 @@
 // its first Q loads overlap the tail of the state kernel, and it waits for that grid
 // (griddepcontrol.wait) only before touching the partials.
 //
-// With the convolution on, two small kernels (the generator MLP) and a TMA-staged
-// depth-wise convolution pass over V and o follow.
+// With the convolution on, the generator's hidden layer (a tiny kernel) runs between the
+// state pass and the apply pass, its output layer beside the apply pass, and a TMA-staged
+// depth-wise convolution pass over V and o follows both.
 //
 // Partial layout per (batch, head, chunk), in floats:
 //   [0, 4096) KV[a][e], [4096, 4160) z[a], [4160, 4224) vsum[e]
@@ -363,10 +364,11 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
 
-  // A grid launched behind this one with programmatic serialisation (the convolution's generator)
-  // may start once every thread here has passed this point; the rectifier warps pass it only
-  // after the state pass is complete, which is all the generator depends on.
-  if (warp >= 4) griddep_launch_dependents();
+  // A grid launched behind this one with programmatic serialisation (the output layer of the
+  // convolution's generator) may start once this grid lets its dependents go.  It reads what the
+  // grids before this one wrote, so no warp here does that before it knows that those grids are
+  // complete: the rectifier warps after their griddepcontrol.wait, the other warps after the first
+  // barrier that the rectifier warps have arrived on.
 
   if (warp == 4) {
     // ================= TMA producer and MMA issuer (one elected lane) =================
@@ -396,6 +398,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       }
       const int s = it % kApplyStages, b = it & 1;
       ok = warp_wait(&bars->relu_done[s], (it / kApplyStages) & 1, &bars->abort_flag, status);
+      if (it == 0) griddep_launch_dependents();
       if (ok && it >= 2) ok = warp_wait(&bars->d_empty[b], ((it >> 1) - 1) & 1, &bars->abort_flag, status);
       if (!ok) break;
       tc_fence_after();
@@ -422,7 +425,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     }
   } else if (warp < 4) {
     // ================= rectifier warps: thread r = 32 warp + lane owns token row r of every tile =================
-    griddep_wait();                                    // the state pass (and anything before it) has completed
+    griddep_wait();                                    // the grids before this one (state pass, generator's hidden layer) are complete
     griddep_launch_dependents();
     bool ok = *reinterpret_cast<volatile int*>(status) == 0;
     {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
@@ -522,6 +525,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       // The tile's MMAs were issued after all 128 rectifier threads had published its rows and
       // denominators, so the accumulator being complete means the denominators are in place.
       ok = warp_wait(&bars->d_full[b], (it >> 1) & 1, &bars->abort_flag, status);
+      if (it == 0) griddep_launch_dependents();
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / (den_sm[(it & (kDenRing - 1)) * kApplyTok + row] + eps);
@@ -787,7 +791,8 @@ __global__ void __launch_bounds__(128)
 gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W1, const float* __restrict__ b1,
                   float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n) {
   __shared__ float red[4];
-  griddep_launch_dependents();
+  griddep_wait();                                      // the state pass is complete
+  griddep_launch_dependents();                         // the apply grid may set up and load Q meanwhile
   const int r = blockIdx.x, b = blockIdx.y, C = H * kD;
   float s = 0.f;
   for (int c = threadIdx.x; c < C; c += 128) {
@@ -811,7 +816,8 @@ gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W
 __global__ void __launch_bounds__(256)
 gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, const float* __restrict__ b2,
                float* __restrict__ w, int B, int T, int R) {
-  griddep_wait();                                      // the hidden layer (launched just before) is complete
+  // Launched behind the apply grid, which lets its dependents go only after it has seen the hidden
+  // layer's grid complete: hidden is final here and this grid runs beside the apply pass.
   const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
   const bool t_ok = t < T;
   const float* wrow = W2 + (size_t)(t_ok ? t : 0) * R;
@@ -847,6 +853,9 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
       if (t_ok && part == 0 && b0 + bb < B) w[(size_t)(b0 + bb) * T + t] = sres + (b2 ? b2[t] : 0.f);
     }
   }
+  // The convolution pass is launched behind this grid in plain stream order and adds into what the
+  // apply pass writes: this grid must not retire before the apply grid has.
+  griddep_wait();
 }
 
 // ---- host side ---------------------------------------------------------------------------
@@ -927,8 +936,33 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+
+  // With the convolution on, the generator's hidden layer (tiny; it needs the state pass only) goes
+  // between the state pass and the apply pass, and its output layer behind the apply pass, beside
+  // which it runs.  Every launch from here to the output layer uses programmatic serialisation;
+  // each grid waits for its predecessor (griddepcontrol.wait) before it reads what that one wrote,
+  // the output layer at its very end, so that stream order still means "apply pass complete" for
+  // the convolution pass that follows it.
+  float* hidden = (float*)(ws + p.off_hidden);
+  if (a.dwc && a.dwc->R > 0) {      // R == 0: static kernels, the output layer just broadcasts b2
+    const jv_dwc& d = *a.dwc;
+    cudaLaunchConfig_t hcfg = {};
+    hcfg.stream = st;
+    hcfg.attrs = attr;
+    hcfg.numAttrs = 1;
+    hcfg.gridDim = dim3(d.R, s.B);
+    hcfg.blockDim = dim3(128);
+    e = cudaLaunchKernelEx(&hcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
+                           p.nchunk, p.state_elems, 1.f / (float)N);
+    count_launch();
+    if (e != cudaSuccess) return e;
+  }
+
   // apply pass: one wave of two CTAs per SM, spans of whole 128-token tiles; launched so that its
-  // set-up overlaps the tail of the state pass
+  // set-up overlaps the tail of the grid before it
   int nspan = (2 * 148) / BH;
   if (nspan < 1) nspan = 1;
   int span = ceil_div(ceil_div(N, nspan), kApplyTok) * kApplyTok;
@@ -939,9 +973,6 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   cfg.blockDim = dim3(kApplyThreads);
   cfg.dynamicSmemBytes = kApplySmem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, lin_apply_kernel, mq, mo, (const float*)partial, status, N, span, p.nchunk,
@@ -953,25 +984,12 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     const __nv_bfloat16* v = (const __nv_bfloat16*)a.v;
     __nv_bfloat16* o = (__nv_bfloat16*)a.o;
     const jv_dwc& d = *a.dwc;
-    float* hidden = (float*)(ws + p.off_hidden);
     float* wk = (float*)(ws + p.off_kernel);
-    // Both generator kernels run beside the apply pass: they are launched with programmatic
-    // serialisation, the first one does not wait for the apply grid (it needs the state pass only,
-    // which the apply grid has waited for before it lets its dependents start), the second one
-    // waits for the first.
     const int T = s.H * kD * d.k * d.k;
     cudaLaunchConfig_t gcfg = {};
     gcfg.stream = st;
     gcfg.attrs = attr;
     gcfg.numAttrs = 1;
-    if (d.R > 0) {           // R == 0: static kernels, the output layer below just broadcasts b2
-      gcfg.gridDim = dim3(d.R, s.B);
-      gcfg.blockDim = dim3(128);
-      e = cudaLaunchKernelEx(&gcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
-                             p.nchunk, p.state_elems, 1.f / (float)N);
-      count_launch();
-      if (e != cudaSuccess) return e;
-    }
     gcfg.gridDim = dim3(ceil_div(T, 32));
     gcfg.blockDim = dim3(256);
     e = cudaLaunchKernelEx(&gcfg, gen_out_kernel, (const float*)hidden, d.W2, d.b2, wk, (int)s.B, T, (int)d.R);
