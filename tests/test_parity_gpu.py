@@ -125,6 +125,49 @@ def test_linear_with_static_dwc(jv, oracle, both_paths, dtype, ksz):
     assert rel_err(out, oracle.linear_attn(q, k, v, Hg, Wg, dwc=d)) <= TOL[dtype]
 
 
+@pytest.mark.parametrize("case", [(2, 4, 48, 40), (1, 2, 16, 16), (1, 16, 24, 24), (4, 8, 32, 32)],
+                         ids=lambda c: "x".join(map(str, c)))
+def test_linear_dwc_with_poisoned_scratch_and_output(jv, oracle, case):
+    """The convolution chain is several kernels that overlap through programmatic launches; a kernel that
+    starts before the one it depends on has finished reads whatever the buffers held.  Scratch and output
+    start as NaN here and the call is repeated, so an ordering mistake cannot pass on stale data."""
+    B, H, Hg, Wg = case
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, 64, "bf16", seed=60 + B + H)
+    d = inputs.dwc_weights(H * 64, 32, 3, 321)
+    ref = oracle.linear_attn(q, k, v, Hg, Wg, dwc=d)
+    dq, dk, dv = _dev((q, k, v))
+    dd = dwc_to_device(d, DEV)
+    shape = jv.make_shape(dq, Hg, Wg)
+    ws = jv.alloc_workspace("L", shape, jv.make_dwc(dd, DEV), DEV)
+    out = torch.empty_like(dq)
+    for rep in range(4):
+        ws.fill_(0xFF)                       # every fp32 word a NaN
+        out.fill_(float("nan"))
+        jv.linear_attn(dq, dk, dv, Hg, Wg, dwc=dd, out=out, ws=ws)
+        torch.cuda.synchronize()
+        assert rel_err(out, ref) <= TOL["bf16"], rep
+
+
+# ------------------------------------------------------------------ other model sizes and grids
+@pytest.mark.parametrize("case", [(1, 12, 64, 128, 64), (1, 24, 32, 64, 64), (1, 4, 24, 40, 128)],
+                         ids=["vitb_64x128", "giant_32x64", "d128_24x40"])
+def test_other_model_shapes(jv, oracle, case):
+    """Non-square grids (a 1024x2048 image at patch 16 is 64x128 tokens) with 12 and 24 heads on the
+    tensor-core kernels, and head_dim 128 on the shape-generic kernels; sampled (batch, head) pairs."""
+    B, H, Hg, Wg, D = case
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, D, "bf16", seed=H + D)
+    dq, dk, dv = _dev((q, k, v))
+    d = inputs.dwc_weights(H * D, 32, 3, 11)
+    ol = jv.linear_attn(dq, dk, dv, Hg, Wg, dwc=dwc_to_device(d, DEV)).cpu()
+    ow = jv.window_attn(dq, dk, dv, Hg, Wg, 16, 16).cpu()
+    of = jv.full_attn(dq, dk, dv, Hg, Wg).cpu()
+    assert rel_err(ol, oracle.linear_attn(q, k, v, Hg, Wg, dwc=d)) <= TOL["bf16"]
+    for b, h in sample_heads(B, H, 3, H):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        assert rel_err(ow[sl], oracle.window_attn(q[sl], k[sl], v[sl], Hg, Wg, 16, 16)) <= TOL["bf16"], ("W", b, h)
+        assert rel_err(of[sl], oracle.full_attn(q[sl], k[sl], v[sl])) <= TOL["bf16"], ("F", b, h)
+
+
 def test_explicit_scale_and_eps(jv, oracle, both_paths):
     q, k, v = inputs.custom_qkv(1, 2, 16 * 16, 64, "bf16", seed=8)
     dq, dk, dv = _dev((q, k, v))
