@@ -2,6 +2,8 @@
 // Every argument error is reported before anything is launched.
 #include <atomic>
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -81,7 +83,11 @@ jv_status check_proj(const jv_shape* s, const void* const* ptrs, int nptr, int n
   return JV_OK;
 }
 
-jv_status from_cuda(cudaError_t e) { return e == cudaSuccess ? JV_OK : JV_ERR_CUDA; }
+jv_status from_cuda(cudaError_t e) {
+  if (e == cudaSuccess) return JV_OK;
+  if (getenv("JETVIT_DEBUG")) fprintf(stderr, "libjetvit: CUDA error %d (%s)\n", (int)e, cudaGetErrorString(e));
+  return JV_ERR_CUDA;
+}
 
 float pick_scale(float scale, int D) { return scale > 0.f ? scale : 1.f / sqrtf((float)D); }
 
@@ -89,6 +95,12 @@ float pick_scale(float scale, int D) { return scale > 0.f ? scale : 1.f / sqrtf(
 jv_status run_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* s, int wh, int ww,
                    float scale, bool full, cudaStream_t st) {
   AttnArgs a{q, k, v, o, s->B * s->H, s->Hg, s->Wg, s->D, wh, ww, pick_scale(scale, s->D), s->dtype};
+  const bool one_window = full || (wh >= s->Hg && ww >= s->Wg);
+  if (!g_force_generic.load() && one_window && attn_f4_supported(a)) {
+    int* status = device_status_ptr();
+    if (!status) return JV_ERR_CUDA;
+    return from_cuda(launch_attn_f4(a, status, st));
+  }
   if (!g_force_generic.load() && attn_tc_supported(a, full)) {
     int* status = device_status_ptr();
     if (!status) return JV_ERR_CUDA;

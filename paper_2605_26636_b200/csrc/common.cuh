@@ -64,6 +64,9 @@ cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st);
 // (wh, ww) windows, ww a power of two dividing 128, wh*ww a multiple of 128 and <= 256...
 bool attn_tc_supported(const AttnArgs& a, bool full);
 cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream_t st);
+// tcgen05 path for full attention over long sequences (bf16, D == 64, N >= 1024): four query tiles per CTA
+bool attn_f4_supported(const AttnArgs& a);
+cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st);
 
 struct LinArgs {
   const void *q, *k, *v;
