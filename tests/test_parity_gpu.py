@@ -168,6 +168,32 @@ def test_other_model_shapes(jv, oracle, case):
         assert rel_err(of[sl], oracle.full_attn(q[sl], k[sl], v[sl])) <= TOL["bf16"], ("F", b, h)
 
 
+@pytest.mark.parametrize("case", [(1, 3, 32, 32), (1, 2, 37, 29), (2, 1, 35, 40), (1, 1, 31, 33)],
+                         ids=lambda c: "x".join(map(str, c)))
+def test_full_attention_long_sequences(jv, oracle, case):
+    """N >= 1024 runs on the kernel with four query tiles per CTA: tile counts of 8, 9, 11 (the last item
+    of a head holds one or three tiles) with ragged last key tiles, and 1023 tokens just below the switch."""
+    B, H, Hg, Wg = case
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, 64, "bf16", seed=Hg + Wg)
+    out, check = guarded_empty(q.shape, torch.bfloat16, DEV)
+    jv.full_attn(*_dev((q, k, v)), Hg, Wg, out=out)
+    check()
+    assert rel_err(out, oracle.full_attn(q, k, v)) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("n_tokens", [512, 2048])
+def test_full_attention_with_a_rising_reference(jv, oracle, n_tokens):
+    """Scores that grow along the sequence make the running softmax reference move again and again
+    (accumulator rescaled many times); a sharp step in the middle makes it jump by far more than 2^8."""
+    q, k, v = inputs.custom_qkv(1, 2, n_tokens, 64, "bf16", seed=n_tokens)
+    ramp = torch.linspace(0.0, 1.0, n_tokens).view(1, 1, n_tokens, 1)
+    u = q[:, :, :1, :].float()                      # keys lean more and more towards the first query
+    k2 = (k.float() + 6.0 * ramp * u).to(torch.bfloat16)
+    k2[:, :, n_tokens // 2] = (40.0 * u[:, :, 0]).to(torch.bfloat16)
+    out = jv.full_attn(*_dev((q, k2, v)))
+    assert rel_err(out, oracle.full_attn(q, k2, v)) <= TOL["bf16"]
+
+
 def test_explicit_scale_and_eps(jv, oracle, both_paths):
     q, k, v = inputs.custom_qkv(1, 2, 16 * 16, 64, "bf16", seed=8)
     dq, dk, dv = _dev((q, k, v))
