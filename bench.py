@@ -40,9 +40,9 @@ METRIC = "mixer tokens/sec (L+W+F stack at ViT-L shapes)"
 UNIT = "tokens/s"
 STEP_SCHEDULE = "LWF"
 WIN = 16
-# DRAM bytes of one attn_tc_kernel launch running F at the DINOv3-L shape, from the ncu capture
+# DRAM bytes of one attn_f4_kernel launch (F at the DINOv3-L shape), from the ncu capture
 # summarised in profiles/ (None when the kernel has changed since the capture)
-ATTN_F_DRAM_BYTES = 247_510_000
+ATTN_F_DRAM_BYTES = 247_130_000
 
 
 def load_peaks():
@@ -421,7 +421,7 @@ def run_cuda(args):
     # the timed region (events around the F layer of every step)
     f_ms = layer_ms[STEP_SCHEDULE.index("F")]
     f_tf = f_flops / f_ms / 1e9
-    roofline = {"kernel": "attn_tc_kernel as jv_full_attn (one launch per step)", "bound": "tensor", "achieved": f_tf,
+    roofline = {"kernel": "attn_f4_kernel as jv_full_attn (one launch per step)", "bound": "tensor", "achieved": f_tf,
                 "peak": tf, "unit": "TFLOP/s", "frac": f_tf / tf, "traffic": ATTN_F_DRAM_BYTES,
                 "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
                 "peak_source": peaks["source"] + " bf16 burst", "ms_per_launch": f_ms,

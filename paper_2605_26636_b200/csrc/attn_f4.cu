@@ -63,7 +63,8 @@ struct F4Params {
   int N;                 // tokens per (batch, head)
   int ntiles;            // key (and query) tiles per head: ceil(N / 128)
   int qgroups;           // groups of four query tiles per head
-  int total_items;       // (batch*head, group), group fastest
+  int n_full;            // items [0, n_full) are whole groups, (batch*head, group) with the group fastest;
+  int total_items;       // items [n_full, total_items) are half groups (two query tiles), see launch_attn_f4
   FastDiv div_qgroups;
   float scale_log2;      // softmax scale * log2(e)
 };
@@ -318,20 +319,38 @@ constexpr uint32_t kIdescQK = idesc(kTile, kSub, 0);
 constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
 
 struct Item {
-  int bh, qt0;      // (batch, head) and the first of the item's four query tiles
+  int bh, qt0, nt;  // (batch, head), the first of the item's query tiles, and how many it has (4 or 2)
 };
+// kHalves: the launch has half groups (n_full < total_items); without them the decode is one division.
+template <bool kHalves>
 __device__ __forceinline__ Item decode_item(const F4Params& p, int i) {
   Item it;
-  it.bh = fdiv(i, p.div_qgroups);
-  it.qt0 = kQT * (i - it.bh * p.qgroups);
+  if (kHalves) {
+    const int half = i - p.n_full;                 // >= 0: a half group
+    const int g = half < 0 ? i : p.n_full + (half >> 1);
+    it.bh = fdiv(g, p.div_qgroups);
+    it.qt0 = kQT * (g - it.bh * p.qgroups) + (half < 0 ? 0 : 2 * (half & 1));
+    it.nt = half < 0 ? kQT : 2;
+  } else {
+    it.bh = fdiv(i, p.div_qgroups);
+    it.qt0 = kQT * (i - it.bh * p.qgroups);
+    it.nt = kQT;
+  }
   return it;
+}
+// query tile t of the item exists: inside the item and inside the head
+template <bool kHalves>
+__device__ __forceinline__ bool tile_exists(const Item& it, int t, int ntiles) {
+  return (!kHalves || t < it.nt) && it.qt0 + t < ntiles;
 }
 
 // ---- the kernel ------------------------------------------------------------------
 // CTA c works on items c, c + gridDim.x, ...  Every role walks the same item sequence on its own;
 // ring stages and barrier parities follow running counters.  A query tile past the last one of
-// the head (the last item of a head whose tile count is not a multiple of four) is skipped by its
-// softmax warps; its issuer still takes part in the ring protocol so that arrival counts hold.
+// the head (the last item of a head whose tile count is not a multiple of four), or past the item's
+// own two tiles (a half group), is skipped by its softmax warps; its issuer still takes part in the
+// ring protocol so that arrival counts hold.  A half group without any tile is skipped by every role.
+template <bool kHalves>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
@@ -390,12 +409,13 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     int s = 0;                 // ring stage of the next key tile
     uint32_t par = 1;          // parity of the "empty" phase this pass over the ring waits for
     int issued_v = 0;          // for the abort path: V copies issued so far
-    for (int i = item0; i < p.total_items && ok; i += item_step, ++n) {
-      const Item it = decode_item(p, i);
+    for (int i = item0; i < p.total_items && ok; i += item_step) {
+      const Item it = decode_item<kHalves>(p, i);
+      if (kHalves && !tile_exists<kHalves>(it, 0, ntiles)) continue;
       for (int t = 0; t < kQT && ok; ++t) {
         ok = warp_wait(&bar->q_empty[t], (n & 1) ^ 1, bar, p.status);
         if (!ok) break;
-        if (it.qt0 + t < ntiles && elect_one()) {
+        if (tile_exists<kHalves>(it, t, ntiles) && elect_one()) {
           mbar_expect_tx(&bar->q_full[t], kTileBytes);
           tma_load_3d(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], 0, (it.qt0 + t) * kTile, it.bh);
         }
@@ -419,6 +439,7 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         ++issued_v;
         if (++s == kStages) { s = 0; par ^= 1; }
       }
+      ++n;
     }
     if (!ok && lane == 0) {
       // let the copies still in flight land before the CTA leaves (bounded by the same limit)
@@ -441,8 +462,9 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     uint32_t pcnt[2] = {0, 0};              // steps published so far per tile: parity of p_full
     uint32_t qcnt[2] = {0, 0};              // items in which the tile existed: parity of q_full
     for (int i = item0; i < p.total_items && ok; i += item_step) {
-      const Item it = decode_item(p, i);
-      const bool ex[2] = {it.qt0 + tb < ntiles, it.qt0 + tb + 1 < ntiles};
+      const Item it = decode_item<kHalves>(p, i);
+      if (kHalves && !tile_exists<kHalves>(it, 0, ntiles)) continue;
+      const bool ex[2] = {tile_exists<kHalves>(it, tb, ntiles), tile_exists<kHalves>(it, tb + 1, ntiles)};
       for (int u = 0; u <= nsteps && ok; ++u) {
         const bool has_qk = u < nsteps, has_pv = u > 0;
         if (has_qk && (u & 1) == 0) {       // first half of a key tile: its K must have landed
@@ -525,8 +547,8 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     uint32_t ocnt = 0;                // items seen by this tile: parity of o_full
 
     for (int i = item0; i < p.total_items && ok; i += item_step) {
-      const Item it = decode_item(p, i);
-      if (it.qt0 + t >= ntiles) continue;          // this query tile does not exist
+      const Item it = decode_item<kHalves>(p, i);
+      if (!tile_exists<kHalves>(it, t, ntiles)) continue;   // this query tile does not exist
       float m = -INFINITY, l = 0.f;
       for (int u = 0; u < nsteps; ++u) {
         ok = warp_wait(&bar->s_full[t], scnt & 1, bar, p.status);
@@ -707,18 +729,12 @@ cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st) {
   }
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attn_f4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(attn_f4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attn_f4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  F4Params p;
-  p.status = status;
-  p.N = N;
-  p.ntiles = ceil_div(N, kTile);
-  p.qgroups = ceil_div(p.ntiles, kQT);
-  p.total_items = p.qgroups * a.BH;
-  p.div_qgroups = make_fastdiv((uint32_t)p.qgroups);
-  p.scale_log2 = a.scale * 1.4426950408889634f;
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
@@ -729,8 +745,24 @@ cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st) {
       return cudaErrorUnknown;
     }
   }
+  F4Params p;
+  p.status = status;
+  p.N = N;
+  p.ntiles = ceil_div(N, kTile);
+  p.qgroups = ceil_div(p.ntiles, kQT);
+  // Items are dealt out round-robin, so the last round is as long as a full one however few CTAs it
+  // keeps busy.  When it would keep at most half of them busy, its groups are split into half groups
+  // of two query tiles (a serial per-tile chain makes those finish in a little over half the time).
+  const int groups = p.qgroups * a.BH;
+  const int rem = groups % num_sms;
+  const int split = (rem > 0 && rem <= num_sms / 2) ? rem : 0;
+  p.n_full = groups - split;
+  p.total_items = groups + split;
+  p.div_qgroups = make_fastdiv((uint32_t)p.qgroups);
+  p.scale_log2 = a.scale * 1.4426950408889634f;
   const int grid = p.total_items < num_sms ? p.total_items : num_sms;
-  attn_f4_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  if (split) attn_f4_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  else attn_f4_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   count_launch();
   return cudaGetLastError();
 }
