@@ -27,14 +27,14 @@
 // Every mbarrier wait is bounded: a wait that runs out sets the device status word,
 // raises a CTA-wide abort flag, and every role falls through to the common teardown
 // (tensor memory is always released).
-#include <cuda.h>
-
 #include <type_traits>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace jv {
 namespace {
+
+using namespace tc;
 
 constexpr int kD = 64;
 constexpr int kTile = 128;                 // tokens per tile (MMA M and key-tile N)
@@ -43,21 +43,9 @@ constexpr int kStages = 4;                 // K and V ring depth
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSub = 64;                    // keys per softmax / MMA step: half a key tile
+constexpr int kPolyOf8 = 2;                 // of every 8 score pairs, this many take the polynomial exponential
 // Tensor-memory columns: S(t, b) at kColS + (2 t + b) * 64, O(t) at kColO + 64 t, P(t, b) at kColP + (2 t + b) * 32
 constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
-
-// Division by a run-time constant without a divide: q = (umulhi(n, mul) + n) >> shr, exact for
-// 0 <= n < 2^31 (mul = floor(2^32 (2^shr - d) / d) + 1, shr = ceil(log2 d)).
-struct FastDiv {
-  uint32_t mul, shr, d;
-};
-inline FastDiv make_fastdiv(uint32_t d) {
-  uint32_t l = 0;
-  while ((1ull << l) < d) ++l;
-  return FastDiv{(uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1), l, d};
-}
-__device__ __forceinline__ int fdiv(int n, const FastDiv& f) { return (int)((__umulhi((uint32_t)n, f.mul) + (uint32_t)n) >> f.shr); }
 
 struct TcParams {
   __nv_bfloat16* o;
@@ -109,253 +97,6 @@ struct __align__(8) Barriers {
 constexpr size_t kSmemTiles = (6 + 2 * kStages) * (size_t)kTileBytes;          // Q[2][2] K[kStages] V[kStages] O[2]
 constexpr size_t kSmemBytes = kSmemTiles + sizeof(Barriers) + 1024;            // + alignment slack
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Non-blocking test of a phase: used to take a barrier's round trip off the critical path
-// (test early, consume the answer later, fall back to mbar_wait if it was not yet complete).
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false (after flagging the status word and the CTA abort flag)
-// if the phase did not complete in time or another role already aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* b, int* status) {
-  if (mbar_try(bar, parity)) return true;
-  unsigned long long t0 = 0;
-  for (uint32_t spin = 0;; ++spin) {
-    if (mbar_try(bar, parity)) return true;
-    if ((spin & 63u) == 63u) {
-      if (b->abort_flag) return false;
-      const unsigned long long now = globaltimer();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
-        b->abort_flag = 1;
-        atomicOr(status, kStatusTimeout);
-        return false;
-      }
-    }
-  }
-}
-
-// The same for a whole converged warp, with a warp-uniform outcome.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Barriers* b, int* status) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, b, status));
-}
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
-                                            int c2, int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-
-// ---- tcgen05 wrappers -------------------------------------------------------------
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// One lane of a converged warp (the same one every time for a full warp).
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
-  return pred != 0;
-}
-// The tcgen05 issue wrappers below are called by a whole converged warp; one elected lane issues.
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  if (elect_one())
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  if (elect_one())
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  if (elect_one())
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// Waits for this thread's outstanding tensor-memory loads.  The registers of the load are
-// threaded through the statement so that no use of them can be scheduled ahead of the wait.
-__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :: "memory");
-}
-
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-// Two fp32 values in one 64-bit register: the packed fp32x2 arithmetic of sm_100.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-
-// ---- softmax building blocks: 32 scores of one query row at a time -------------------
-constexpr uint32_t kNegInf = 0xff800000u;
-__device__ __forceinline__ void max32(const uint32_t (&v)[32], float (&mx)[4]) {
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      mx[u] = max3(mx[u], __uint_as_float(v[8 * i + 2 * u]), __uint_as_float(v[8 * i + 2 * u + 1]));
-}
-// exp2 on the FMA pipe, for part of the scores (the MUFU unit, 16 results per clock and SM,
-// is the tightest resource of softmax attention at head_dim 64).  x = n + f with n = round(x),
-// f in [-0.5, 0.5]; 2^f by a degree-3 minimax polynomial (relative error 7.5e-5, well below
-// the bf16 rounding of P); n goes straight into the exponent field.  Valid for x in [-126, 126].
-constexpr float kPolyC0 = 0.9999280571937561f, kPolyC1 = 0.6932609677314758f;
-constexpr float kPolyC2 = 0.2426111251115799f, kPolyC3 = 0.0551716685295105f;
-constexpr float kRoundMagic = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-__device__ __forceinline__ void exp2_poly2(uint64_t x, float& p0, float& p1) {
-  float x0, x1;
-  unpack2(x, x0, x1);
-  x = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-  const uint64_t t = add2(x, pack2(kRoundMagic, kRoundMagic));
-  const uint64_t n = add2(t, pack2(-kRoundMagic, -kRoundMagic));
-  const uint64_t f = fma2(n, pack2(-1.f, -1.f), x);
-  uint64_t q = fma2(f, pack2(kPolyC3, kPolyC3), pack2(kPolyC2, kPolyC2));
-  q = fma2(q, f, pack2(kPolyC1, kPolyC1));
-  q = fma2(q, f, pack2(kPolyC0, kPolyC0));
-  float q0, q1, t0, t1;
-  unpack2(q, q0, q1);
-  unpack2(t, t0, t1);
-  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
-  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
-}
-
-#ifndef JV_POLY_PAIRS_OF_8
-#define JV_POLY_PAIRS_OF_8 2   // of every 8 score pairs, this many take the polynomial path
-#endif
-// p = exp2(s * sl2 + mneg) for 32 scores; adds them into four packed partial sums and packs
-// them to bf16 pairs (even key in the low half).  kTrack also folds the scores into mx.
-template <bool kTrack>
-__device__ __forceinline__ void exp32(const uint32_t (&v)[32], uint64_t sl2x2, uint64_t mnegx2, uint64_t (&lsum)[4],
-                                      uint32_t (&pk)[16], float (&mx)[4]) {
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const float s0 = __uint_as_float(v[2 * i]), s1 = __uint_as_float(v[2 * i + 1]);
-    if (kTrack) mx[i & 3] = max3(mx[i & 3], s0, s1);
-    const uint64_t x = fma2(pack2(s0, s1), sl2x2, mnegx2);
-    float p0, p1;
-    if ((i & 7) < JV_POLY_PAIRS_OF_8) {
-      exp2_poly2(x, p0, p1);
-    } else {
-      float x0, x1;
-      unpack2(x, x0, x1);
-      p0 = ex2(x0);
-      p1 = ex2(x1);
-    }
-    lsum[i & 3] = add2(lsum[i & 3], pack2(p0, p1));
-    pk[i] = pack_bf16(p0, p1);
-  }
-}
-
-// Shared-memory matrix descriptors (128-byte swizzle; 8-row groups 1024 bytes apart).
-//   K-major operand  ([rows][64 bf16], used for Q and K): advance 32 bytes per K step of 16.
-//   MN-major operand ([keys][64 bf16] used as B = V):      advance 2048 bytes per K step of 16 keys.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) /* LBO (unused) */ | (64ull << 32) /* SBO = 1024 B */ |
-         (1ull << 46) /* descriptor version */ | (2ull << 61) /* SWIZZLE_128B */;
-}
-// Instruction descriptor, kind::f16: D fp32, A and B bf16.
-constexpr uint32_t idesc(uint32_t M, uint32_t N, uint32_t b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
-}
 constexpr uint32_t kIdescQK = idesc(kTile, kSub, 0);
 constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
 
@@ -438,7 +179,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const Item it = decode_item(p, i);
       if (it.qt0 >= it.ntiles) continue;
       const int qb = n & 1;
-      ok = warp_wait(&bar->q_empty[qb], ((n >> 1) & 1) ^ 1, bar, p.status);
+      ok = warp_wait(&bar->q_empty[qb], ((n >> 1) & 1) ^ 1, &bar->abort_flag, p.status);
       if (!ok) break;
       if (elect_one()) {
         mbar_expect_tx(&bar->q_full[qb], 2 * kTileBytes);
@@ -448,14 +189,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       __syncwarp();
       for (int j = 0; j < it.ntiles; ++j) {
-        ok = warp_wait(&bar->k_empty[s], par, bar, p.status);
+        ok = warp_wait(&bar->k_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s], kTileBytes);
           tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
         }
         __syncwarp();
-        ok = warp_wait(&bar->v_empty[s], par, bar, p.status);
+        ok = warp_wait(&bar->v_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s], kTileBytes);
@@ -507,8 +248,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     auto issue_qk = [&](int h, int jq, int ntiles_q, int n_q) -> bool {
       const int qb = n_q & 1;
       if (h == 0) {
-        if (jq == 0 && !warp_wait(&bar->q_full[qb], (n_q >> 1) & 1, bar, p.status)) return false;
-        if (!warp_wait(&bar->k_full[s1], ph1, bar, p.status)) return false;
+        if (jq == 0 && !warp_wait(&bar->q_full[qb], (n_q >> 1) & 1, &bar->abort_flag, p.status)) return false;
+        if (!warp_wait(&bar->k_full[s1], ph1, &bar->abort_flag, p.status)) return false;
         tc_fence_after();
       }
       const uint32_t kb = sK + s1 * kTileBytes + h * (kSub * kD * 2), qa = sQ + (2 * qb + t) * kTileBytes;
@@ -534,10 +275,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       Item itn{};
       if (nxt >= 0) itn = decode_item(p, nxt);
       for (int j = 0; j < it.ntiles && ok; ++j) {
-        ok = warp_wait(&bar->v_full[s], ph, bar, p.status);
+        ok = warp_wait(&bar->v_full[s], ph, &bar->abort_flag, p.status);
         const bool last = j + 1 == it.ntiles;
         for (int h = 0; h < 2 && ok; ++h) {
-          ok = warp_wait(&bar->p_full[t][h], g_par, bar, p.status);
+          ok = warp_wait(&bar->p_full[t][h], g_par, &bar->abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
@@ -607,9 +348,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const uint64_t mnegx2 = pack2(mneg, mneg);
       uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
       uint32_t pk[16];
-      exp32<false>(va, sl2x2, mnegx2, lsum, pk, mx4);
+      exp32<false, kPolyOf8>(va, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tPb, pk);
-      exp32<false>(vb, sl2x2, mnegx2, lsum, pk, mx4);
+      exp32<false, kPolyOf8>(vb, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tPb + 16, pk);
       float a0, a1, b0, b1;
       unpack2(add2(lsum[0], lsum[1]), a0, a1);
@@ -637,11 +378,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tmem_ld32(tSb, va);
       tmem_wait_ld(va);
       tmem_ld32(tSb + 32, vb);
-      exp32<true>(va, sl2x2, mnegx2, lsum, pk, mx4);
+      exp32<true, kPolyOf8>(va, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tPb, pk);
       next_ready = mbar_test(next_bar, next_parity);   // round trip hidden behind the second half
       tmem_wait_ld(vb);
-      exp32<true>(vb, sl2x2, mnegx2, lsum, pk, mx4);
+      exp32<true, kPolyOf8>(vb, sl2x2, mnegx2, lsum, pk, mx4);
       tmem_st16(tPb + 16, pk);
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       float a0, a1, b0, b1;
@@ -685,7 +426,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const uint32_t sOt = sO + t * kTileBytes;
     unsigned char* sOt_ptr = smem + (size_t)(4 + 2 * kStages + t) * kTileBytes;
     auto epi_load = [&](uint32_t (&ob)[32]) -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->o_full[t], done.par, bar, p.status))) return false;
+      if (!__all_sync(0xffffffffu, mbar_wait(&bar->o_full[t], done.par, &bar->abort_flag, p.status))) return false;
       tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
@@ -760,7 +501,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int j = u >> 1, h = u & 1;
         // warp-uniform outcome: the tensor-memory accesses below are warp-collective
         if (!__all_sync(0xffffffffu, next_ready)) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], g_par, bar, p.status));
+          ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], g_par, &bar->abort_flag, p.status));
           if (!ok) return false;
         }
         tc_fence_after();
@@ -819,9 +560,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           // tells us; after the last step of the run there are no further scores, and pv_done
           // (committed after each P V of the run's last key tile) does.
           if (has_next)
-            ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, bar, p.status));
+            ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, &bar->abort_flag, p.status));
           else
-            ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, bar, p.status));
+            ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, &bar->abort_flag, p.status));
           if (!ok) return false;
           tc_fence_after();
 #pragma unroll
@@ -892,23 +633,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 }
 
 // ---- host side ----------------------------------------------------------------------
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = (EncodeFn)ptr;
-  }
-  return fn;
-}
-
 struct Geometry {
   int gridW, gridH, win_w, win_h, box_w, box_h, step_x, step_y, nwx, nwy, tiles_per_window;
 };

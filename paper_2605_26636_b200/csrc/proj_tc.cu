@@ -20,12 +20,12 @@
 //
 // Every mbarrier wait is bounded; a wait that runs out sets the device status word and the
 // CTA's abort flag, and every role falls through to the teardown that frees tensor memory.
-#include <cuda.h>
-
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace jv {
 namespace {
+
+using namespace tc;
 
 constexpr int kD = 64;                       // head_dim = K block = feature block
 constexpr int kBM = 128;                     // tokens per tile
@@ -37,7 +37,6 @@ constexpr int kStages = 4;
 constexpr int kThreads = 256;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kStagingBytes = 32 * kD * 2;   // one warp's 32 tokens x 64 features
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct __align__(8) Barriers {
   uint64_t full[kStages], empty[kStages];
@@ -61,116 +60,8 @@ struct ProjParams {
   int N;                   // tokens per batch element
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* b, int* status) {
-  if (mbar_try(bar, parity)) return true;
-  unsigned long long t0 = 0;
-  for (uint32_t spin = 0;; ++spin) {
-    if (mbar_try(bar, parity)) return true;
-    if ((spin & 63u) == 63u) {
-      if (b->abort_flag) return false;
-      const unsigned long long now = globaltimer();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
-        b->abort_flag = 1;
-        atomicOr(status, kStatusTimeout);
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, Barriers* b, int* status) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, b, status));
-}
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
-  return pred != 0;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  if (elect_one())
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  if (elect_one())
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :: "memory");
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-// Shared-memory matrix descriptor of a K-major operand ([rows][64 bf16], 128-byte swizzle,
-// 8-row groups 1024 bytes apart); advance the address by 32 bytes per K step of 16.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major.
-constexpr uint32_t idesc(uint32_t M, uint32_t N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
-}
-constexpr uint32_t kIdesc = idesc(kBM, kBN);
+// Instruction descriptor: M128 N256, both operands K-major
+constexpr uint32_t kIdesc = idesc(kBM, kBN, 0);
 
 struct Tile {
   int b, tok0, f0;   // batch element, first token, first feature
@@ -236,7 +127,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     for (int i = tile0; i < p.total_tiles && ok; i += tile_step) {
       const Tile t = decode_tile(p, i);
       for (int kb = 0; kb < p.kblocks; ++kb) {
-        ok = warp_wait(&bar->empty[s], par, bar, p.status);
+        ok = warp_wait(&bar->empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           const uint32_t dst = sRing + s * kStageBytes;
@@ -263,12 +154,12 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     uint32_t ph = 0;
     for (int i = tile0; i < p.total_tiles && ok; i += tile_step, ++n) {
       const int a = n & 1;
-      ok = warp_wait(&bar->acc_empty[a], ((n >> 1) & 1) ^ 1, bar, p.status);   // epilogue has read tile n - 2
+      ok = warp_wait(&bar->acc_empty[a], ((n >> 1) & 1) ^ 1, &bar->abort_flag, p.status);   // epilogue has read tile n - 2
       if (!ok) break;
       tc_fence_after();
       const uint32_t d = tmem + a * kBN;
       for (int kb = 0; kb < p.kblocks; ++kb) {
-        ok = warp_wait(&bar->full[s], ph, bar, p.status);
+        ok = warp_wait(&bar->full[s], ph, &bar->abort_flag, p.status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = sRing + s * kStageBytes, sb = sa + kABytes;
@@ -298,7 +189,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     for (int i = tile0; i < p.total_tiles && ok; i += tile_step, ++n) {
       const Tile t = decode_tile(p, i);
       const int a = n & 1;
-      ok = warp_wait(&bar->acc_full[a], (n >> 1) & 1, bar, p.status);
+      ok = warp_wait(&bar->acc_full[a], (n >> 1) & 1, &bar->abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
       const int tok = t.tok0 + 32 * q4;
@@ -367,23 +258,6 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
 }
 
 // ---- host side ----------------------------------------------------------------------
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = (EncodeFn)ptr;
-  }
-  return fn;
-}
-
 // bf16 tensor (inner, rows, outer), contiguous, with a box of (64, box_rows, 1)
 bool map3(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint64_t outer, uint32_t box_rows) {
   const cuuint64_t dims[3] = {inner, rows, outer};
