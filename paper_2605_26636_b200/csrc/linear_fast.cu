@@ -27,12 +27,13 @@
 //
 // Partial layout per (batch, head, chunk), in floats:
 //   [0, 4096) KV[a][e], [4096, 4160) z[a], [4160, 4224) vsum[e]
-#include <cuda.h>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace jv {
 namespace {
+
+using namespace tc;
 
 constexpr int kD = 64;
 constexpr int kTileTok = 64;                  // tokens per shared-memory tile
@@ -40,59 +41,7 @@ constexpr int kTileBytes = kTileTok * kD * 2; // 8 KB
 constexpr int kOffZ = kD * kD, kOffVsum = kD * kD + kD;
 constexpr int kConsumers = 128;               // 4 MMA warps
 constexpr int kThreads = kConsumers + 32;     // + 1 producer warp
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait of a whole (converged) warp with a warp-uniform outcome.  On expiry the
-// status word and the CTA's abort flag are set and every role leaves its loop.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status) {
-  bool ok = mbar_try(bar, parity);
-  if (!ok) {
-    unsigned long long t0 = 0;
-    for (uint32_t spin = 0;; ++spin) {
-      if (mbar_try(bar, parity)) { ok = true; break; }
-      if ((spin & 63u) == 63u) {
-        if (*abort_flag) break;
-        const unsigned long long now = globaltimer();
-        if (t0 == 0) t0 = now;
-        else if (now - t0 > kWaitLimitNs) {
-          *abort_flag = 1;
-          atomicOr(status, kStatusTimeout);
-          break;
-        }
-      }
-    }
-  }
-  return __all_sync(0xffffffffu, ok);
-}
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}\n" : "=r"(pred));
-  return pred != 0;
-}
 // 64 tokens x 64 channels of a [B*H, N, 64] tensor -> shared memory (128-byte swizzle);
 // tokens past N arrive as zeros.
 __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int tok, int bh) {
@@ -289,36 +238,8 @@ constexpr int kDenRing = 8;                             // denominators of the t
 constexpr size_t kApplySmem = (size_t)(kApplyStages + 2) * kApplyTileBytes + kTileBytes + 1024 + kD * sizeof(float) +
                               (size_t)kDenRing * kApplyTok * sizeof(float) + sizeof(ApplyBars);
 
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, B MN-major, M = 128, N = 64.
-constexpr uint32_t kIdescApply = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-// Waits for this thread's outstanding tensor-memory loads; the registers are threaded through
-// the statement so that no use of them can be scheduled ahead of the wait.
-__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :: "memory");
-}
-
+constexpr uint32_t kIdescApply = idesc(128, 64, 1);
 __global__ void __launch_bounds__(kApplyThreads, 2)
 lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapO,
                  const float* __restrict__ partial, int* status, int N, int span_tokens, int nchunk, int state_elems,
@@ -649,12 +570,6 @@ struct __align__(8) DwBars {
 };
 constexpr size_t kDwSmem = (size_t)kDwStages * kDwStageBytes + 1024 + sizeof(DwBars);
 
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c1, int c2, int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-
 __global__ void __launch_bounds__(kDwThreads, 2)
 dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapOld,
                 const __grid_constant__ CUtensorMap mapOst, const float* __restrict__ w, int* status, int H,
@@ -689,8 +604,8 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
         const int bh = i / npatch, pt = i - bh * npatch;
         const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
         mbar_expect_tx(&bars->full[s], kDwVBytes + kDwOBytes);
-        tma_load_4d(smem + s * kDwStageBytes, &mapV, &bars->full[s], x0 - 1, y0 - 1, bh);
-        tma_load_4d(smem + s * kDwStageBytes + 23552, &mapOld, &bars->full[s], x0, y0, bh);
+        tma_load_4d(smem + s * kDwStageBytes, &mapV, &bars->full[s], 0, x0 - 1, y0 - 1, bh);
+        tma_load_4d(smem + s * kDwStageBytes + 23552, &mapOld, &bars->full[s], 0, x0, y0, bh);
       }
       __syncwarp();
       ++issued;
@@ -859,22 +774,6 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
 }
 
 // ---- host side ---------------------------------------------------------------------------
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeFn encode_fn() {
-  static EncodeFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      return nullptr;
-    fn = (EncodeFn)ptr;
-  }
-  return fn;
-}
-// [BH, N, 64] bf16 as a 3-D tensor (channel, token, batch*head); box = 64 channels x box_tok tokens
 bool make_map(CUtensorMap* m, const void* ptr, int BH, int N, int box_tok) {
   EncodeFn enc = encode_fn();
   if (!enc) return false;
