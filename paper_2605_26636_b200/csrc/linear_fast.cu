@@ -556,13 +556,15 @@ __device__ __forceinline__ uint64_t fma2f(uint64_t a, uint64_t b, uint64_t c) {
 // ---- o += depth-wise 3 x 3 convolution of V, staged through shared memory by TMA ----------------
 // Persistent CTAs loop over patches of 8 grid rows x 16 grid columns of one (batch, head).  Per
 // patch the producer warp brings in the 10 x 18 halo of V (out-of-grid taps arrive as the zeros
-// of the padding) and the 8 x 16 patch of o; warp w owns patch row w: a lane owns 4 channels
-// (8 bytes) and 8 consecutive tokens and slides the 3 x 3 window along x, adds the result to o in
-// place, and the warp writes its row back with one TMA store (clipped at the grid edge).
+// of the padding); warp w owns patch row w: a lane owns 4 channels (8 bytes) and 8 consecutive
+// tokens and slides the 3 x 3 window along x; the warp rounds its row of the result to bf16 and
+// adds it into o with one TMA reduction (cp.reduce.async.bulk.tensor .add, clipped at the grid
+// edge), so o is never read here.  Every element of o receives exactly one addition: the result
+// does not depend on the order of the patches.
 constexpr int kDwStages = 2;
 constexpr int kDwVBytes = 10 * 18 * 128;            // 23040
 constexpr int kDwOBytes = 8 * 16 * 128;             // 16384
-constexpr int kDwStageBytes = 23552 + kDwOBytes;    // V halo (padded to a multiple of 512) + o patch
+constexpr int kDwStageBytes = 23552 + kDwOBytes;    // V halo (padded to a multiple of 512) + the convolved patch on its way out
 constexpr int kDwThreads = 288;                     // 8 row warps + 1 producer warp
 struct __align__(8) DwBars {
   uint64_t full[kDwStages], empty[kDwStages];
@@ -571,8 +573,7 @@ struct __align__(8) DwBars {
 constexpr size_t kDwSmem = (size_t)kDwStages * kDwStageBytes + 1024 + sizeof(DwBars);
 
 __global__ void __launch_bounds__(kDwThreads, 2)
-dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapOld,
-                const __grid_constant__ CUtensorMap mapOst, const float* __restrict__ w, int* status, int H,
+dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapOst, const float* __restrict__ w, int* status, int H,
                 int Hg, int ncol_blocks, int npatch, int total_items) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -603,9 +604,8 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
       if (elect_one()) {
         const int bh = i / npatch, pt = i - bh * npatch;
         const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
-        mbar_expect_tx(&bars->full[s], kDwVBytes + kDwOBytes);
+        mbar_expect_tx(&bars->full[s], kDwVBytes);
         tma_load_4d(smem + s * kDwStageBytes, &mapV, &bars->full[s], 0, x0 - 1, y0 - 1, bh);
-        tma_load_4d(smem + s * kDwStageBytes + 23552, &mapOld, &bars->full[s], 0, x0, y0, bh);
       }
       __syncwarp();
       ++issued;
@@ -651,18 +651,15 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
     unsigned char* os = smem_al + (size_t)s * kDwStageBytes + 23552 + (warp * 16 + half * 8) * 128 + c4 * 8;
 #pragma unroll
     for (int hk = 0; hk < 2; ++hk) {                       // two runs of four tokens: keeps the window in registers
-      uint2 vr[3][6], cur[4];
+      uint2 vr[3][6];
 #pragma unroll
       for (int dy = 0; dy < 3; ++dy)
 #pragma unroll
         for (int k = 0; k < 6; ++k)
           vr[dy][k] = *reinterpret_cast<const uint2*>(vs + ((warp + dy) * 18 + half * 8 + 4 * hk + k) * 128);
 #pragma unroll
-      for (int k = 0; k < 4; ++k) cur[k] = *reinterpret_cast<const uint2*>(os + (4 * hk + k) * 128);
-#pragma unroll
       for (int k = 0; k < 4; ++k) {
-        uint64_t a01 = pack2f(__uint_as_float(cur[k].x << 16), __uint_as_float(cur[k].x & 0xffff0000u));
-        uint64_t a23 = pack2f(__uint_as_float(cur[k].y << 16), __uint_as_float(cur[k].y & 0xffff0000u));
+        uint64_t a01 = 0ull, a23 = 0ull;
 #pragma unroll
         for (int dy = 0; dy < 3; ++dy)
 #pragma unroll
@@ -686,7 +683,7 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
     __syncwarp();
     if (lane == 0) {
       if (y0 + warp < Hg)      // a row below the grid is not stored at all; columns past the edge are clipped by the store
-        asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        asm volatile("cp.reduce.async.bulk.tensor.4d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
                    ::"l"(&mapOst), "r"(smem + s * kDwStageBytes + 23552 + warp * 2048), "r"(0), "r"(x0), "r"(y0 + warp), "r"(bh)
                    : "memory");
       asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -898,9 +895,8 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     const int run = 32;
     dim3 g4(ceil_div(ceil_div(N, run), 8), BH);
     if (a.dwc->k == 3) {
-      CUtensorMap mvg, mol, mos;
-      if (!make_map_grid(&mvg, a.v, BH, s.Hg, s.Wg, 18, 10) || !make_map_grid(&mol, a.o, BH, s.Hg, s.Wg, 16, 8) ||
-          !make_map_grid(&mos, a.o, BH, s.Hg, s.Wg, 16, 1))
+      CUtensorMap mvg, mos;
+      if (!make_map_grid(&mvg, a.v, BH, s.Hg, s.Wg, 18, 10) || !make_map_grid(&mos, a.o, BH, s.Hg, s.Wg, 16, 1))
         return cudaErrorInvalidValue;
       static bool dw_attr = false;
       if (!dw_attr) {
@@ -911,7 +907,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
       const long long items = (long long)npatch * BH;
       if (items > 0x7fffffffll) return cudaErrorInvalidValue;
       const int grid = (int)(items < 2 * 148 ? items : 2 * 148);
-      dwc3_tma_kernel<<<grid, kDwThreads, kDwSmem, st>>>(mvg, mol, mos, w, status, s.H, s.Hg, ncb, npatch, (int)items);
+      dwc3_tma_kernel<<<grid, kDwThreads, kDwSmem, st>>>(mvg, mos, w, status, s.H, s.Hg, ncb, npatch, (int)items);
     } else
       dwc_add_kernel<5><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
     count_launch();
