@@ -620,6 +620,10 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
   }
 
   // ================= row warps =================
+  // The kernels w come from the grid before this one, which retires only after the apply pass: from
+  // here on w is final and o holds the attention output.  (The producer warp above does not wait:
+  // V is an input of the call.)
+  griddep_wait();
   const int c4 = lane & 15, half = lane >> 4;              // channels 4 c4 .. 4 c4 + 3; tokens 8 half .. 8 half + 7
   uint64_t w01[9], w23[9];
   int cur_bh = -1;
@@ -730,6 +734,7 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
                float* __restrict__ w, int B, int T, int R) {
   // Launched behind the apply grid, which lets its dependents go only after it has seen the hidden
   // layer's grid complete: hidden is final here and this grid runs beside the apply pass.
+  griddep_launch_dependents();                         // the convolution grid may set up and prefetch V
   const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
   const bool t_ok = t < T;
   const float* wrow = W2 + (size_t)(t_ok ? t : 0) * R;
@@ -907,7 +912,15 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
       const long long items = (long long)npatch * BH;
       if (items > 0x7fffffffll) return cudaErrorInvalidValue;
       const int grid = (int)(items < 2 * 148 ? items : 2 * 148);
-      dwc3_tma_kernel<<<grid, kDwThreads, kDwSmem, st>>>(mvg, mos, w, status, s.H, s.Hg, ncb, npatch, (int)items);
+      cudaLaunchConfig_t dcfg = {};
+      dcfg.gridDim = dim3(grid);
+      dcfg.blockDim = dim3(kDwThreads);
+      dcfg.dynamicSmemBytes = kDwSmem;
+      dcfg.stream = st;
+      dcfg.attrs = attr;
+      dcfg.numAttrs = 1;
+      e = cudaLaunchKernelEx(&dcfg, dwc3_tma_kernel, mvg, mos, w, status, (int)s.H, (int)s.Hg, ncb, npatch, (int)items);
+      if (e != cudaSuccess) return e;
     } else
       dwc_add_kernel<5><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
     count_launch();
