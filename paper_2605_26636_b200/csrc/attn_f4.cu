@@ -109,7 +109,8 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
                const F4Params p) {
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
   const uint32_t sQ = smem_u32(smem), sK = sQ + kQT * kTileBytes, sV = sK + kStages * kTileBytes;
   const uint32_t sO = sV + kStages * kTileBytes;      // output staging, one tile per query tile

@@ -89,7 +89,8 @@ __global__ void __launch_bounds__(kThreads)
 lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                  float* __restrict__ partial, int* status, int N, int chunk_tokens, int state_elems) {
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
+  unsigned char* smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem = smem_u32(smem_al);      // stage s: K tile at s * 16 KB, V tile at s * 16 KB + 8 KB
   Ring* ring = reinterpret_cast<Ring*>(smem_al + (size_t)kStateStages * 2 * kTileBytes);
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
@@ -245,7 +246,8 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
                  const float* __restrict__ partial, int* status, int N, int span_tokens, int nchunk, int state_elems,
                  float eps) {
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
+  unsigned char* smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem = smem_u32(smem_al);                                       // Q ring
   unsigned char* out_ptr = smem_al + (size_t)kApplyStages * kApplyTileBytes;     // 2 staging tiles
   const uint32_t out_sm = smem + kApplyStages * kApplyTileBytes;
@@ -576,7 +578,8 @@ __global__ void __launch_bounds__(kDwThreads, 2)
 dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapOst, const float* __restrict__ w, int* status, int H,
                 int Hg, int ncol_blocks, int npatch, int total_items) {
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem_al = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
+  unsigned char* smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem = smem_u32(smem_al);
   DwBars* bars = reinterpret_cast<DwBars*>(smem_al + (size_t)kDwStages * kDwStageBytes);
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;

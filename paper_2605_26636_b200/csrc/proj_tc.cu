@@ -80,7 +80,8 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
                const __grid_constant__ CUtensorMap mapD0, const __grid_constant__ CUtensorMap mapD1,
                const __grid_constant__ CUtensorMap mapD2, const ProjParams p) {
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
   const uint32_t sRing = smem_u32(smem), sStage = sRing + kStages * kStageBytes;
 
