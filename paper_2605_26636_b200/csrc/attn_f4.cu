@@ -42,7 +42,10 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kFirstSoftmaxWarp = 3;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSub = 64;                    // keys per step
-constexpr int kPolyOf8 = 1;                 // of every 8 score pairs, this many take the polynomial exponential
+#ifndef JV_POLY_OF_8
+#define JV_POLY_OF_8 2
+#endif
+constexpr int kPolyOf8 = JV_POLY_OF_8;                 // of every 8 score pairs, this many take the polynomial exponential
 // Tensor-memory columns: S_t (and P_t over its first 32 columns) at 64 t, O_t at 256 + 64 t
 constexpr uint32_t kColS = 0, kColO = 256;
 

@@ -43,7 +43,10 @@ constexpr int kStages = 4;                 // K and V ring depth
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSub = 64;                    // keys per softmax / MMA step: half a key tile
-constexpr int kPolyOf8 = 2;                 // of every 8 score pairs, this many take the polynomial exponential
+#ifndef JV_POLY_OF_8
+#define JV_POLY_OF_8 1
+#endif
+constexpr int kPolyOf8 = JV_POLY_OF_8;                 // of every 8 score pairs, this many take the polynomial exponential
 // Tensor-memory columns: S(t, b) at kColS + (2 t + b) * 64, O(t) at kColO + 64 t, P(t, b) at kColP + (2 t + b) * 32
 constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
 
