@@ -544,22 +544,13 @@ dwc_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ 
   }
 }
 
-// packed fp32x2 helpers of the convolution kernel
-__device__ __forceinline__ uint64_t pack2f(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ uint64_t fma2f(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
 // ---- o += depth-wise 3 x 3 convolution of V, staged through shared memory by TMA ----------------
 // Persistent CTAs loop over patches of 8 grid rows x 16 grid columns of one (batch, head).  Per
 // patch the producer warp brings in the 10 x 18 halo of V (out-of-grid taps arrive as the zeros
 // of the padding); warp w owns patch row w: a lane owns 4 channels (8 bytes) and 8 consecutive
-// tokens and slides the 3 x 3 window along x; the warp rounds its row of the result to bf16 and
+// tokens and slides the 3 x 3 window along x (each input row widened to fp32 once, scalar FMAs:
+// packed fp32x2 FMAs cost more in register-pair moves here than they save); the warp rounds its
+// row of the result to bf16 and
 // adds it into o with one TMA reduction (cp.reduce.async.bulk.tensor .add, clipped at the grid
 // edge), so o is never read here.  Every element of o receives exactly one addition: the result
 // does not depend on the order of the patches.
@@ -628,7 +619,7 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
   // V is an input of the call.)
   griddep_wait();
   const int c4 = lane & 15, half = lane >> 4;              // channels 4 c4 .. 4 c4 + 3; tokens 8 half .. 8 half + 7
-  uint64_t w01[9], w23[9];
+  float wt[4][9];                                          // weights of this thread's 4 channels, [channel][tap]
   int cur_bh = -1;
   int s = 0;
   uint32_t par = 0;
@@ -636,7 +627,7 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
   for (int i = blockIdx.x; i < total_items && ok; i += gridDim.x) {
     const int bh = i / npatch, pt = i - bh * npatch;
     const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
-    if (bh != cur_bh) {      // weights of this thread's 4 channels: w[ch][tap] -> per tap two fp32 pairs
+    if (bh != cur_bh) {
       cur_bh = bh;
       const int b = bh / H, h = bh - b * H;
       const float4* wp = reinterpret_cast<const float4*>(w + ((size_t)b * H * kD + (size_t)h * kD + 4 * c4) * 9);
@@ -647,38 +638,42 @@ dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant_
         wf[4 * k] = t4.x; wf[4 * k + 1] = t4.y; wf[4 * k + 2] = t4.z; wf[4 * k + 3] = t4.w;
       }
 #pragma unroll
-      for (int tap = 0; tap < 9; ++tap) {
-        w01[tap] = pack2f(wf[tap], wf[9 + tap]);
-        w23[tap] = pack2f(wf[18 + tap], wf[27 + tap]);
-      }
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int tap = 0; tap < 9; ++tap) wt[c][tap] = wf[9 * c + tap];
     }
     ok = warp_wait(&bars->full[s], par, &bars->abort_flag, status);
     if (!ok) break;
     const unsigned char* vs = smem_al + (size_t)s * kDwStageBytes + c4 * 8;            // halo: [10][18][128 B]
     unsigned char* os = smem_al + (size_t)s * kDwStageBytes + 23552 + (warp * 16 + half * 8) * 128 + c4 * 8;
 #pragma unroll
-    for (int hk = 0; hk < 2; ++hk) {                       // two runs of four tokens: keeps the window in registers
-      uint2 vr[3][6];
+    for (int hk = 0; hk < 2; ++hk) {                       // two runs of four tokens
+      float acc[4][4];
 #pragma unroll
-      for (int dy = 0; dy < 3; ++dy)
+      for (int k = 0; k < 4; ++k)
 #pragma unroll
-        for (int k = 0; k < 6; ++k)
-          vr[dy][k] = *reinterpret_cast<const uint2*>(vs + ((warp + dy) * 18 + half * 8 + 4 * hk + k) * 128);
+        for (int c = 0; c < 4; ++c) acc[k][c] = 0.f;
+#pragma unroll
+      for (int dy = 0; dy < 3; ++dy) {
+        float u[6][4];                                     // the six tokens of this input row, widened once
+#pragma unroll
+        for (int k = 0; k < 6; ++k) {
+          const uint2 t2 = *reinterpret_cast<const uint2*>(vs + ((warp + dy) * 18 + half * 8 + 4 * hk + k) * 128);
+          u[k][0] = __uint_as_float(t2.x << 16);
+          u[k][1] = __uint_as_float(t2.x & 0xffff0000u);
+          u[k][2] = __uint_as_float(t2.y << 16);
+          u[k][3] = __uint_as_float(t2.y & 0xffff0000u);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+          for (int dx = 0; dx < 3; ++dx)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[k][c] = fmaf(wt[c][3 * dy + dx], u[k + dx][c], acc[k][c]);
+      }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        uint64_t a01 = 0ull, a23 = 0ull;
-#pragma unroll
-        for (int dy = 0; dy < 3; ++dy)
-#pragma unroll
-          for (int dx = 0; dx < 3; ++dx) {
-            const uint2 t2 = vr[dy][k + dx];
-            a01 = fma2f(w01[3 * dy + dx], pack2f(__uint_as_float(t2.x << 16), __uint_as_float(t2.x & 0xffff0000u)), a01);
-            a23 = fma2f(w23[3 * dy + dx], pack2f(__uint_as_float(t2.y << 16), __uint_as_float(t2.y & 0xffff0000u)), a23);
-          }
-        float r0, r1, r2, r3;
-        asm("mov.b64 {%0, %1}, %2;" : "=f"(r0), "=f"(r1) : "l"(a01));
-        asm("mov.b64 {%0, %1}, %2;" : "=f"(r2), "=f"(r3) : "l"(a23));
-        __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc[k][0], acc[k][1]), hi = __floats2bfloat162_rn(acc[k][2], acc[k][3]);
         uint2 out;
         out.x = *reinterpret_cast<uint32_t*>(&lo);
         out.y = *reinterpret_cast<uint32_t*>(&hi);
