@@ -216,6 +216,50 @@ def test_degenerate_inputs(jv, oracle, both_paths):
     assert rel_err(jv.window_attn(dq, dk, dv, 16, 16, 16, 16), oracle.window_attn(qb, kb, v, 16, 16, 16, 16)) <= TOL["bf16"]
 
 
+def test_back_to_back_calls_match_isolated_calls_bit_for_bit(jv):
+    """Every kernel is deterministic, so a chain of calls enqueued without any synchronisation (kernels of
+    neighbouring calls overlap through programmatic launches and share the workspace) must reproduce, bit
+    for bit, what each call gives when it runs alone between two synchronisations."""
+    B, H, Hg, Wg = 2, 4, 40, 36
+    N, C = Hg * Wg, 64 * H
+    q, k, v = _dev(inputs.custom_qkv(B, H, N, 64, "bf16", seed=77))
+    d = dwc_to_device(inputs.dwc_weights(C, 32, 3, 5), DEV)
+    x = inputs.normal((B, N, C), 991, "bf16").to(DEV)
+    w, b = (t.to(DEV) for t in inputs.proj_weights(3 * C, C, 992))
+    wo, bo = (t.to(DEV) for t in inputs.proj_weights(C, C, 993))
+    shape = jv.make_shape(q, Hg, Wg)
+    ws = jv.alloc_workspace("L", shape, jv.make_dwc(d, DEV), DEV)
+
+    def chain(sync):
+        outs = []
+        def done(t):
+            if sync:
+                torch.cuda.synchronize()
+            outs.append(t)
+        q1, k1, v1 = jv.qkv_proj(x, w, b, H, Hg, Wg)
+        done(q1)
+        o1 = jv.linear_attn(q1, k1, v1, Hg, Wg, dwc=d, ws=ws)
+        done(o1)
+        o2 = jv.linear_attn(q, k, v, Hg, Wg, ws=ws)              # same workspace, no convolution
+        done(o2)
+        o3 = jv.window_attn(q1, k1, v1, Hg, Wg, 16, 16)
+        done(o3)
+        o4 = jv.linear_attn(k, q, v, Hg, Wg, dwc=d, ws=ws)
+        done(o4)
+        o5 = jv.full_attn(q1, k1, v1)
+        done(o5)
+        done(jv.out_proj(o4, wo, bo, Hg, Wg))
+        torch.cuda.synchronize()
+        return outs
+
+    ref = chain(sync=True)
+    for rep in range(3):
+        ws.fill_(0xFF)
+        got = chain(sync=False)
+        for i, (a, r) in enumerate(zip(got, ref)):
+            assert torch.equal(a, r), (rep, i)
+
+
 def test_bit_determinism(jv):
     w = inputs.WORKLOADS["dinov3_l"]
     q, k, v = _dev(inputs.custom_qkv(2, 4, 64 * 64, 64, "bf16", seed=3))
