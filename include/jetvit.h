@@ -28,7 +28,9 @@
  *             before anything is launched.  There is no CPU fallback: without a
  *             usable sm_100 device the calls return JV_ERR_CUDA/JV_ERR_UNSUPPORTED.
  *             Kernels bound every wait; one that gives up records
- *             JV_ERR_TIMEOUT, which jv_device_status() reports.
+ *             JV_ERR_TIMEOUT, which jv_device_status() reports.  With the
+ *             environment variable JETVIT_DEBUG set, a call that returns
+ *             JV_ERR_CUDA also prints the CUDA error string to stderr.
  *   Precision bf16 tensors: bf16 tensor-core products with fp32 accumulation,
  *             fp32 softmax / state, round-to-nearest-even output.  f32 tensors:
  *             fp32 arithmetic throughout (no tf32).
