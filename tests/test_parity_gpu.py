@@ -194,6 +194,19 @@ def test_full_attention_with_a_rising_reference(jv, oracle, n_tokens):
     assert rel_err(out, oracle.full_attn(q, k2, v)) <= TOL["bf16"]
 
 
+def test_full_and_linear_take_any_token_count(jv, oracle):
+    """F and L (without the convolution) do not look at the grid: a DINOv3 sequence with its five prefix
+    tokens (CLS + 4 registers) in front of a 64x64 grid is just 4101 tokens, passed as a 1 x 4101 grid."""
+    B, H, n_tok = 1, 3, 5 + 64 * 64
+    q, k, v = inputs.custom_qkv(B, H, n_tok, 64, "bf16", seed=4101)
+    dq, dk, dv = _dev((q, k, v))
+    of = jv.full_attn(dq, dk, dv, 1, n_tok)
+    ol = jv.linear_attn(dq, dk, dv, 1, n_tok)
+    assert rel_err(ol, oracle.linear_attn(q, k, v, 1, n_tok)) <= TOL["bf16"]
+    sl = (slice(0, 1), slice(1, 2))
+    assert rel_err(of[sl], oracle.full_attn(q[sl], k[sl], v[sl])) <= TOL["bf16"]
+
+
 def test_explicit_scale_and_eps(jv, oracle, both_paths):
     q, k, v = inputs.custom_qkv(1, 2, 16 * 16, 64, "bf16", seed=8)
     dq, dk, dv = _dev((q, k, v))
