@@ -14,8 +14,8 @@
  * Conventions shared by every call
  *   Tensors   q, k, v, o are DEVICE pointers to [B, H, N, D] contiguous arrays,
  *             D fastest, N = Hg * Wg, token t at grid position (t / Wg, t % Wg).
- *             All four have the element type jv_shape.dtype; o must not alias an
- *             input.  Pointers must be 16-byte aligned.
+ *             All four have the element type jv_shape.dtype; o must not share a
+ *             byte with an input.  Pointers must be 16-byte aligned.
  *   Ownership The caller owns every buffer and the stream.  The library never
  *             allocates or frees device memory; scratch comes from the caller
  *             through (ws, ws_bytes), sized by jv_workspace_bytes(), 256-byte
@@ -27,10 +27,17 @@
  *   Errors    Return codes only.  Every argument error is found on the host
  *             before anything is launched.  There is no CPU fallback: without a
  *             usable sm_100 device the calls return JV_ERR_CUDA/JV_ERR_UNSUPPORTED.
- *             Kernels bound every wait; one that gives up records
- *             JV_ERR_TIMEOUT, which jv_device_status() reports.  With the
- *             environment variable JETVIT_DEBUG set, a call that returns
- *             JV_ERR_CUDA also prints the CUDA error string to stderr.
+ *             Kernels bound every wait (2 s); one that gives up sets a sticky
+ *             per-device status word and returns, and jv_device_status()
+ *             reports JV_ERR_TIMEOUT.  While the word is set, the tensor-core
+ *             kernels (bf16, D = 64) that are launched leave at once WITHOUT
+ *             writing their output: calls keep returning JV_OK (they only
+ *             enqueue) and o keeps its old contents until jv_device_status()
+ *             has been called, which reads and clears the word.  A caller that
+ *             must know that its results are valid calls jv_device_status()
+ *             after the work it cares about.  With the environment variable
+ *             JETVIT_DEBUG set, a call that returns JV_ERR_CUDA also prints
+ *             the CUDA error string to stderr.
  *   Precision bf16 tensors: bf16 tensor-core products with fp32 accumulation,
  *             fp32 softmax / state, round-to-nearest-even output.  f32 tensors:
  *             fp32 arithmetic throughout (no tf32).
@@ -48,7 +55,7 @@ extern "C" {
 typedef enum {
   JV_OK = 0,
   JV_ERR_INVALID_ARG = 1,  /* null / misaligned pointer, non-positive size, bad schedule character */
-  JV_ERR_UNSUPPORTED = 2,  /* shape or dtype outside what the kernels cover (e.g. D > 256) */
+  JV_ERR_UNSUPPORTED = 2,  /* shape or dtype outside what the kernels cover (e.g. D > 128) */
   JV_ERR_WORKSPACE = 3,    /* ws is NULL, misaligned or smaller than jv_workspace_bytes() */
   JV_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed */
   JV_ERR_TIMEOUT = 5       /* a kernel gave up on a bounded wait */
@@ -118,10 +125,13 @@ jv_status jv_linear_attn(const void* q, const void* k, const void* v, void* o, c
  * passes only inputs and outputs.  The call allocates nothing and frees nothing.
  *
  *   Limit     jv_workspace_bytes('L', shape, dwc) must not exceed JV_STATIC_SCRATCH_BYTES
- *             (16 MiB: enough for B*H*N up to about 3.9 M token-heads at D = 64, e.g.
- *             B=8, H=16, 64x64 grid, or B=1, H=16, 128x128 grid).  Larger problems are
- *             refused with JV_ERR_WORKSPACE before anything is launched; use
- *             jv_linear_attn with your own buffer for those.
+ *             (16 MiB).  The scratch grows with B * H (one or more 16.5 KiB partial
+ *             states per (batch, head): about 6 MiB for B=8, H=16 on a 64x64 grid, 5 MiB
+ *             for B=1, H=16 on a 128x128 grid), not with the token count, plus
+ *             B * H * D * k * k * 4 bytes of kernels with the convolution; roughly
+ *             B * H <= 480 fits.  Larger problems are refused with JV_ERR_WORKSPACE
+ *             before anything is launched; use jv_linear_attn with your own buffer
+ *             for those.
  *   Cost      every GPU on which the library is loaded carries the 16 MiB array until the
  *             process exits, whether or not this function is ever called.
  *   Set-up    the first call on each device looks up the array's device address (that
@@ -174,7 +184,7 @@ jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* c
 
 /*
  * The projections either side of a mixer (the W_Q, W_K, W_V and W_O that a searched model
- * inherits from its base model for every block, Sec. 3.3), as tensor-core GEMMs that write
+ * inherits from its base model for every block, Sec. 3.2.4), as tensor-core GEMMs that write
  * and read the mixers' [B, H, N, D] layout directly: no transpose pass between projection
  * and mixer.  bf16 only, D = 64 only (JV_ERR_UNSUPPORTED otherwise); C = H * D.
  *
@@ -202,6 +212,17 @@ jv_status jv_out_proj(const void* o, const void* w, const float* bias, void* y, 
  * call, or JV_ERR_CUDA if the stream reports a CUDA error.
  */
 jv_status jv_device_status(void* cuda_stream);
+
+/*
+ * Self-test of the bounded waits (for test suites; the paper has no counterpart).  Enqueues a
+ * one-warp kernel that waits, through the same bounded wait the mixers use, on a barrier
+ * that nothing ever completes; after limit_us microseconds (1 .. 1000000) the wait gives up,
+ * sets the sticky status word exactly as a mixer kernel would, and the kernel returns.
+ * Nothing faults or hangs and the context stays usable.  gave_up is NULL or a DEVICE pointer
+ * to an int that receives 1 if the wait ran out.  Afterwards jv_device_status() returns
+ * JV_ERR_TIMEOUT once, then JV_OK.
+ */
+jv_status jv_selftest_wait_timeout(uint32_t limit_us, int32_t* gave_up, void* cuda_stream);
 
 /*
  * Tuning / dispatch switch, mainly for tests: 0 (default) lets every call pick

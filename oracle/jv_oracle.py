@@ -153,7 +153,7 @@ def hybrid_mixers(schedule, q, k, v, Hg, Wg, win_h, win_w, scale=None, eps=1e-6,
 
 
 def qkv_proj(x, w, bias, H):
-    """The block's input projection W_Q | W_K | W_V (Sec. 3.3: inherited linear layers),
+    """The block's input projection W_Q | W_K | W_V (Sec. 3.2.4: inherited linear layers),
     written out as the definition: x [B, N, C], w [3C, C] (row = output feature
     which*C + h*D + e), bias [3C] or None -> q, k, v, each [B, H, N, D] with D = C / H:
     q[b, h, n, e] = sum_c x[b, n, c] w[h*D + e, c] + bias[h*D + e], and k, v from the
@@ -175,7 +175,7 @@ def qkv_proj(x, w, bias, H):
 
 
 def out_proj(o, w, bias):
-    """The block's output projection W_O (Sec. 3.3): o [B, H, N, D], w [C, C] with C = H*D
+    """The block's output projection W_O (Sec. 3.2.4): o [B, H, N, D], w [C, C] with C = H*D
     (column = input feature h*D + e), bias [C] or None -> y [B, N, C]:
     y[b, n, f] = sum_{h, e} o[b, h, n, e] w[f, h*D + e] + bias[f]."""
     o, w = _f64(o), _f64(w)

@@ -17,6 +17,16 @@ std::atomic<int32_t> g_force_generic{0};
 
 bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
 
+// [a, a + na) and [b, b + nb) share at least one byte
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + nb && y < x + na;
+}
+
+size_t tensor_bytes(const jv_shape* s) {
+  return (size_t)s->B * s->H * s->Hg * s->Wg * s->D * (s->dtype == JV_F32 ? 4 : 2);
+}
+
 jv_status check_shape(const jv_shape* s) {
   if (!s) return JV_ERR_INVALID_ARG;
   if (s->B <= 0 || s->H <= 0 || s->Hg <= 0 || s->Wg <= 0 || s->D <= 0) return JV_ERR_INVALID_ARG;
@@ -33,8 +43,8 @@ jv_status check_shape(const jv_shape* s) {
 jv_status check_tensors(const void* q, const void* k, const void* v, const void* o, const jv_shape* s) {
   if (!q || !k || !v || !o) return JV_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return JV_ERR_INVALID_ARG;
-  if (o == q || o == k || o == v) return JV_ERR_INVALID_ARG;
-  (void)s;
+  const size_t n = tensor_bytes(s);      // o may not share a byte with an input
+  if (overlaps(o, n, q, n) || overlaps(o, n, k, n) || overlaps(o, n, v, n)) return JV_ERR_INVALID_ARG;
   return JV_OK;
 }
 
@@ -71,15 +81,16 @@ jv_status check_device() {
   return major == 10 ? JV_OK : JV_ERR_UNSUPPORTED;
 }
 
-jv_status check_proj(const jv_shape* s, const void* const* ptrs, int nptr, int nin) {
+// ptrs[0 .. nin) are inputs, ptrs[nin .. nptr) outputs; bytes[i] is the extent of ptrs[i]
+jv_status check_proj(const jv_shape* s, const void* const* ptrs, const size_t* bytes, int nptr, int nin) {
   jv_status st = check_shape(s);
   if (st != JV_OK) return st;
   for (int i = 0; i < nptr; ++i)
     if (!ptrs[i] || !aligned(ptrs[i], 16)) return JV_ERR_INVALID_ARG;
-  for (int i = nin; i < nptr; ++i)           // outputs alias neither an input nor each other
+  if (s->dtype != JV_BF16 || s->D != 64) return JV_ERR_UNSUPPORTED;   // (the extents below assume both)
+  for (int i = nin; i < nptr; ++i)           // outputs overlap neither an input nor each other
     for (int j = 0; j < i; ++j)
-      if (ptrs[i] == ptrs[j]) return JV_ERR_INVALID_ARG;
-  if (s->dtype != JV_BF16 || s->D != 64) return JV_ERR_UNSUPPORTED;
+      if (overlaps(ptrs[i], bytes[i], ptrs[j], bytes[j])) return JV_ERR_INVALID_ARG;
   return JV_OK;
 }
 
@@ -133,6 +144,26 @@ int* device_status_ptr() {
 }
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return -1; }
+  return dev;
+}
+
+int device_sm_count() {
+  static std::atomic<int> cache[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0 || dev >= kMaxDevices) return kDefaultSmCount;
+  int n = cache[dev].load(std::memory_order_relaxed);
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    return kDefaultSmCount;
+  }
+  cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
 
 }  // namespace jv
 
@@ -227,8 +258,11 @@ jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* c
 
 jv_status jv_qkv_proj(const void* x, const void* w, const float* bias, void* q, void* k, void* v,
                       const jv_shape* shape, void* cuda_stream) {
+  if (!shape) return JV_ERR_INVALID_ARG;
   const void* ptrs[5] = {x, w, q, k, v};
-  jv_status st = check_proj(shape, ptrs, 5, 2);
+  const size_t C = (size_t)shape->H * shape->D, nt = (size_t)shape->B * shape->Hg * shape->Wg * C * 2;
+  const size_t bytes[5] = {nt, 3 * C * C * 2, nt, nt, nt};
+  jv_status st = check_proj(shape, ptrs, bytes, 5, 2);
   if (st != JV_OK) return st;
   if (bias && !aligned(bias, 16)) return JV_ERR_INVALID_ARG;
   if ((st = check_device()) != JV_OK) return st;
@@ -240,8 +274,11 @@ jv_status jv_qkv_proj(const void* x, const void* w, const float* bias, void* q, 
 
 jv_status jv_out_proj(const void* o, const void* w, const float* bias, void* y, const jv_shape* shape,
                       void* cuda_stream) {
+  if (!shape) return JV_ERR_INVALID_ARG;
   const void* ptrs[3] = {o, w, y};
-  jv_status st = check_proj(shape, ptrs, 3, 2);
+  const size_t C = (size_t)shape->H * shape->D, nt = (size_t)shape->B * shape->Hg * shape->Wg * C * 2;
+  const size_t bytes[3] = {nt, C * C * 2, nt};
+  jv_status st = check_proj(shape, ptrs, bytes, 3, 2);
   if (st != JV_OK) return st;
   if (bias && !aligned(bias, 16)) return JV_ERR_INVALID_ARG;
   if ((st = check_device()) != JV_OK) return st;

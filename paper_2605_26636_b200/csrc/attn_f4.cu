@@ -466,24 +466,15 @@ cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st) {
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attn_f4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attn_f4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
-      num_sms = 0;
-      cudaGetLastError();
-      return cudaErrorUnknown;
-    }
-  }
+  static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
+  cudaError_t e = smem_opt_in.run([] {
+    cudaError_t r = cudaFuncSetAttribute(attn_f4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (r == cudaSuccess)
+      r = cudaFuncSetAttribute(attn_f4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    return r;
+  });
+  if (e != cudaSuccess) return e;
+  const int num_sms = device_sm_count();
   F4Params p;
   p.status = status;
   p.N = N;

@@ -688,12 +688,11 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
+  cudaError_t e = smem_opt_in.run([] {
+    return cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  });
+  if (e != cudaSuccess) return e;
   TcParams p;
   p.o = (__nv_bfloat16*)a.o;
   p.status = status;
@@ -717,16 +716,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   p.div_nwx = make_fastdiv((uint32_t)p.nwx);
   p.scale_log2 = a.scale * 1.4426950408889634f;
   // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no more)
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
-      num_sms = 0;
-      cudaGetLastError();
-      return cudaErrorUnknown;
-    }
-  }
+  const int num_sms = device_sm_count();
   const int grid = p.total_items < num_sms ? p.total_items : num_sms;
   attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
   count_launch();

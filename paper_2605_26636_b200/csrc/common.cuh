@@ -5,17 +5,46 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "jetvit.h"
 
 namespace jv {
 
 // ---- device status word ---------------------------------------------------
-// One int per device context lives in status.cu; kernels receive its device
-// address and OR error bits into it.  Bit 0: a bounded wait ran out.
+// One int per device lives in api.cu; kernels receive its device address and OR
+// error bits into it.  Bit 0: a bounded wait ran out.
 constexpr int kStatusTimeout = 1;
 
 int* device_status_ptr();        // device address of the status word (nullptr on failure)
 void count_launch(int n = 1);    // launch counter behind jv_launch_count()
+
+// ---- per-device facts --------------------------------------------------------
+// The library may be used on several GPUs from one process (one device current per
+// call), so whatever CUDA keeps per device is cached per device here.
+constexpr int kMaxDevices = 64;
+constexpr int kDefaultSmCount = 148;   // B200; used for planning when no device can be asked
+int current_device();            // index of the current device, -1 if it cannot be read
+int device_sm_count();           // SM count of the current device (kDefaultSmCount without one)
+
+// Runs `f` (which returns a cudaError_t) once per device, with that device current:
+// the opt-in to more than 48 KB of dynamic shared memory is a per-device function
+// attribute.  Two host threads may both run f; it is idempotent.
+class OncePerDevice {
+ public:
+  template <typename F>
+  cudaError_t run(F f) {
+    const int d = current_device();
+    if (d < 0 || d >= kMaxDevices) return f();
+    if (done_[d].load(std::memory_order_acquire)) return cudaSuccess;
+    const cudaError_t e = f();
+    if (e == cudaSuccess) done_[d].store(1, std::memory_order_release);
+    return e;
+  }
+
+ private:
+  std::atomic<int> done_[kMaxDevices] = {};
+};
 
 // ---- element access -------------------------------------------------------
 __device__ __forceinline__ float to_f32(float x) { return x; }
@@ -60,8 +89,8 @@ struct AttnArgs {
   int dtype;
 };
 cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st);
-// tcgen05 path: bf16, D == 64.  full = true: F over all N tokens; else W with
-// (wh, ww) windows, ww a power of two dividing 128, wh*ww a multiple of 128 and <= 256...
+// tcgen05 path: bf16, D == 64.  full = true: F over all N tokens; else W with (wh, ww)
+// windows whose width ww is a power of two <= 128 (a tile is a box of ww x 128/ww tokens).
 bool attn_tc_supported(const AttnArgs& a, bool full);
 cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream_t st);
 // tcgen05 path for full attention over long sequences (bf16, D == 64, N >= 1024): four query tiles per CTA
@@ -79,6 +108,10 @@ struct LinArgs {
 cudaError_t launch_linear_generic(const LinArgs& a, const LinPlan& p, cudaStream_t st);
 bool linear_fast_supported(const LinArgs& a);
 cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t st);
+// bf16, D == 64, 3 x 3 kernels: the apply pass with the convolution fused in
+bool linear_conv_supported(const LinArgs& a);
+cudaError_t launch_linear_apply_conv(const LinArgs& a, const LinPlan& p, const float* partial, const float* w,
+                                     int* status, bool programmatic, cudaStream_t st);
 // shared by both linear paths: hidden = SiLU(W1 s + b1), w = W2 hidden + b2, with
 // s = vsum / N read from vsum[bh * bh_stride + e]
 cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float* vsum, int bh_stride,

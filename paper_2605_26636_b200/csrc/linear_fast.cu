@@ -21,24 +21,24 @@
 // its first Q loads overlap the tail of the state kernel, and it waits for that grid
 // (griddepcontrol.wait) only before touching the partials.
 //
-// With the convolution on, the generator's hidden layer (a tiny kernel) runs between the
-// state pass and the apply pass, its output layer beside the apply pass, and a TMA-staged
-// depth-wise convolution pass over V and o follows both.
+// With the convolution on, the generator's two layers (tiny kernels laid out for latency) run
+// between the state pass and the apply pass.  3 x 3 kernels: the apply pass is the fused
+// apply + convolution kernel of linear_conv.cu.  5 x 5 kernels: the apply pass above, the output
+// layer beside it, and a read-modify-write convolution pass over o behind both.
 //
 // Partial layout per (batch, head, chunk), in floats:
 //   [0, 4096) KV[a][e], [4096, 4160) z[a], [4160, 4224) vsum[e]
 
-#include "tc_common.cuh"
+#include "lin_common.cuh"
 
 namespace jv {
 namespace {
 
 using namespace tc;
+using namespace lin;
 
-constexpr int kD = 64;
 constexpr int kTileTok = 64;                  // tokens per shared-memory tile
 constexpr int kTileBytes = kTileTok * kD * 2; // 8 KB
-constexpr int kOffZ = kD * kD, kOffVsum = kD * kD + kD;
 constexpr int kConsumers = 128;               // 4 MMA warps
 constexpr int kThreads = kConsumers + 32;     // + 1 producer warp
 
@@ -49,8 +49,6 @@ __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* m
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(tok), "r"(bh) : "memory");
 }
-__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
@@ -61,20 +59,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint32_t relu_bf16x2(uint32_t x) {
-  __nv_bfloat162 v = *reinterpret_cast<__nv_bfloat162*>(&x);
-  v = __hmax2(v, __float2bfloat162_rn(0.f));
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-__device__ __forceinline__ float2 bf16x2_to_f2(uint32_t x) {
-  return make_float2(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
-}
-
-// Byte offset of 16-byte chunk `ch` (0..7) of row `row` in a [rows][64 bf16] tile in the
-// 128-byte-swizzle layout (what TMA writes): chunks are XORed with the row index mod 8, so
-// ldmatrix reads of 8 rows hit 8 distinct bank groups.
-__device__ __forceinline__ uint32_t tile_off(int row, int ch) { return (uint32_t)(row * 128 + ((ch ^ (row & 7)) << 4)); }
-
 struct __align__(8) Ring {
   uint64_t full[8], empty[8];
   volatile uint32_t abort_flag;
@@ -115,6 +99,9 @@ lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant
 
   if (warp == 4) {
     // ================= TMA producer =================
+    // K is read exactly once in the whole call: it makes room in L2 first.  With the convolution
+    // on, V is read again by the apply pass: L2 is asked to keep it.
+    const uint64_t pol_k = l2_policy_evict_first(), pol_v = l2_policy_evict_last();
     int s = 0;
     uint32_t par = 1;
     int issued = 0;
@@ -125,8 +112,9 @@ lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant
       if (elect_one()) {
         mbar_expect_tx(&ring->full[s], 2 * kTileBytes);
         const int tok = t_begin + it * kTileTok;     // a chunk's last tile may run past t_end: only by whole
-        tma_load_tile(smem + s * 2 * kTileBytes, &mapK, &ring->full[s], tok, bh);              // zero rows past N
-        tma_load_tile(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], tok, bh);
+        tma_load_3d_hint(smem + s * 2 * kTileBytes, &mapK, &ring->full[s], 0, tok, bh, pol_k);   // zero rows past N
+        if (kVsum) tma_load_3d_hint(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], 0, tok, bh, pol_v);
+        else tma_load_tile(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], tok, bh);
       }
       __syncwarp();
       ++issued;
@@ -351,6 +339,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     griddep_wait();                                    // the grids before this one (state pass, generator's hidden layer) are complete
     griddep_launch_dependents();
     bool ok = *reinterpret_cast<volatile int*>(status) == 0;
+    if (!ok) bars->abort_flag = 1;                     // an earlier kernel gave up: every role of this CTA falls through at once
     {  // second pass of the reduction: chunk partials summed in a fixed order; KV -> bf16 MMA operand, z in fp32
       const float* P = partial + (size_t)bh * nchunk * state_elems;
 #pragma unroll
@@ -544,259 +533,146 @@ dwc_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ 
   }
 }
 
-// ---- o += depth-wise 3 x 3 convolution of V, staged through shared memory by TMA ----------------
-// Persistent CTAs loop over patches of 8 grid rows x 16 grid columns of one (batch, head).  Per
-// patch the producer warp brings in the 10 x 18 halo of V (out-of-grid taps arrive as the zeros
-// of the padding); warp w owns patch row w: a lane owns 4 channels (8 bytes) and 8 consecutive
-// tokens and slides the 3 x 3 window along x (each input row widened to fp32 once, scalar FMAs:
-// packed fp32x2 FMAs cost more in register-pair moves here than they save); the warp rounds its
-// row of the result to bf16 and
-// adds it into o with one TMA reduction (cp.reduce.async.bulk.tensor .add, clipped at the grid
-// edge), so o is never read here.  Every element of o receives exactly one addition: the result
-// does not depend on the order of the patches.
-constexpr int kDwStages = 2;
-constexpr int kDwVBytes = 10 * 18 * 128;            // 23040
-constexpr int kDwOBytes = 8 * 16 * 128;             // 16384
-constexpr int kDwStageBytes = 23552 + kDwOBytes;    // V halo (padded to a multiple of 512) + the convolved patch on its way out
-constexpr int kDwThreads = 288;                     // 8 row warps + 1 producer warp
-struct __align__(8) DwBars {
-  uint64_t full[kDwStages], empty[kDwStages];
-  volatile uint32_t abort_flag;
-};
-constexpr size_t kDwSmem = (size_t)kDwStages * kDwStageBytes + 1024 + sizeof(DwBars);
-
-__global__ void __launch_bounds__(kDwThreads, 2)
-dwc3_tma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapOst, const float* __restrict__ w, int* status, int H,
-                int Hg, int ncol_blocks, int npatch, int total_items) {
-  extern __shared__ unsigned char smem_raw[];
-  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
-  unsigned char* smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  const uint32_t smem = smem_u32(smem_al);
-  DwBars* bars = reinterpret_cast<DwBars*>(smem_al + (size_t)kDwStages * kDwStageBytes);
-  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kDwStages; ++s) {
-      mbar_init(&bars->full[s], 1);
-      mbar_init(&bars->empty[s], 8);            // one arrival per row warp
-    }
-    bars->abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  __syncthreads();
-  if (*reinterpret_cast<volatile int*>(status) != 0) return;
-
-  if (warp == 8) {
-    // ================= TMA producer =================
-    int s = 0, issued = 0;
-    uint32_t par = 1;
-    bool ok = true;
-    for (int i = blockIdx.x; i < total_items; i += gridDim.x) {
-      ok = warp_wait(&bars->empty[s], par, &bars->abort_flag, status);
-      if (!ok) break;
-      if (elect_one()) {
-        const int bh = i / npatch, pt = i - bh * npatch;
-        const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
-        mbar_expect_tx(&bars->full[s], kDwVBytes);
-        tma_load_4d(smem + s * kDwStageBytes, &mapV, &bars->full[s], 0, x0 - 1, y0 - 1, bh);
-      }
-      __syncwarp();
-      ++issued;
-      if (++s == kDwStages) { s = 0; par ^= 1; }
-    }
-    if (!ok && lane == 0) {
-      const unsigned long long t0 = globaltimer();
-      for (int g = max(0, issued - kDwStages); g < issued; ++g)
-        while (!mbar_try(&bars->full[g % kDwStages], (g / kDwStages) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
-    }
-    return;
-  }
-
-  // ================= row warps =================
-  // The kernels w come from the grid before this one, which retires only after the apply pass: from
-  // here on w is final and o holds the attention output.  (The producer warp above does not wait:
-  // V is an input of the call.)
-  griddep_wait();
-  const int c4 = lane & 15, half = lane >> 4;              // channels 4 c4 .. 4 c4 + 3; tokens 8 half .. 8 half + 7
-  float wt[4][9];                                          // weights of this thread's 4 channels, [channel][tap]
-  int cur_bh = -1;
-  int s = 0;
-  uint32_t par = 0;
-  bool ok = true;
-  for (int i = blockIdx.x; i < total_items && ok; i += gridDim.x) {
-    const int bh = i / npatch, pt = i - bh * npatch;
-    const int y0 = (pt / ncol_blocks) * 8, x0 = (pt % ncol_blocks) * 16;
-    if (bh != cur_bh) {
-      cur_bh = bh;
-      const int b = bh / H, h = bh - b * H;
-      const float4* wp = reinterpret_cast<const float4*>(w + ((size_t)b * H * kD + (size_t)h * kD + 4 * c4) * 9);
-      float wf[36];
-#pragma unroll
-      for (int k = 0; k < 9; ++k) {
-        const float4 t4 = __ldg(wp + k);
-        wf[4 * k] = t4.x; wf[4 * k + 1] = t4.y; wf[4 * k + 2] = t4.z; wf[4 * k + 3] = t4.w;
-      }
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int tap = 0; tap < 9; ++tap) wt[c][tap] = wf[9 * c + tap];
-    }
-    ok = warp_wait(&bars->full[s], par, &bars->abort_flag, status);
-    if (!ok) break;
-    const unsigned char* vs = smem_al + (size_t)s * kDwStageBytes + c4 * 8;            // halo: [10][18][128 B]
-    unsigned char* os = smem_al + (size_t)s * kDwStageBytes + 23552 + (warp * 16 + half * 8) * 128 + c4 * 8;
-#pragma unroll
-    for (int hk = 0; hk < 2; ++hk) {                       // two runs of four tokens
-      float acc[4][4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[k][c] = 0.f;
-#pragma unroll
-      for (int dy = 0; dy < 3; ++dy) {
-        float u[6][4];                                     // the six tokens of this input row, widened once
-#pragma unroll
-        for (int k = 0; k < 6; ++k) {
-          const uint2 t2 = *reinterpret_cast<const uint2*>(vs + ((warp + dy) * 18 + half * 8 + 4 * hk + k) * 128);
-          u[k][0] = __uint_as_float(t2.x << 16);
-          u[k][1] = __uint_as_float(t2.x & 0xffff0000u);
-          u[k][2] = __uint_as_float(t2.y << 16);
-          u[k][3] = __uint_as_float(t2.y & 0xffff0000u);
-        }
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-#pragma unroll
-          for (int dx = 0; dx < 3; ++dx)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) acc[k][c] = fmaf(wt[c][3 * dy + dx], u[k + dx][c], acc[k][c]);
-      }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc[k][0], acc[k][1]), hi = __floats2bfloat162_rn(acc[k][2], acc[k][3]);
-        uint2 out;
-        out.x = *reinterpret_cast<uint32_t*>(&lo);
-        out.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(os + (4 * hk + k) * 128) = out;
-      }
-    }
-    // this warp's row (16 tokens, 2 KB) back to global memory; the stage is free once the store has read it
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    if (lane == 0) {
-      if (y0 + warp < Hg)      // a row below the grid is not stored at all; columns past the edge are clipped by the store
-        asm volatile("cp.reduce.async.bulk.tensor.4d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
-                   ::"l"(&mapOst), "r"(smem + s * kDwStageBytes + 23552 + warp * 2048), "r"(0), "r"(x0), "r"(y0 + warp), "r"(bh)
-                   : "memory");
-      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-      asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-      mbar_arrive(&bars->empty[s]);
-    }
-    __syncwarp();
-    if (++s == kDwStages) { s = 0; par ^= 1; }
-  }
-  if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
-
 // ---- kernel generator of the squeeze dynamic convolution (Sec. 3.2.1), tuned for latency ------
-// hidden[b][r] = SiLU(b1[r] + sum_c W1[r][c] * mean_v[b][c]); one block per (r, b).  mean_v comes
-// straight from the chunk partials' v-sums (summed in a fixed order).
-__global__ void __launch_bounds__(128)
+// Both layers sit on the critical path between the state pass and the apply pass, so each is laid
+// out as ONE round trip of independent loads followed by arithmetic.
+//
+// hidden[b][r] = SiLU(b1[r] + sum_c W1[r][c] * mean_v[b][c]).  A block serves 8 values of r for one
+// sample: per tile of 1024 channels it forms the means (the chunk partials' v-sums, summed in chunk
+// order) in shared memory while the rows of W1 are already on their way, then warp w takes row r0 + w.
+constexpr int kGenTile = 1024;
+__global__ void __launch_bounds__(256)
 gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W1, const float* __restrict__ b1,
-                  float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n) {
-  __shared__ float red[4];
-  griddep_wait();                                      // the state pass is complete
-  griddep_launch_dependents();                         // the apply grid may set up and load Q meanwhile
-  const int r = blockIdx.x, b = blockIdx.y, C = H * kD;
-  float s = 0.f;
-  for (int c = threadIdx.x; c < C; c += 128) {
-    const int h = c / kD, e = c % kD;
-    const float* pv = partial + (size_t)(b * H + h) * nchunk * state_elems + kOffVsum + e;
-    float m = 0.f;
-    for (int k = 0; k < nchunk; ++k) m += pv[(size_t)k * state_elems];
-    s = fmaf(__ldg(&W1[(size_t)r * C + c]), m * inv_n, s);
+                  float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n, int early_trigger) {
+  __shared__ __align__(16) float s_sm[kGenTile];
+  // early_trigger: the grids behind this one each wait for their predecessor before they read its
+  // output, so they may be resident (set up, prefetching inputs of the call) while this one waits.
+  if (early_trigger) griddep_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * 8 + warp, b = blockIdx.y, C = H * kD;
+  const bool r_ok = r < R;
+  const float* wrow = W1 + (size_t)(r_ok ? r : 0) * C;
+  float dot = 0.f;
+  bool waited = false;
+  for (int c0 = 0; c0 < C; c0 += kGenTile) {           // C is a multiple of 64
+    float4 wv[kGenTile / 128];                         // this lane's part of the row: W1 is an input of the call
+#pragma unroll
+    for (int i = 0; i < kGenTile / 128; ++i) {
+      const int c = c0 + 4 * lane + 128 * i;
+      wv[i] = (r_ok && c < C) ? __ldg(reinterpret_cast<const float4*>(wrow + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (!waited) {
+      griddep_wait();                                  // the state pass is complete
+      if (!early_trigger) griddep_launch_dependents(); // the apply grid may set up and load Q meanwhile
+      waited = true;
+    }
+    __syncthreads();                                   // the previous tile's means have been consumed
+#pragma unroll
+    for (int i = 0; i < kGenTile / 256; ++i) {
+      const int c = c0 + threadIdx.x + 256 * i;
+      float m = 0.f;
+      if (c < C) {
+        const float* pv = partial + (size_t)(b * H + c / kD) * nchunk * state_elems + kOffVsum + c % kD;
+        for (int k = 0; k < nchunk; ++k) m += __ldcg(pv + (size_t)k * state_elems);
+      }
+      s_sm[threadIdx.x + 256 * i] = m * inv_n;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kGenTile / 128; ++i) {
+      const float4 sv = *reinterpret_cast<const float4*>(s_sm + 4 * lane + 128 * i);
+      dot = fmaf(wv[i].x, sv.x, fmaf(wv[i].y, sv.y, fmaf(wv[i].z, sv.z, fmaf(wv[i].w, sv.w, dot))));
+    }
   }
-  s = warp_sum(s);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const float x = ((red[0] + red[1]) + (red[2] + red[3])) + (b1 ? b1[r] : 0.f);
+  dot = warp_sum(dot);
+  if (lane == 0 && r_ok) {
+    const float x = dot + (b1 ? b1[r] : 0.f);
     hidden[(size_t)b * R + r] = x / (1.f + expf(-x));
   }
 }
 // w[b][t] = b2[t] + sum_r W2[t][r] * hidden[b][r]; 8 lanes per output t, 32 outputs per block, all
-// samples.  A lane's W2 values (r = part, part + 8, ...) are fetched 16 at a time, all loads in
-// flight together, and reused for up to 8 samples.
+// samples (8 at a time, their hidden vectors in shared memory).  kVec (R a multiple of 4): a lane's
+// part of the W2 row is fetched as float4, the whole row in flight at once.
+constexpr int kGenMaxR = 1024;
+template <bool kVec>
 __global__ void __launch_bounds__(256)
 gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, const float* __restrict__ b2,
-               float* __restrict__ w, int B, int T, int R) {
-  // Launched behind the apply grid, which lets its dependents go only after it has seen the hidden
-  // layer's grid complete: hidden is final here and this grid runs beside the apply pass.
-  griddep_launch_dependents();                         // the convolution grid may set up and prefetch V
+               float* __restrict__ w, int B, int T, int R, int wait_first) {
+  __shared__ __align__(16) float h_sm[8 * kGenMaxR];
+  // wait_first = 0: launched behind the apply grid, which lets its dependents go only after it has
+  // seen the hidden layer's grid complete: hidden is final here and this grid runs beside the apply
+  // pass; it waits at its end (below).  wait_first = 1: launched directly behind the hidden layer
+  // (or the state pass, with static kernels), ahead of the fused apply + convolution grid: it waits
+  // for its predecessor before it reads hidden.
+  griddep_launch_dependents();                         // the grid behind this one may set up and prefetch
   const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
   const bool t_ok = t < T;
   const float* wrow = W2 + (size_t)(t_ok ? t : 0) * R;
+  constexpr int kPer = kVec ? 4 : 16;                  // loads per lane and 128 values of r
+  bool waited = wait_first == 0;
   for (int b0 = 0; b0 < B; b0 += 8) {
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    const int nb = min(8, B - b0);
     for (int r0 = 0; r0 < R; r0 += 128) {
-      float wv[16];
+      float wv[16];                                    // W2 is an input of the call: on its way before the wait
+      if (kVec) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int r = r0 + part + 8 * i;
-        wv[i] = r < R ? __ldg(wrow + r) : 0.f;
+        for (int i = 0; i < kPer; ++i) {
+          const int r = r0 + 4 * part + 32 * i;
+          const float4 x = r < R ? __ldg(reinterpret_cast<const float4*>(wrow + r)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          wv[4 * i] = x.x; wv[4 * i + 1] = x.y; wv[4 * i + 2] = x.z; wv[4 * i + 3] = x.w;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int r = r0 + part + 8 * i;
+          wv[i] = r < R ? __ldg(wrow + r) : 0.f;
+        }
+      }
+      if (r0 == 0) {                                   // this group of samples' hidden vectors -> shared memory
+        if (!waited) { griddep_wait(); waited = true; }
+        __syncthreads();
+        for (int i = threadIdx.x; i < nb * R; i += 256) h_sm[(i / R) * kGenMaxR + i % R] = __ldcg(hidden + (size_t)b0 * R + i);
+        __syncthreads();
       }
 #pragma unroll
       for (int bb = 0; bb < 8; ++bb) {
-        if (b0 + bb < B) {
-          const float* hp = hidden + (size_t)(b0 + bb) * R;
+        if (bb < nb) {
+          const float* hp = h_sm + bb * kGenMaxR + r0;
+          if (kVec) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int r = r0 + part + 8 * i;
-            if (r < R) acc[bb] = fmaf(wv[i], __ldg(hp + r), acc[bb]);
+            for (int i = 0; i < kPer; ++i) {
+              const int r = 4 * part + 32 * i;
+              if (r0 + r < R) {
+                const float4 hv = *reinterpret_cast<const float4*>(hp + r);
+                acc[bb] = fmaf(wv[4 * i], hv.x, fmaf(wv[4 * i + 1], hv.y, fmaf(wv[4 * i + 2], hv.z, fmaf(wv[4 * i + 3], hv.w, acc[bb]))));
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) {
+              const int r = part + 8 * i;
+              if (r0 + r < R) acc[bb] = fmaf(wv[i], hp[r], acc[bb]);
+            }
           }
         }
       }
     }
+    if (R == 0 && !waited) { griddep_wait(); waited = true; }   // static kernels: nothing to read, but completion must chain
 #pragma unroll
     for (int bb = 0; bb < 8; ++bb) {
       float sres = acc[bb];
       sres += __shfl_xor_sync(0xffffffffu, sres, 1);
       sres += __shfl_xor_sync(0xffffffffu, sres, 2);
       sres += __shfl_xor_sync(0xffffffffu, sres, 4);
-      if (t_ok && part == 0 && b0 + bb < B) w[(size_t)(b0 + bb) * T + t] = sres + (b2 ? b2[t] : 0.f);
+      if (t_ok && part == 0 && bb < nb) w[(size_t)(b0 + bb) * T + t] = sres + (b2 ? b2[t] : 0.f);
     }
   }
-  // The convolution pass is launched behind this grid in plain stream order and adds into what the
-  // apply pass writes: this grid must not retire before the apply grid has.
-  griddep_wait();
-}
-
-// ---- host side ---------------------------------------------------------------------------
-bool make_map(CUtensorMap* m, const void* ptr, int BH, int N, int box_tok) {
-  EncodeFn enc = encode_fn();
-  if (!enc) return false;
-  const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)BH};
-  const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)N * kD * 2};
-  const cuuint32_t box[3] = {(cuuint32_t)kD, (cuuint32_t)box_tok, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// [BH, Hg, Wg, 64] bf16 as a 4-D tensor (channel, x, y, batch*head), no swizzle
-bool make_map_grid(CUtensorMap* m, const void* ptr, int BH, int Hg, int Wg, int box_x, int box_y) {
-  EncodeFn enc = encode_fn();
-  if (!enc) return false;
-  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)Wg, (cuuint64_t)Hg, (cuuint64_t)BH};
-  const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)Wg * kD * 2, (cuuint64_t)Hg * Wg * kD * 2};
-  const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)box_x, (cuuint32_t)box_y, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  // wait_first = 0: the convolution pass is launched behind this grid and adds into what the apply
+  // pass writes: this grid must not retire before the apply grid has.
+  if (!wait_first) griddep_wait();
 }
 
 }  // namespace
@@ -814,25 +690,26 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   if (!status) return cudaErrorUnknown;
 
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map(&mq, a.q, BH, N, kApplyTok) || !make_map(&mk, a.k, BH, N, kTileTok) ||
-      !make_map(&mv, a.v, BH, N, kTileTok) || !make_map(&mo, a.o, BH, N, 32))
+  if (!make_map_tokens(&mq, a.q, BH, N, kApplyTok) || !make_map_tokens(&mk, a.k, BH, N, kTileTok) ||
+      !make_map_tokens(&mv, a.v, BH, N, kTileTok) || !make_map_tokens(&mo, a.o, BH, N, 32))
     return cudaErrorInvalidValue;
 
-  static bool attr_done = false;   // > 48 KB of dynamic shared memory needs the opt-in, once per process
-  if (!attr_done) {
-    cudaError_t e;
-    if ((e = cudaFuncSetAttribute(lin_state_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStateSmem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(lin_state_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStateSmem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(lin_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApplySmem)) != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
+  cudaError_t e = smem_opt_in.run([] {
+    cudaError_t r;
+    if ((r = cudaFuncSetAttribute(lin_state_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStateSmem)) != cudaSuccess) return r;
+    if ((r = cudaFuncSetAttribute(lin_state_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStateSmem)) != cudaSuccess) return r;
+    return cudaFuncSetAttribute(lin_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kApplySmem);
+  });
+  if (e != cudaSuccess) return e;
+  const int num_sms = device_sm_count();
   dim3 g1(p.nchunk, BH);
   if (a.dwc)
     lin_state_kernel<true><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems);
   else
     lin_state_kernel<false><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems);
   count_launch();
-  cudaError_t e = cudaGetLastError();
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
 
   cudaLaunchAttribute attr[1];
@@ -846,23 +723,44 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   // the output layer at its very end, so that stream order still means "apply pass complete" for
   // the convolution pass that follows it.
   float* hidden = (float*)(ws + p.off_hidden);
+  const bool fused_conv = a.dwc && linear_conv_supported(a);
   if (a.dwc && a.dwc->R > 0) {      // R == 0: static kernels, the output layer just broadcasts b2
     const jv_dwc& d = *a.dwc;
     cudaLaunchConfig_t hcfg = {};
     hcfg.stream = st;
     hcfg.attrs = attr;
     hcfg.numAttrs = 1;
-    hcfg.gridDim = dim3(d.R, s.B);
-    hcfg.blockDim = dim3(128);
+    hcfg.gridDim = dim3(ceil_div(d.R, 8), s.B);
+    hcfg.blockDim = dim3(256);
     e = cudaLaunchKernelEx(&hcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
-                           p.nchunk, p.state_elems, 1.f / (float)N);
+                           p.nchunk, p.state_elems, 1.f / (float)N, fused_conv ? 1 : 0);
     count_launch();
     if (e != cudaSuccess) return e;
   }
 
+  if (fused_conv) {
+    // 3 x 3 kernels: state -> [hidden layer] -> output layer -> apply pass with the convolution fused in.
+    // Every grid behind the state pass is launched with programmatic serialisation and waits for its
+    // predecessor before it reads that one's output, so completion is transitive along the chain.
+    const jv_dwc& d = *a.dwc;
+    float* wk = (float*)(ws + p.off_kernel);
+    const int T = s.H * kD * d.k * d.k;
+    cudaLaunchConfig_t gcfg = {};
+    gcfg.stream = st;
+    gcfg.attrs = attr;
+    gcfg.numAttrs = 1;
+    gcfg.gridDim = dim3(ceil_div(T, 32));
+    gcfg.blockDim = dim3(256);
+    e = cudaLaunchKernelEx(&gcfg, (d.R % 4 == 0) ? gen_out_kernel<true> : gen_out_kernel<false>, (const float*)hidden, d.W2,
+                           d.b2, wk, (int)s.B, T, (int)d.R, 1);
+    count_launch();
+    if (e != cudaSuccess) return e;
+    return launch_linear_apply_conv(a, p, partial, wk, status, true, st);
+  }
+
   // apply pass: one wave of two CTAs per SM, spans of whole 128-token tiles; launched so that its
   // set-up overlaps the tail of the grid before it
-  int nspan = (2 * 148) / BH;
+  int nspan = (2 * num_sms) / BH;
   if (nspan < 1) nspan = 1;
   int span = ceil_div(ceil_div(N, nspan), kApplyTok) * kApplyTok;
   if (span < 4 * kApplyTok) span = 4 * kApplyTok;
@@ -891,35 +789,16 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     gcfg.numAttrs = 1;
     gcfg.gridDim = dim3(ceil_div(T, 32));
     gcfg.blockDim = dim3(256);
-    e = cudaLaunchKernelEx(&gcfg, gen_out_kernel, (const float*)hidden, d.W2, d.b2, wk, (int)s.B, T, (int)d.R);
+    e = cudaLaunchKernelEx(&gcfg, (d.R % 4 == 0) ? gen_out_kernel<true> : gen_out_kernel<false>, (const float*)hidden, d.W2,
+                           d.b2, wk, (int)s.B, T, (int)d.R, 0);
     count_launch();
     if (e != cudaSuccess) return e;
     const float* w = (const float*)(ws + p.off_kernel);
     const int run = 32;
     dim3 g4(ceil_div(ceil_div(N, run), 8), BH);
-    if (a.dwc->k == 3) {
-      CUtensorMap mvg, mos;
-      if (!make_map_grid(&mvg, a.v, BH, s.Hg, s.Wg, 18, 10) || !make_map_grid(&mos, a.o, BH, s.Hg, s.Wg, 16, 1))
-        return cudaErrorInvalidValue;
-      static bool dw_attr = false;
-      if (!dw_attr) {
-        if ((e = cudaFuncSetAttribute(dwc3_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDwSmem)) != cudaSuccess) return e;
-        dw_attr = true;
-      }
-      const int ncb = ceil_div(s.Wg, 16), npatch = ncb * ceil_div(s.Hg, 8);
-      const long long items = (long long)npatch * BH;
-      if (items > 0x7fffffffll) return cudaErrorInvalidValue;
-      const int grid = (int)(items < 2 * 148 ? items : 2 * 148);
-      cudaLaunchConfig_t dcfg = {};
-      dcfg.gridDim = dim3(grid);
-      dcfg.blockDim = dim3(kDwThreads);
-      dcfg.dynamicSmemBytes = kDwSmem;
-      dcfg.stream = st;
-      dcfg.attrs = attr;
-      dcfg.numAttrs = 1;
-      e = cudaLaunchKernelEx(&dcfg, dwc3_tma_kernel, mvg, mos, w, status, (int)s.H, (int)s.Hg, ncb, npatch, (int)items);
-      if (e != cudaSuccess) return e;
-    } else
+    // 5 x 5 kernels (3 x 3 ones took the fused path above): a read-modify-write pass over o
+    if (a.dwc->k == 3) dwc_add_kernel<3><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
+    else
       dwc_add_kernel<5><<<g4, 256, 0, st>>>(v, o, w, s.H, s.Hg, s.Wg, run);
     count_launch();
   }

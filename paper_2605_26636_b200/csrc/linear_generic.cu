@@ -18,7 +18,7 @@ LinPlan lin_plan(const jv_shape& s, const jv_dwc* dwc) {
   // Chunks: as many as fit one wave of two CTAs per SM over all (batch, head) pairs, each a
   // multiple of 128 tokens and at least 512 tokens long so that the partials stay small next
   // to K and V.  One wave means no tail, and chunks of equal length finish together.
-  int want = (2 * 148) / BH;
+  int want = (2 * device_sm_count()) / BH;
   if (want < 1) want = 1;
   int chunk = ceil_div(ceil_div(N, want), 128) * 128;
   if (chunk < 512) chunk = 512;

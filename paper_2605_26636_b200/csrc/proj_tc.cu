@@ -1,5 +1,5 @@
 // The linear projections either side of a token mixer (the inherited W_Q, W_K, W_V and W_O
-// of every block, Sec. 3.3) as tcgen05 GEMMs that read and write the mixers' [B, H, N, 64]
+// of every block, Sec. 3.2.4) as tcgen05 GEMMs that read and write the mixers' [B, H, N, 64]
 // layout directly, so that no transpose pass runs between the projection and the mixer.
 //
 //   qkv:  x [B, N, C] (C = H * 64)  times  w [3C, C]^T  ->  q, k, v [B, H, N, 64]
@@ -301,24 +301,15 @@ cudaError_t launch_proj_tc(bool qkv, const void* x, const void* w, const float* 
   }
   if (!ok) return cudaErrorInvalidValue;
 
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(proj_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(proj_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0) {
-      num_sms = 0;
-      cudaGetLastError();
-      return cudaErrorUnknown;
-    }
-  }
+  static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
+  cudaError_t e = smem_opt_in.run([] {
+    cudaError_t r = cudaFuncSetAttribute(proj_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (r == cudaSuccess)
+      r = cudaFuncSetAttribute(proj_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    return r;
+  });
+  if (e != cudaSuccess) return e;
+  const int num_sms = device_sm_count();
   ProjParams p;
   p.bias = bias;
   p.status = status;

@@ -63,8 +63,9 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false (after flagging the status word and the CTA abort flag)
-// if the phase did not complete in time or another role already aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status) {
+// if the phase did not complete within limit_ns or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t spin = 0;; ++spin) {
@@ -73,7 +74,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) {
+      else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicOr(status, kStatusTimeout);
         return false;
@@ -85,6 +86,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 // The same for a whole converged warp, with a warp-uniform outcome.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status) {
   return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+}
+__device__ __forceinline__ bool warp_wait_limit(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status,
+                                                unsigned long long limit_ns) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, limit_ns));
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {

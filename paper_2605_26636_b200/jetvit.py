@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
                                        ctypes.POINTER(vp), ctypes.POINTER(vp), shp, i32, i32, f32, f32,
                                        ctypes.POINTER(dwc), vp, sz, vp]
         L.jv_device_status.argtypes = [vp]
+        L.jv_selftest_wait_timeout.argtypes = [ctypes.c_uint32, vp, vp]
+        L.jv_selftest_wait_timeout.restype = ctypes.c_int
         L.jv_qkv_proj.argtypes = [vp, vp, vp, vp, vp, vp, shp, vp]
         L.jv_out_proj.argtypes = [vp, vp, vp, vp, shp, vp]
         for f in (L.jv_linear_attn, L.jv_window_attn, L.jv_full_attn, L.jv_hybrid_mixers, L.jv_device_status,
@@ -162,6 +164,8 @@ def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict
     with torch.cuda.device(q.device):
         if ws is None:
             ws = alloc_workspace("L", shape, d, q.device)
+            if ws is not None and stream is not None:
+                ws.record_stream(stream)      # freed by torch on the current stream, used on `stream`
         wp, wn = _ws_args(ws)
         st = lib().jv_linear_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
                                   float(eps), ctypes.byref(d) if d is not None else None, wp, wn, _stream(stream))
@@ -243,6 +247,8 @@ def hybrid_mixers(schedule: str, q: Sequence[torch.Tensor], k, v, Hg: int, Wg: i
                 if m == "L":
                     need = max(need, workspace_bytes("L", shape, dstructs[l] if dstructs else None))
             ws = torch.empty(max(need, 256), dtype=torch.uint8, device=q[0].device) if need else None
+            if ws is not None and stream is not None:
+                ws.record_stream(stream)      # freed by torch on the current stream, used on `stream`
         wp, wn = _ws_args(ws)
         st = lib().jv_hybrid_mixers(n, schedule.encode(), arr(q), arr(k), arr(v), arr(out), ctypes.byref(shape),
                                     int(win_h), int(win_w), float(scale), float(eps), dptr, wp, wn, _stream(stream))
@@ -298,6 +304,14 @@ def out_proj(o, w, bias, Hg: int, Wg: int, out=None, stream=None) -> torch.Tenso
                                ctypes.byref(shape), _stream(stream))
     _raise(st, "jv_out_proj")
     return y
+
+
+def selftest_wait_timeout(limit_us: int, gave_up: Optional[torch.Tensor] = None, stream=None) -> None:
+    """jv_selftest_wait_timeout: enqueues a kernel whose bounded wait runs out after ``limit_us``
+    microseconds and sets the sticky status word.  ``gave_up``: optional int32 CUDA tensor (1 element)."""
+    st = lib().jv_selftest_wait_timeout(int(limit_us), None if gave_up is None else gave_up.data_ptr(),
+                                        _stream(stream))
+    _raise(st, "jv_selftest_wait_timeout")
 
 
 def device_status(stream=None) -> int:

@@ -50,7 +50,11 @@ def test_workspace_bytes_host_logic(L):
     assert jv.workspace_bytes("X", shp) == 0
 
 
-def _call_linear(L, shp, q=256, k=512, v=768, o=1024, eps=1e-6, dwc=None, ws=4096, ws_bytes=1 << 40):
+# fake device addresses, spaced further apart than any tensor of the shapes used here
+FQ, FK, FV, FO, FWS = 1 << 20, 2 << 20, 3 << 20, 4 << 20, 5 << 20
+
+
+def _call_linear(L, shp, q=FQ, k=FK, v=FV, o=FO, eps=1e-6, dwc=None, ws=FWS, ws_bytes=1 << 40):
     return L.jv_linear_attn(q, k, v, o, ctypes.byref(shp), eps, dwc, ws, ws_bytes, None)
 
 
@@ -59,15 +63,20 @@ def test_argument_errors_are_found_before_any_launch(L):
     argument error, which it can only do if validation precedes the launch."""
     shp = jv.JvShape(1, 2, 8, 8, 64, jv.JV_F32)
     assert _call_linear(L, shp, q=None) == jv.JV_ERR_INVALID_ARG
-    assert _call_linear(L, shp, q=260) == jv.JV_ERR_INVALID_ARG            # misaligned
-    assert _call_linear(L, shp, o=256) == jv.JV_ERR_INVALID_ARG            # o aliases q
+    assert _call_linear(L, shp, q=FQ + 4) == jv.JV_ERR_INVALID_ARG         # misaligned
+    assert _call_linear(L, shp, o=FQ) == jv.JV_ERR_INVALID_ARG             # o aliases q
+    nbytes = 1 * 2 * 8 * 8 * 64 * 4
+    assert _call_linear(L, shp, o=FV + nbytes - 16) == jv.JV_ERR_INVALID_ARG   # o overlaps the tail of v
+    assert _call_linear(L, shp, o=FK - nbytes + 16) == jv.JV_ERR_INVALID_ARG   # the tail of o overlaps k
+    if not torch.cuda.is_available():   # o right behind v, sharing no byte, passes validation
+        assert _call_linear(L, shp, o=FV + nbytes) in (jv.JV_ERR_CUDA, jv.JV_ERR_UNSUPPORTED)
     assert _call_linear(L, shp, eps=-1.0) == jv.JV_ERR_INVALID_ARG
     assert _call_linear(L, shp, ws=None) == jv.JV_ERR_WORKSPACE
-    assert _call_linear(L, shp, ws=4100) == jv.JV_ERR_WORKSPACE            # misaligned workspace
+    assert _call_linear(L, shp, ws=FWS + 4) == jv.JV_ERR_WORKSPACE            # misaligned workspace
     assert _call_linear(L, shp, ws_bytes=16) == jv.JV_ERR_WORKSPACE
     bad = jv.JvDwc(4, 8, 1, None, 1, None)
     assert _call_linear(L, shp, dwc=ctypes.byref(bad)) == jv.JV_ERR_INVALID_ARG
-    static_ok = jv.JvDwc(3, 0, None, None, None, 4096)          # R = 0: static kernels in b2
+    static_ok = jv.JvDwc(3, 0, None, None, None, 6 << 20)          # R = 0: static kernels in b2
     static_bad = jv.JvDwc(3, 0, None, None, None, None)
     assert _call_linear(L, shp, dwc=ctypes.byref(static_bad)) == jv.JV_ERR_INVALID_ARG
     if not torch.cuda.is_available():   # with fake addresses a call that passes validation may only run where nothing can launch
@@ -76,17 +85,17 @@ def test_argument_errors_are_found_before_any_launch(L):
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 0, jv.JV_F32)) == jv.JV_ERR_INVALID_ARG
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 512, jv.JV_F32)) == jv.JV_ERR_UNSUPPORTED
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 30, jv.JV_BF16)) == jv.JV_ERR_UNSUPPORTED
-    assert L.jv_window_attn(256, 512, 768, 1024, ctypes.byref(shp), 0, 4, 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
-    assert L.jv_full_attn(256, 512, 768, None, ctypes.byref(shp), 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
-    assert L.jv_full_attn(256, 512, 768, 1024, None, 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
+    assert L.jv_window_attn(FQ, FK, FV, FO, ctypes.byref(shp), 0, 4, 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
+    assert L.jv_full_attn(FQ, FK, FV, None, ctypes.byref(shp), 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
+    assert L.jv_full_attn(FQ, FK, FV, FO, None, 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
 
 
 def test_hybrid_schedule_is_validated_before_any_launch(L):
     shp = jv.JvShape(1, 2, 8, 8, 64, jv.JV_F32)
     n = 3
-    arr = lambda base: (ctypes.c_void_p * n)(*[base + 4096 * i for i in range(n)])
+    arr = lambda base: (ctypes.c_void_p * n)(*[base + (64 << 10) * i for i in range(n)])
     q, k, v, o = arr(1 << 20), arr(2 << 20), arr(3 << 20), arr(4 << 20)
-    call = lambda sched, nl=n, ws=4096, wsb=1 << 40: L.jv_hybrid_mixers(
+    call = lambda sched, nl=n, ws=8 << 20, wsb=1 << 40: L.jv_hybrid_mixers(
         nl, sched, q, k, v, o, ctypes.byref(shp), 4, 4, 0.0, 1e-6, None, ws, wsb, None)
     assert call(b"LWX") == jv.JV_ERR_INVALID_ARG
     assert call(b"LW") == jv.JV_ERR_INVALID_ARG          # shorter than n_layers
@@ -99,7 +108,7 @@ def test_hybrid_schedule_is_validated_before_any_launch(L):
 def test_no_device_means_an_error_not_a_fallback(L):
     shp = jv.JvShape(1, 2, 8, 8, 64, jv.JV_F32)
     assert _call_linear(L, shp) in (jv.JV_ERR_CUDA, jv.JV_ERR_UNSUPPORTED)
-    assert L.jv_full_attn(256, 512, 768, 1024, ctypes.byref(shp), 0.0, None, 0, None) in (
+    assert L.jv_full_attn(FQ, FK, FV, FO, ctypes.byref(shp), 0.0, None, 0, None) in (
         jv.JV_ERR_CUDA, jv.JV_ERR_UNSUPPORTED)
     with pytest.raises(ValueError):
         t = torch.zeros(1, 2, 64, 64)

@@ -1,4 +1,4 @@
-"""The projections either side of a mixer (W_Q | W_K | W_V before it, W_O after it; Sec. 3.3:
+"""The projections either side of a mixer (W_Q | W_K | W_V before it, W_O after it; Sec. 3.2.4:
 the linear layers every block inherits).  CPU tests pin the oracle's two functions to things
 other than themselves; GPU tests compare jv_qkv_proj / jv_out_proj with the oracle element by
 element on the same seeded inputs (bf16 tensors, fp32 accumulation: 2e-2 of the output rms)."""
@@ -159,8 +159,8 @@ def test_projection_mixer_projection_at_full_size(jv, oracle):
 def test_projection_argument_errors(jv):
     L = jv.lib()
     good = jv.JvShape(1, 2, 4, 4, 64, jv.JV_BF16)
-    t = torch.zeros(1 << 16, dtype=torch.bfloat16, device=DEV)
-    p = [t.data_ptr() + 8192 * i for i in range(6)]
+    t = torch.zeros(1 << 19, dtype=torch.bfloat16, device=DEV)
+    p = [t.data_ptr() + (128 << 10) * i for i in range(6)]       # further apart than any operand here (w: 96 KB)
     call = lambda shp, ptrs=p, bias=None: L.jv_qkv_proj(ptrs[0], ptrs[1], bias, ptrs[2], ptrs[3], ptrs[4],
                                                        ctypes.byref(shp), None)
     assert call(jv.JvShape(1, 2, 4, 4, 64, jv.JV_F32)) == jv.JV_ERR_UNSUPPORTED
@@ -168,6 +168,7 @@ def test_projection_argument_errors(jv):
     assert call(jv.JvShape(0, 2, 4, 4, 64, jv.JV_BF16)) == jv.JV_ERR_INVALID_ARG
     assert call(good, [p[0], p[1], p[2], p[2], p[4]]) == jv.JV_ERR_INVALID_ARG      # k aliases q
     assert call(good, [p[0], p[1], p[0], p[3], p[4]]) == jv.JV_ERR_INVALID_ARG      # q aliases x
+    assert call(good, [p[0], p[1], p[2], p[2] + 4096 - 16, p[4]]) == jv.JV_ERR_INVALID_ARG   # k overlaps the tail of q
     assert call(good, [p[0] + 2, p[1], p[2], p[3], p[4]]) == jv.JV_ERR_INVALID_ARG  # misaligned
     assert call(good, bias=p[5] + 4) == jv.JV_ERR_INVALID_ARG
     assert L.jv_out_proj(p[0], p[1], None, None, ctypes.byref(good), None) == jv.JV_ERR_INVALID_ARG
