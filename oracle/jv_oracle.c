@@ -248,3 +248,168 @@ void jvo_linear_attn(const double* q, const double* k, const double* v, double* 
   }
   free(wall);
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Prefix tokens beside the grid.
+ *
+ * The backbones the method converts (Sec. 4.1: DINOv3, DepthAnythingV2) carry a class token
+ * and register tokens in front of the patch tokens.  The paper defines its window partition
+ * (Sec. 3.2.2) and the convolution on V (Sec. 3.2.1, Eq. 4) on the feature map only and is
+ * silent about these tokens; the reading taken here:
+ *   - a sequence is P prefix tokens followed by the N = Hg*Wg grid tokens (row-major grid);
+ *   - F (Eq. 1) and the linear attention proper (Eq. 2) are global: all P + N tokens are
+ *     queries and keys (both are indifferent to where a token sits);
+ *   - W (Sec. 3.2.2): a grid token attends the tokens of its window and the P prefix tokens;
+ *     a prefix token attends all P + N tokens;
+ *   - the depth-wise convolution and the average pooling that feeds its kernel generator see
+ *     the feature map only: prefix rows of V are neither pooled nor convolved, and a prefix
+ *     token's output is its linear-attention output alone.
+ * With P = 0 each function below performs exactly the operations of its counterpart above,
+ * in the same order.
+ * ------------------------------------------------------------------------------------------ */
+
+/* q, k, v, o: [BH][P + Hg*Wg][D]. */
+void jvo_window_attn_prefix(const double* q, const double* k, const double* v, double* o,
+                            int64_t BH, int64_t P, int64_t Hg, int64_t Wg, int64_t D,
+                            int64_t wh, int64_t ww, double scale) {
+  const int64_t N = Hg * Wg, T = P + N;
+#pragma omp parallel
+  {
+    double* s = (double*)malloc(sizeof(double) * (size_t)T);
+    int64_t* idx = (int64_t*)malloc(sizeof(int64_t) * (size_t)T);
+#pragma omp for collapse(2) schedule(dynamic, 16)
+    for (int64_t g = 0; g < BH; ++g) {
+      for (int64_t i = 0; i < T; ++i) {
+        /* the keys token i attends, as token indices */
+        int64_t nk = 0;
+        if (i < P) {
+          for (int64_t j = 0; j < T; ++j) idx[nk++] = j;
+        } else {
+          const int64_t y = (i - P) / Wg, x = (i - P) % Wg;
+          const int64_t y0 = (y / wh) * wh, x0 = (x / ww) * ww;
+          const int64_t y1 = (y0 + wh < Hg) ? y0 + wh : Hg;
+          const int64_t x1 = (x0 + ww < Wg) ? x0 + ww : Wg;
+          for (int64_t j = 0; j < P; ++j) idx[nk++] = j;
+          for (int64_t yy = y0; yy < y1; ++yy)
+            for (int64_t xx = x0; xx < x1; ++xx) idx[nk++] = P + yy * Wg + xx;
+        }
+        const double* qi = q + (g * T + i) * D;
+        double* oi = o + (g * T + i) * D;
+        double m = -INFINITY;
+        for (int64_t c = 0; c < nk; ++c) {
+          const double* kj = k + (g * T + idx[c]) * D;
+          double dot = 0.0;
+          for (int64_t e = 0; e < D; ++e) dot += qi[e] * kj[e];
+          s[c] = dot * scale;
+          if (s[c] > m) m = s[c];
+        }
+        double denom = 0.0;
+        for (int64_t e = 0; e < D; ++e) oi[e] = 0.0;
+        for (int64_t c = 0; c < nk; ++c) {
+          const double* vj = v + (g * T + idx[c]) * D;
+          double p = exp(s[c] - m);
+          denom += p;
+          for (int64_t e = 0; e < D; ++e) oi[e] += p * vj[e];
+        }
+        for (int64_t e = 0; e < D; ++e) oi[e] /= denom;
+      }
+    }
+    free(s);
+    free(idx);
+  }
+}
+
+/* Kernel generator with prefix tokens: the average pooling runs over the N grid tokens only.
+ * v: [B*H][P + N][D]; w: [B][C*k*k]. */
+void jvo_dwc_generate_prefix(const double* v, double* w, int64_t B, int64_t H, int64_t P, int64_t N,
+                             int64_t D, int64_t dwc_k, int64_t R, const double* W1, const double* b1,
+                             const double* W2, const double* b2) {
+  const int64_t C = H * D, kk = dwc_k * dwc_k, T = P + N;
+  for (int64_t b = 0; b < B; ++b) {
+    double* s = (double*)calloc((size_t)C, sizeof(double));
+    double* hid = (double*)calloc((size_t)(R > 0 ? R : 1), sizeof(double));
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t e = 0; e < D; ++e) {
+        const double* vg = v + ((b * H + h) * T + P) * D;   /* first grid token */
+        double acc = 0.0;
+        for (int64_t j = 0; j < N; ++j) acc += vg[j * D + e];
+        s[h * D + e] = acc / (double)N;
+      }
+    for (int64_t r = 0; r < R; ++r) {
+      double acc = b1 ? b1[r] : 0.0;
+      for (int64_t c = 0; c < C; ++c) acc += W1[r * C + c] * s[c];
+      hid[r] = silu(acc);
+    }
+    for (int64_t t = 0; t < C * kk; ++t) {
+      double acc = b2 ? b2[t] : 0.0;
+      for (int64_t r = 0; r < R; ++r) acc += W2[t * R + r] * hid[r];
+      w[b * C * kk + t] = acc;
+    }
+    free(s);
+    free(hid);
+  }
+}
+
+/* q, k, v, o: [B*H][P + Hg*Wg][D]. */
+void jvo_linear_attn_prefix(const double* q, const double* k, const double* v, double* o,
+                            int64_t B, int64_t H, int64_t P, int64_t Hg, int64_t Wg, int64_t D, double eps,
+                            int64_t dwc_k, int64_t R, const double* W1, const double* b1,
+                            const double* W2, const double* b2) {
+  const int64_t N = Hg * Wg, T = P + N, C = H * D;
+
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t g = 0; g < B * H; ++g) {
+    const double* qg = q + g * T * D;
+    const double* kg = k + g * T * D;
+    const double* vg = v + g * T * D;
+    double* og = o + g * T * D;
+    double* KV = (double*)calloc((size_t)(D * D), sizeof(double));
+    double* z = (double*)calloc((size_t)D, sizeof(double));
+    for (int64_t j = 0; j < T; ++j)          /* prefix and grid tokens alike */
+      for (int64_t a = 0; a < D; ++a) {
+        double pk = kg[j * D + a] > 0.0 ? kg[j * D + a] : 0.0;
+        z[a] += pk;
+        for (int64_t e = 0; e < D; ++e) KV[a * D + e] += pk * vg[j * D + e];
+      }
+    for (int64_t i = 0; i < T; ++i) {
+      double denom = eps;
+      for (int64_t e = 0; e < D; ++e) og[i * D + e] = 0.0;
+      for (int64_t a = 0; a < D; ++a) {
+        double pq = qg[i * D + a] > 0.0 ? qg[i * D + a] : 0.0;
+        denom += pq * z[a];
+        for (int64_t e = 0; e < D; ++e) og[i * D + e] += pq * KV[a * D + e];
+      }
+      for (int64_t e = 0; e < D; ++e) og[i * D + e] /= denom;
+    }
+    free(KV);
+    free(z);
+  }
+
+  if (dwc_k <= 0) return;
+
+  const int64_t kk = dwc_k * dwc_k, p = (dwc_k - 1) / 2;
+  double* wall = (double*)calloc((size_t)(B * C * kk), sizeof(double));
+  jvo_dwc_generate_prefix(v, wall, B, H, P, N, D, dwc_k, R, W1, b1, W2, b2);
+  for (int64_t b = 0; b < B; ++b) {
+    const double* w = wall + b * C * kk;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t h = 0; h < H; ++h)
+      for (int64_t y = 0; y < Hg; ++y) {
+        const double* vg = v + ((b * H + h) * T + P) * D;   /* the grid part of V */
+        double* og = o + ((b * H + h) * T + P) * D;
+        for (int64_t x = 0; x < Wg; ++x)
+          for (int64_t e = 0; e < D; ++e) {
+            const double* wc = w + (h * D + e) * kk;
+            double acc = 0.0;
+            for (int64_t dy = 0; dy < dwc_k; ++dy)
+              for (int64_t dx = 0; dx < dwc_k; ++dx) {
+                int64_t yy = y + dy - p, xx = x + dx - p;
+                if (yy < 0 || yy >= Hg || xx < 0 || xx >= Wg) continue;
+                acc += wc[dy * dwc_k + dx] * vg[(yy * Wg + xx) * D + e];
+              }
+            og[(y * Wg + x) * D + e] += acc;
+          }
+      }
+  }
+  free(wall);
+}

@@ -44,8 +44,13 @@ def _load():
         lib.jvo_dwc_generate.argtypes = [_c_dp] * 2 + [_i64] * 6 + [_c_dp] * 4
         lib.jvo_linear_attn.argtypes = ([_c_dp] * 4 + [_i64] * 5 + [ctypes.c_double]
                                         + [_i64] * 2 + [_c_dp] * 4)
+        lib.jvo_window_attn_prefix.argtypes = [_c_dp] * 4 + [_i64] * 7 + [ctypes.c_double]
+        lib.jvo_dwc_generate_prefix.argtypes = [_c_dp] * 2 + [_i64] * 7 + [_c_dp] * 4
+        lib.jvo_linear_attn_prefix.argtypes = ([_c_dp] * 4 + [_i64] * 6 + [ctypes.c_double]
+                                               + [_i64] * 2 + [_c_dp] * 4)
         for f in (lib.jvo_full_attn, lib.jvo_window_attn, lib.jvo_dwc_generate,
-                  lib.jvo_linear_attn):
+                  lib.jvo_linear_attn, lib.jvo_window_attn_prefix, lib.jvo_dwc_generate_prefix,
+                  lib.jvo_linear_attn_prefix):
             f.restype = None
         _lib = lib
     return _lib
@@ -79,23 +84,30 @@ def full_attn(q, k, v, scale=None) -> np.ndarray:
     return o
 
 
-def window_attn(q, k, v, Hg, Wg, win_h, win_w, scale=None) -> np.ndarray:
-    """Sec. 3.2.2 window attention.  q, k, v: [B,H,Hg*Wg,D]."""
+def window_attn(q, k, v, Hg, Wg, win_h, win_w, scale=None, prefix=0, _force_prefix_code=False) -> np.ndarray:
+    """Sec. 3.2.2 window attention.  q, k, v: [B,H,prefix + Hg*Wg,D]; ``prefix`` tokens in
+    front of the grid tokens attend, and are attended by, everything (see jv_oracle.c)."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, H, N, D = q.shape
-    assert N == Hg * Wg and k.shape == q.shape and v.shape == q.shape
+    assert N == prefix + Hg * Wg and k.shape == q.shape and v.shape == q.shape
     if scale is None or scale <= 0:
         scale = 1.0 / np.sqrt(D)
     o = np.empty_like(q)
-    _load().jvo_window_attn(_p(q), _p(k), _p(v), _p(o), B * H, Hg, Wg, D,
-                            win_h, win_w, float(scale))
+    if prefix == 0 and not _force_prefix_code:
+        _load().jvo_window_attn(_p(q), _p(k), _p(v), _p(o), B * H, Hg, Wg, D,
+                                win_h, win_w, float(scale))
+    else:
+        _load().jvo_window_attn_prefix(_p(q), _p(k), _p(v), _p(o), B * H, prefix, Hg, Wg, D,
+                                       win_h, win_w, float(scale))
     return o
 
 
-def dwc_generate(v, dwc) -> np.ndarray:
-    """Dynamic depth-wise kernels [B, C, k, k] from V [B,H,N,D] (Sec. 3.2.1)."""
+def dwc_generate(v, dwc, prefix=0, _force_prefix_code=False) -> np.ndarray:
+    """Dynamic depth-wise kernels [B, C, k, k] from V [B,H,prefix + N,D] (Sec. 3.2.1); the
+    pooling runs over the N grid tokens only."""
     v = _f64(v)
     B, H, N, D = v.shape
+    N -= prefix
     kk, R = int(dwc["k"]), int(dwc["R"])
     W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
     b1 = None if dwc.get("b1") is None else _f64(dwc["b1"])
@@ -103,20 +115,34 @@ def dwc_generate(v, dwc) -> np.ndarray:
     C = H * D
     assert W1.shape == (R, C) and W2.shape == (C * kk * kk, R)
     w = np.empty((B, C, kk, kk), dtype=np.float64)
-    _load().jvo_dwc_generate(_p(v), _p(w), B, H, N, D, kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+    if prefix == 0 and not _force_prefix_code:
+        _load().jvo_dwc_generate(_p(v), _p(w), B, H, N, D, kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+    else:
+        _load().jvo_dwc_generate_prefix(_p(v), _p(w), B, H, prefix, N, D, kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
     return w
 
 
-def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None) -> np.ndarray:
+def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None, prefix=0, _force_prefix_code=False) -> np.ndarray:
     """JetViT linear-attention block (Eqs. 2, 4).  ``dwc``: None or a dict with
-    keys k, R, W1 [R,C], b1 [R] or None, W2 [C*k*k,R], b2 [C*k*k] or None."""
+    keys k, R, W1 [R,C], b1 [R] or None, W2 [C*k*k,R], b2 [C*k*k] or None.
+    q, k, v: [B,H,prefix + Hg*Wg,D]; prefix tokens take part in the attention, not in the
+    convolution or its pooling (see jv_oracle.c)."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, H, N, D = q.shape
-    assert N == Hg * Wg and k.shape == q.shape and v.shape == q.shape
+    assert N == prefix + Hg * Wg and k.shape == q.shape and v.shape == q.shape
     o = np.empty_like(q)
+    old = prefix == 0 and not _force_prefix_code
+
+    def call(kk, R, W1, b1, W2, b2):
+        if old:
+            _load().jvo_linear_attn(_p(q), _p(k), _p(v), _p(o), B, H, Hg, Wg, D, float(eps),
+                                    kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+        else:
+            _load().jvo_linear_attn_prefix(_p(q), _p(k), _p(v), _p(o), B, H, prefix, Hg, Wg, D, float(eps),
+                                           kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+
     if dwc is None:
-        _load().jvo_linear_attn(_p(q), _p(k), _p(v), _p(o), B, H, Hg, Wg, D, float(eps),
-                                0, 0, None, None, None, None)
+        call(0, 0, None, None, None, None)
         return o
     kk, R = int(dwc["k"]), int(dwc["R"])
     C = H * D
@@ -129,22 +155,21 @@ def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None) -> np.ndarray:
         W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
         assert W1.shape == (R, C) and W2.shape == (C * kk * kk, R)
     assert kk % 2 == 1
-    _load().jvo_linear_attn(_p(q), _p(k), _p(v), _p(o), B, H, Hg, Wg, D, float(eps),
-                            kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
+    call(kk, R, W1, b1, W2, b2)
     return o
 
 
-def hybrid_mixers(schedule, q, k, v, Hg, Wg, win_h, win_w, scale=None, eps=1e-6, dwc=None):
+def hybrid_mixers(schedule, q, k, v, Hg, Wg, win_h, win_w, scale=None, eps=1e-6, dwc=None, prefix=0):
     """Per-layer L/W/F schedule over a stack of independent layers.
-    q, k, v: sequences of [B,H,N,D] arrays, one per layer; dwc: None or a
+    q, k, v: sequences of [B,H,prefix + N,D] arrays, one per layer; dwc: None or a
     per-layer sequence whose entries may be None."""
     out = []
     for l, m in enumerate(schedule):
         if m == "L":
             out.append(linear_attn(q[l], k[l], v[l], Hg, Wg, eps,
-                                   None if dwc is None else dwc[l]))
+                                   None if dwc is None else dwc[l], prefix=prefix))
         elif m == "W":
-            out.append(window_attn(q[l], k[l], v[l], Hg, Wg, win_h, win_w, scale))
+            out.append(window_attn(q[l], k[l], v[l], Hg, Wg, win_h, win_w, scale, prefix=prefix))
         elif m == "F":
             out.append(full_attn(q[l], k[l], v[l], scale))
         else:

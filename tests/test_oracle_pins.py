@@ -426,3 +426,119 @@ def test_bf16_store_floor(oracle):
     rms = np.sqrt(np.mean(ref * ref))
     assert np.abs(stored - ref).max() / rms > 2e-2
     assert np.all(np.abs(stored - ref) <= 2.0 ** -8 * np.abs(ref) * (1 + 1e-6))
+
+
+# ------------------------------------------------------------------ prefix tokens beside the grid
+
+
+def test_prefix_golden_2x2(oracle):
+    g = _golden("prefix_2x2.txt")
+    t = lambda key: g[key].reshape(1, 1, 5, 1)
+    o = oracle.window_attn(t("w_q"), t("w_k"), t("w_v"), 2, 2, 1, 1, scale=1.0, prefix=1)
+    assert np.allclose(o.ravel(), g["w_o_1x1"], atol=1e-14)
+    o = oracle.window_attn(t("w_q"), t("w_k"), t("w_v"), 2, 2, 2, 2, scale=1.0, prefix=1)
+    assert np.allclose(o.ravel(), g["w_o_2x2"], atol=1e-14)
+    static = {"k": 3, "R": 0, "b2": np.ones(9)}
+    o = oracle.linear_attn(t("l_q"), t("l_k"), t("l_v"), 2, 2, eps=float(g["l_eps"][0]), dwc=static, prefix=1)
+    assert np.allclose(o.ravel(), g["l_o"], atol=1e-13)
+    gen = {"k": 3, "R": 1, "W1": np.ones((1, 1)), "b1": None, "W2": np.ones((9, 1)), "b2": None}
+    w = oracle.dwc_generate(t("l_v"), gen, prefix=1)
+    assert np.allclose(w.ravel(), g["gen_w"][0], atol=1e-14)
+
+
+@pytest.mark.parametrize("case", [(1, 2, 7, 5, 8, 4, 4), (2, 1, 9, 9, 16, 3, 5), (1, 1, 4, 6, 8, 2, 3)])
+def test_prefix_zero_is_the_plain_function_bit_for_bit(oracle, case):
+    """With no prefix tokens the prefix-aware code performs the same operations in the same order."""
+    B, H, Hg, Wg, D, wh, ww = case
+    r = _rng(900 + Hg)
+    q, k, v = (r.standard_normal((B, H, Hg * Wg, D)) for _ in range(3))
+    C = H * D
+    d = {"k": 3, "R": 4, "W1": r.standard_normal((4, C)), "b1": r.standard_normal(4),
+         "W2": r.standard_normal((C * 9, 4)), "b2": r.standard_normal(C * 9)}
+    assert np.array_equal(oracle.window_attn(q, k, v, Hg, Wg, wh, ww),
+                          oracle.window_attn(q, k, v, Hg, Wg, wh, ww, _force_prefix_code=True))
+    assert np.array_equal(oracle.linear_attn(q, k, v, Hg, Wg, dwc=d),
+                          oracle.linear_attn(q, k, v, Hg, Wg, dwc=d, _force_prefix_code=True))
+    assert np.array_equal(oracle.linear_attn(q, k, v, Hg, Wg), oracle.linear_attn(q, k, v, Hg, Wg, _force_prefix_code=True))
+    assert np.array_equal(oracle.dwc_generate(v, d), oracle.dwc_generate(v, d, _force_prefix_code=True))
+
+
+@pytest.mark.parametrize("P", [1, 5])
+def test_prefix_window_is_block_masked_full_attention(oracle, P):
+    """W with prefix tokens == Eq. 1 under the explicit mask "same window, or either token is a
+    prefix token ... for a prefix query" written as matrix algebra; ragged grid (7 x 5, 4 x 4 windows)."""
+    Hg, Wg, D, wh, ww = 7, 5, 8, 4, 4
+    r = _rng(910 + P)
+    q, k, v = (r.standard_normal((1, 2, P + Hg * Wg, D)) for _ in range(3))
+    N = Hg * Wg
+    ys, xs = np.divmod(np.arange(N), Wg)
+    same = ((ys // wh)[:, None] == (ys // wh)[None, :]) & ((xs // ww)[:, None] == (xs // ww)[None, :])
+    M = np.ones((P + N, P + N), dtype=bool)
+    M[P:, P:] = same                     # grid query x grid key: same window; everything else attends
+    got = oracle.window_attn(q, k, v, Hg, Wg, wh, ww, prefix=P)
+    for h in range(2):
+        want = _softmax_bruteforce(q[0, h], k[0, h], v[0, h], 1.0 / np.sqrt(D), M)
+        assert np.abs(got[0, h] - want).max() < TOL
+
+
+def test_prefix_one_window_over_the_grid_is_full_attention(oracle):
+    """A window at least as large as the grid: every token attends all P + N tokens (Eq. 1)."""
+    P, Hg, Wg, D = 3, 5, 6, 8
+    r = _rng(920)
+    q, k, v = (r.standard_normal((2, 2, P + Hg * Wg, D)) for _ in range(3))
+    assert np.abs(oracle.window_attn(q, k, v, Hg, Wg, 8, 8, prefix=P) - oracle.full_attn(q, k, v)).max() < TOL
+
+
+def test_prefix_linear_core_does_not_care_where_a_token_sits(oracle):
+    """Without the convolution the linear block is global: P prefix tokens in front of an Hg x Wg
+    grid is the same as a 1 x (P + N) grid, and equals the naive O(N^2) form over all tokens."""
+    P, Hg, Wg, D = 5, 6, 7, 8
+    r = _rng(930)
+    q, k, v = (r.standard_normal((1, 2, P + Hg * Wg, D)) for _ in range(3))
+    got = oracle.linear_attn(q, k, v, Hg, Wg, eps=0.5, prefix=P)
+    assert np.abs(got - oracle.linear_attn(q, k, v, 1, P + Hg * Wg, eps=0.5)).max() < TOL
+    for h in range(2):
+        a, b = np.maximum(q[0, h], 0), np.maximum(k[0, h], 0)
+        S = a @ b.T
+        want = (S @ v[0, h]) / (S.sum(axis=1, keepdims=True) + 0.5)
+        assert np.abs(got[0, h] - want).max() < TOL
+
+
+@pytest.mark.parametrize("ksz", [3, 5])
+def test_prefix_convolution_and_pooling_see_the_grid_only(oracle, ksz):
+    """O = LA(all tokens) + conv2d(V_grid) on grid rows, LA alone on prefix rows; the library
+    depth-wise conv2d (float64) supplies the convolution, the generator is checked through
+    adaptive_avg_pool2d + linear + silu on the grid part; changing the prefix rows of V by a huge
+    amount changes neither the kernels nor the convolution term."""
+    P, B, H, Hg, Wg, D, R = 4, 2, 2, 6, 5, 4, 3
+    C, N = H * D, Hg * Wg
+    r = _rng(940 + ksz)
+    q, k, v = (r.standard_normal((B, H, P + N, D)) for _ in range(3))
+    d = {"k": ksz, "R": R, "W1": r.standard_normal((R, C)), "b1": r.standard_normal(R),
+         "W2": r.standard_normal((C * ksz * ksz, R)), "b2": r.standard_normal(C * ksz * ksz)}
+    w = oracle.dwc_generate(v, d, prefix=P)
+    img = torch.from_numpy(v[:, :, P:, :]).permute(0, 1, 3, 2).reshape(B, C, Hg, Wg)     # channel c = h*D + e
+    s = torch.nn.functional.adaptive_avg_pool2d(img, 1).reshape(B, C)
+    hid = torch.nn.functional.silu(torch.nn.functional.linear(s, torch.from_numpy(d["W1"]), torch.from_numpy(d["b1"])))
+    w_lib = torch.nn.functional.linear(hid, torch.from_numpy(d["W2"]), torch.from_numpy(d["b2"])).reshape(B, C, ksz, ksz)
+    assert np.abs(w - w_lib.numpy()).max() < 1e-11
+    v2 = v.copy()
+    v2[:, :, :P, :] += 1e6
+    assert np.array_equal(oracle.dwc_generate(v2, d, prefix=P), w)
+    got = oracle.linear_attn(q, k, v, Hg, Wg, dwc=d, prefix=P)
+    la = oracle.linear_attn(q, k, v, Hg, Wg, prefix=P)
+    conv = torch.cat([torch.nn.functional.conv2d(img[b:b + 1], w_lib[b].reshape(C, 1, ksz, ksz), padding=ksz // 2, groups=C)
+                      for b in range(B)])                                                   # [B, C, Hg, Wg]
+    conv = conv.reshape(B, H, D, N).permute(0, 1, 3, 2).numpy()
+    assert np.abs(got[:, :, P:] - (la[:, :, P:] + conv)).max() < 1e-10
+    assert np.array_equal(got[:, :, :P], la[:, :, :P])
+
+
+def test_prefix_hybrid_schedule_layers_are_independent(oracle):
+    P, Hg, Wg, D = 2, 4, 4, 8
+    r = _rng(950)
+    qs, ks, vs = ([r.standard_normal((1, 1, P + Hg * Wg, D)) for _ in range(3)] for _ in range(3))
+    outs = oracle.hybrid_mixers("LWF", qs, ks, vs, Hg, Wg, 2, 2, prefix=P)
+    assert np.array_equal(outs[0], oracle.linear_attn(qs[0], ks[0], vs[0], Hg, Wg, prefix=P))
+    assert np.array_equal(outs[1], oracle.window_attn(qs[1], ks[1], vs[1], Hg, Wg, 2, 2, prefix=P))
+    assert np.array_equal(outs[2], oracle.full_attn(qs[2], ks[2], vs[2]))
