@@ -13,7 +13,8 @@
  *
  * Conventions shared by every call
  *   Tensors   q, k, v, o are DEVICE pointers to [B, H, N, D] contiguous arrays,
- *             D fastest, N = Hg * Wg, token t at grid position (t / Wg, t % Wg).
+ *             D fastest, N = P + Hg * Wg: P prefix tokens (jv_shape.P, usually 0), then
+ *             grid token t at grid position (t / Wg, t % Wg).
  *             All four have the element type jv_shape.dtype; o must not share a
  *             byte with an input.  Pointers must be 16-byte aligned.
  *   Ownership The caller owns every buffer and the stream.  The library never
@@ -63,10 +64,22 @@ typedef enum {
 
 typedef enum { JV_F32 = 0, JV_BF16 = 1 } jv_dtype;
 
-/* Problem shape.  N = Hg * Wg tokens per (batch, head). */
+/*
+ * Problem shape.  A (batch, head) holds P prefix tokens followed by the Hg * Wg grid tokens:
+ * N = P + Hg * Wg rows of D elements.  P = 0 is the plain feature map.
+ *
+ * Prefix tokens are the class / register tokens that the base models of the paper (Sec. 4.1)
+ * carry in front of their patch tokens.  The paper defines its window partition (Sec. 3.2.2) and
+ * the convolution on V (Sec. 3.2.1, Eq. 4) on the feature map and does not mention them; the
+ * rule implemented here: F (Eq. 1) and the linear attention proper (Eq. 2) are global over all N
+ * tokens; in W a grid token attends its window and the P prefix tokens, a prefix token attends
+ * all N tokens; the convolution and the pooling that feeds its kernel generator see the grid only
+ * (a prefix token's L output is its linear-attention output alone).
+ */
 typedef struct {
   int32_t B, H, Hg, Wg, D;
   int32_t dtype; /* jv_dtype */
+  int32_t P;     /* prefix tokens in front of the grid tokens, >= 0 */
 } jv_shape;
 
 /*
@@ -188,6 +201,7 @@ jv_status jv_hybrid_mixers(int32_t n_layers, const char* schedule, const void* c
  * and read the mixers' [B, H, N, D] layout directly: no transpose pass between projection
  * and mixer.  bf16 only, D = 64 only (JV_ERR_UNSUPPORTED otherwise); C = H * D.
  *
+ * (N = P + Hg * Wg tokens; a projection does not care which of them are prefix tokens.)
  * jv_qkv_proj:  x [B, N, C] (token-major activations), w [3C, C] row-major (output feature
  *   by input feature, the rows ordered q | k | v and, inside each, head-major: row
  *   which*C + h*D + e), bias fp32 [3C] or NULL.

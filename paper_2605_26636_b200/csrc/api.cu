@@ -24,14 +24,14 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 }
 
 size_t tensor_bytes(const jv_shape* s) {
-  return (size_t)s->B * s->H * s->Hg * s->Wg * s->D * (s->dtype == JV_F32 ? 4 : 2);
+  return (size_t)s->B * s->H * shape_tokens(*s) * s->D * (s->dtype == JV_F32 ? 4 : 2);
 }
 
 jv_status check_shape(const jv_shape* s) {
   if (!s) return JV_ERR_INVALID_ARG;
-  if (s->B <= 0 || s->H <= 0 || s->Hg <= 0 || s->Wg <= 0 || s->D <= 0) return JV_ERR_INVALID_ARG;
+  if (s->B <= 0 || s->H <= 0 || s->Hg <= 0 || s->Wg <= 0 || s->D <= 0 || s->P < 0) return JV_ERR_INVALID_ARG;
   if (s->dtype != JV_F32 && s->dtype != JV_BF16) return JV_ERR_INVALID_ARG;
-  if ((int64_t)s->Hg * s->Wg > (1 << 24)) return JV_ERR_UNSUPPORTED;
+  if ((int64_t)s->Hg * s->Wg + s->P > (1 << 24)) return JV_ERR_UNSUPPORTED;
   if ((int64_t)s->B * s->H > 65535) return JV_ERR_UNSUPPORTED;
   if (s->D > 128) return JV_ERR_UNSUPPORTED;
   // rows must keep 16-byte alignment for the vector loads
@@ -105,8 +105,15 @@ float pick_scale(float scale, int D) { return scale > 0.f ? scale : 1.f / sqrtf(
 // ---- enqueue helpers (arguments already validated) ---------------------------
 jv_status run_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* s, int wh, int ww,
                    float scale, bool full, cudaStream_t st) {
-  AttnArgs a{q, k, v, o, s->B * s->H, s->Hg, s->Wg, s->D, wh, ww, pick_scale(scale, s->D), s->dtype};
+  AttnArgs a{q, k, v, o, s->B * s->H, s->Hg, s->Wg, s->D, s->P, wh, ww, pick_scale(scale, s->D), s->dtype};
   const bool one_window = full || (wh >= s->Hg && ww >= s->Wg);
+  if (one_window) {      // every token attends all P + N tokens: where a token sits does not matter
+    a.Hg = 1;
+    a.Wg = shape_tokens(*s);
+    a.P = 0;
+    a.wh = a.Hg;
+    a.ww = a.Wg;
+  }
   if (!g_force_generic.load() && one_window && attn_f4_supported(a)) {
     int* status = device_status_ptr();
     if (!status) return JV_ERR_CUDA;
@@ -115,7 +122,9 @@ jv_status run_attn(const void* q, const void* k, const void* v, void* o, const j
   if (!g_force_generic.load() && attn_tc_supported(a, full)) {
     int* status = device_status_ptr();
     if (!status) return JV_ERR_CUDA;
-    return from_cuda(launch_attn_tc(a, full, status, st));
+    const jv_status r = from_cuda(launch_attn_tc(a, full, status, st));
+    if (r != JV_OK || a.P == 0) return r;
+    return from_cuda(launch_attn_generic(a, st, true));   // the P prefix queries, which attend everything
   }
   return from_cuda(launch_attn_generic(a, st));
 }
@@ -123,6 +132,11 @@ jv_status run_attn(const void* q, const void* k, const void* v, void* o, const j
 jv_status run_linear(const void* q, const void* k, const void* v, void* o, const jv_shape* s, float eps,
                      const jv_dwc* dwc, void* ws, cudaStream_t st) {
   LinArgs a{q, k, v, o, *s, eps, dwc, ws};
+  if (!dwc && s->P > 0) {   // without the convolution the block is global: where a token sits does not matter
+    a.s.Hg = 1;
+    a.s.Wg = shape_tokens(*s);
+    a.s.P = 0;
+  }
   const LinPlan p = lin_plan(*s, dwc);
   if (!g_force_generic.load() && linear_fast_supported(a)) return from_cuda(launch_linear_fast(a, p, st));
   return from_cuda(launch_linear_generic(a, p, st));
@@ -260,7 +274,7 @@ jv_status jv_qkv_proj(const void* x, const void* w, const float* bias, void* q, 
                       const jv_shape* shape, void* cuda_stream) {
   if (!shape) return JV_ERR_INVALID_ARG;
   const void* ptrs[5] = {x, w, q, k, v};
-  const size_t C = (size_t)shape->H * shape->D, nt = (size_t)shape->B * shape->Hg * shape->Wg * C * 2;
+  const size_t C = (size_t)shape->H * shape->D, nt = (size_t)shape->B * shape_tokens(*shape) * C * 2;
   const size_t bytes[5] = {nt, 3 * C * C * 2, nt, nt, nt};
   jv_status st = check_proj(shape, ptrs, bytes, 5, 2);
   if (st != JV_OK) return st;
@@ -276,7 +290,7 @@ jv_status jv_out_proj(const void* o, const void* w, const float* bias, void* y, 
                       void* cuda_stream) {
   if (!shape) return JV_ERR_INVALID_ARG;
   const void* ptrs[3] = {o, w, y};
-  const size_t C = (size_t)shape->H * shape->D, nt = (size_t)shape->B * shape->Hg * shape->Wg * C * 2;
+  const size_t C = (size_t)shape->H * shape->D, nt = (size_t)shape->B * shape_tokens(*shape) * C * 2;
   const size_t bytes[3] = {nt, C * C * 2, nt};
   jv_status st = check_proj(shape, ptrs, bytes, 3, 2);
   if (st != JV_OK) return st;

@@ -24,6 +24,12 @@
 // Tensor memory (512 columns): scores S(t, b) 4 x 64 in [0, 256), accumulators O(t) 2 x 64
 // in [256, 384), probabilities P(t, b) 4 x 32 in [384, 512).
 //
+// Prefix tokens (P of them in front of the grid tokens; W only): every window's queries also
+// attend the P prefix keys.  They come in as one more key tile behind the window's own (a box of
+// a second pair of tensor maps that view the prefix rows in the box's shape), with the keys past P
+// masked like keys outside the grid.  The P prefix queries themselves (which attend everything)
+// are not served here.
+//
 // Every mbarrier wait is bounded: a wait that runs out sets the device status word,
 // raises a CTA-wide abort flag, and every role falls through to the common teardown
 // (tensor memory is always released).
@@ -63,6 +69,7 @@ struct TcParams {
   int qpairs;            // pairs of query tiles per window (by the full window height)
   int total_items;       // work items: (batch*head, window, query-tile pair), pair index fastest
   int lg_box_h;          // log2(box_h)
+  int P;                 // prefix keys behind every window's own key tiles (0: none)
   FastDiv div_qpairs, div_nwin, div_nwx;
   float scale_log2;      // softmax scale * log2(e)
 };
@@ -70,7 +77,8 @@ struct TcParams {
 // One work item of the persistent loop: two query tiles of one window of one (batch, head).
 struct Item {
   int bh, x0, y0, x_end, y_end;   // window origin and valid end (exclusive) in the token grid
-  int ntiles;                     // key tiles of the window
+  int ntiles;                     // tiles of the window (query tiles, and key tiles of its own tokens)
+  int nkt;                        // key tiles: the window's own, then one of prefix tokens if there are any
   int qt0;                        // first of the two query tiles
 };
 __device__ __forceinline__ Item decode_item(const TcParams& p, int i) {
@@ -84,6 +92,7 @@ __device__ __forceinline__ Item decode_item(const TcParams& p, int i) {
   it.x_end = min(it.x0 + p.win_w, p.gridW);
   it.y_end = min(it.y0 + p.win_h, p.gridH);
   it.ntiles = p.step_x ? (it.x_end - it.x0 + kTile - 1) / kTile : (it.y_end - it.y0 + p.box_h - 1) >> p.lg_box_h;
+  it.nkt = it.ntiles + (p.P > 0 ? 1 : 0);
   it.qt0 = 2 * qp;                // an item with qt0 >= ntiles (short edge window) is empty: every role skips it
   return it;
 }
@@ -112,7 +121,7 @@ constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
-               const TcParams p) {
+               const __grid_constant__ CUtensorMap mapKp, const __grid_constant__ CUtensorMap mapVp, const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -123,6 +132,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
   // broadcast from lane 0: lets the compiler keep everything derived from the warp index uniform
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
+
+  // a grid launched behind this one with programmatic serialisation (the prefix queries of W, which
+  // depend on nothing here) may run beside it
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // Once any CTA has flagged a timeout the rest of the grid (and later launches, until the
   // host reads the status) leave at once instead of each running into the same limit.
@@ -192,19 +205,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                       it.y0 + (it.qt0 + t) * p.step_y, it.bh);
       }
       __syncwarp();
-      for (int j = 0; j < it.ntiles; ++j) {
+      for (int j = 0; j < it.nkt; ++j) {
+        const bool pre = j == it.ntiles;               // the tile of prefix keys
         ok = warp_wait(&bar->k_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s], kTileBytes);
-          tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
+          if (pre) tma_load_4d(sK + s * kTileBytes, &mapKp, &bar->k_full[s], 0, 0, 0, it.bh);
+          else tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
         }
         __syncwarp();
         ok = warp_wait(&bar->v_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s], kTileBytes);
-          tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
+          if (pre) tma_load_4d(sV + s * kTileBytes, &mapVp, &bar->v_full[s], 0, 0, 0, it.bh);
+          else tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
         }
         __syncwarp();
         ++issued_v;
@@ -272,15 +288,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     Item it{};
     if (ok) {
       it = decode_item(p, cur);
-      ok = issue_qk(0, 0, it.ntiles, 0) && issue_qk(1, 0, it.ntiles, 0);
+      ok = issue_qk(0, 0, it.nkt, 0) && issue_qk(1, 0, it.nkt, 0);
     }
     while (ok) {
       const int nxt = next_item(cur);
       Item itn{};
       if (nxt >= 0) itn = decode_item(p, nxt);
-      for (int j = 0; j < it.ntiles && ok; ++j) {
+      for (int j = 0; j < it.nkt && ok; ++j) {
         ok = warp_wait(&bar->v_full[s], ph, &bar->abort_flag, p.status);
-        const bool last = j + 1 == it.ntiles;
+        const bool last = j + 1 == it.nkt;
         for (int h = 0; h < 2 && ok; ++h) {
           ok = warp_wait(&bar->p_full[t][h], g_par, &bar->abort_flag, p.status);
           if (!ok) break;
@@ -291,8 +307,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             mma_ts(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, smem_desc(vb + ks * 2048),
                    kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
           if (last && h == 1) tc_commit(&bar->o_full[t]);
-          if (!last) ok = issue_qk(h, j + 1, it.ntiles, n);              // its commit also covers the P V just issued
-          else if (nxt >= 0) ok = issue_qk(h, 0, itn.ntiles, n + 1);     // first key tile of the next item
+          if (!last) ok = issue_qk(h, j + 1, it.nkt, n);                 // its commit also covers the P V just issued
+          else if (nxt >= 0) ok = issue_qk(h, 0, itn.nkt, n + 1);        // first key tile of the next item
           else tc_commit(&bar->pv_done[t]);
         }
         if (ok) tc_commit(&bar->v_empty[s]);
@@ -489,7 +505,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     while (cur >= 0 && ok) {
       const Item it = decode_item(p, cur);
       const int nxt = next_item(cur);
-      const int ntiles = it.ntiles, nsteps = 2 * ntiles;
+      const int ntiles = it.ntiles, nsteps = 2 * it.nkt;
       const int x0 = it.x0, y0 = it.y0, x_end = it.x_end, y_end = it.y_end;
       // Which key tiles have keys that do not exist?  A window narrower than the box makes every
       // tile an edge tile; otherwise only the last tile of the window / sequence can be one.
@@ -517,16 +533,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           m = pend_m;
           pending = false;
         }
-        if (edge_all || (edge_last && j == ntiles - 1)) {
+        const bool pre = j == ntiles;                  // (only with prefix tokens: nsteps covers one more tile)
+        if (pre || edge_all || (edge_last && j == ntiles - 1)) {
           // Edge tile: overwrite the scores of keys that do not exist (outside the grid or the
-          // window) with -inf in tensor memory, then treat the step like any other.
+          // window; in the tile of prefix keys, past the P-th) with -inf in tensor memory, then
+          // treat the step like any other.
           // vx, vy: valid extent of the key tile's box along x and y
           const int vx = x_end - (x0 + j * p.step_x), vy = y_end - (y0 + j * p.step_y);
 #pragma unroll 1
           for (int c = 0; c < 2; ++c) {
             const int k0 = 64 * h + 32 * c;            // first of the 32 keys, as an index into the box
             uint32_t bits = 0;
-            if (p.box_w >= 32) {                       // the 32 keys lie in one box row
+            if (pre) {                                 // box position r holds prefix token r
+              const int nv = p.P - k0;
+              if (nv > 0) bits = nv >= 32 ? 0xffffffffu : ((1u << nv) - 1u);
+            } else if (p.box_w >= 32) {                // the 32 keys lie in one box row
               const int ly = k0 >> lg_bw, lx0 = k0 & (p.box_w - 1);
               const int nv = min(32, vx - lx0);
               if (ly < vy && nv > 0) bits = nv >= 32 ? 0xffffffffu : ((1u << nv) - 1u);
@@ -661,6 +682,7 @@ bool attn_tc_supported(const AttnArgs& a, bool full) {
   if (a.dtype != JV_BF16 || a.D != kD) return false;
   Geometry g;
   if (!geometry(a, full, &g)) return false;
+  if (a.P > kTile) return false;                        // the prefix keys are one key tile
   if ((int64_t)g.nwx * g.nwy * ceil_div(g.tiles_per_window, 2) * a.BH > 0x7fffffffll) return false;
   // 128-byte rows keep every TMA stride a multiple of 16 bytes; the base must be 16-byte aligned (checked by the ABI)
   return encode_fn() != nullptr;
@@ -671,9 +693,10 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   if (!geometry(a, full, &g)) return cudaErrorInvalidValue;
   EncodeFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
-  const int N = a.Hg * a.Wg;
-  CUtensorMap maps[4];
-  const void* ptrs[4] = {a.q, a.k, a.v, a.o};
+  const int N = a.P + a.Hg * a.Wg;                     // tokens per (batch, head): prefix tokens, then the grid
+  CUtensorMap maps[6];
+  const size_t grid0 = (size_t)a.P * kD * 2;           // the grid tokens start behind the prefix rows
+  const void* ptrs[4] = {(const char*)a.q + grid0, (const char*)a.k + grid0, (const char*)a.v + grid0, (char*)a.o + grid0};
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.gridW, (cuuint64_t)g.gridH, (cuuint64_t)a.BH};
   const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.gridW * kD * 2, (cuuint64_t)N * kD * 2};
   const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1};
@@ -688,13 +711,30 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
+  // The prefix rows of K and V in the shape of a key box: prefix token r at box position
+  // (r % box_w, r / box_w).  Positions past P inside the last box row read grid tokens (they exist:
+  // a grid holds at least one box row of tokens) and are masked by the softmax; rows past that are
+  // outside the map and arrive as zeros.
+  maps[4] = maps[1];
+  maps[5] = maps[2];
+  if (a.P > 0) {
+    const cuuint64_t pdims[4] = {(cuuint64_t)kD, (cuuint64_t)g.box_w, (cuuint64_t)ceil_div(a.P, g.box_w), (cuuint64_t)a.BH};
+    const cuuint64_t pstrides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.box_w * kD * 2, (cuuint64_t)N * kD * 2};
+    const void* pptrs[2] = {a.k, a.v};
+    for (int i = 0; i < 2; ++i) {
+      CUresult r = enc(&maps[4 + i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pptrs[i]), pdims, pstrides, box,
+                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+  }
   static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
   cudaError_t e = smem_opt_in.run([] {
     return cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   });
   if (e != cudaSuccess) return e;
   TcParams p;
-  p.o = (__nv_bfloat16*)a.o;
+  p.o = (__nv_bfloat16*)a.o + (size_t)a.P * kD;        // first grid token of (batch, head) 0
   p.status = status;
   p.gridW = g.gridW;
   p.gridH = g.gridH;
@@ -709,6 +749,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   p.nwin = g.nwx * g.nwy;
   p.qpairs = ceil_div(g.tiles_per_window, 2);
   p.total_items = p.qpairs * p.nwin * a.BH;
+  p.P = a.P;
   p.lg_box_h = 0;
   while ((1 << p.lg_box_h) < g.box_h) ++p.lg_box_h;
   p.div_qpairs = make_fastdiv((uint32_t)p.qpairs);
@@ -718,7 +759,7 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no more)
   const int num_sms = device_sm_count();
   const int grid = p.total_items < num_sms ? p.total_items : num_sms;
-  attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
   count_launch();
   return cudaGetLastError();
 }

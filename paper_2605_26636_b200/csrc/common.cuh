@@ -64,6 +64,8 @@ __device__ __forceinline__ float warp_sum(float x) {
 }
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+// tokens per (batch, head): prefix tokens, then the grid
+static inline int shape_tokens(const jv_shape& s) { return s.P + s.Hg * s.Wg; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- plan of the linear-attention workspace --------------------------------
@@ -84,11 +86,12 @@ struct AttnArgs {
   const void *q, *k, *v;
   void* o;
   int BH, Hg, Wg, D;
+  int P;       // prefix tokens in front of the Hg x Wg grid tokens (full attention: folded into the "grid")
   int wh, ww;  // window size (wh >= Hg and ww >= Wg: one window = full attention)
   float scale;
   int dtype;
 };
-cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st);
+cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, bool prefix_rows_only = false);
 // tcgen05 path: bf16, D == 64.  full = true: F over all N tokens; else W with (wh, ww)
 // windows whose width ww is a power of two <= 128 (a tile is a box of ww x 128/ww tokens).
 bool attn_tc_supported(const AttnArgs& a, bool full);

@@ -57,13 +57,13 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
 }
 
 // ---- host side: tensor maps ---------------------------------------------------------------
-// [BH, N, 64] bf16 as (channel, token, batch*head); boxes of box_tok tokens, 128-byte swizzle;
-// tokens past N arrive as zeros.
-inline bool make_map_tokens(CUtensorMap* m, const void* ptr, int BH, int N, int box_tok) {
+// The first N tokens of every (batch, head) of a [BH, ntok, 64] bf16 tensor as (channel, token,
+// batch*head); boxes of box_tok tokens, 128-byte swizzle; tokens past N arrive as zeros.
+inline bool make_map_tokens(CUtensorMap* m, const void* ptr, int BH, int N, int box_tok, int ntok) {
   tc::EncodeFn enc = tc::encode_fn();
   if (!enc) return false;
   const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)BH};
-  const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)N * kD * 2};
+  const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)ntok * kD * 2};
   const cuuint32_t box[3] = {(cuuint32_t)kD, (cuuint32_t)box_tok, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -71,13 +71,15 @@ inline bool make_map_tokens(CUtensorMap* m, const void* ptr, int BH, int N, int 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// [BH, Hg, Wg, 64] bf16 as a 4-D tensor (channel, x, y, batch*head); boxes of box_x x box_y
+// The Hg x Wg grid tokens of a [BH, P + Hg*Wg, 64] bf16 tensor (P prefix tokens in front of the
+// grid of every (batch, head)) as a 4-D tensor (channel, x, y, batch*head); boxes of box_x x box_y
 // tokens; positions outside the grid arrive as zeros on a load and are dropped by a store.
-inline bool make_map_grid(CUtensorMap* m, const void* ptr, int BH, int Hg, int Wg, int box_x, int box_y, bool swizzle128) {
+inline bool make_map_grid(CUtensorMap* m, const void* ptr, int BH, int P, int Hg, int Wg, int box_x, int box_y, bool swizzle128) {
   tc::EncodeFn enc = tc::encode_fn();
   if (!enc) return false;
+  ptr = (const char*)ptr + (size_t)P * kD * 2;       // rows are 128 bytes: the base stays 16-byte aligned
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)Wg, (cuuint64_t)Hg, (cuuint64_t)BH};
-  const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)Wg * kD * 2, (cuuint64_t)Hg * Wg * kD * 2};
+  const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)Wg * kD * 2, (cuuint64_t)(P + Hg * Wg) * kD * 2};
   const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)box_x, (cuuint32_t)box_y, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,

@@ -516,7 +516,8 @@ bool linear_conv_supported(const LinArgs& a) {
   return tiles <= 0x7fffffffll;
 }
 
-// Enqueues the fused apply + convolution pass.  `partial` holds the chunk partials of the state
+// Enqueues the fused apply + convolution pass over the grid tokens (prefix tokens, which the
+// convolution does not see, are left to the plain apply pass).  `partial` holds the chunk partials of the state
 // pass, `w` the kernels [B][C][3][3]; both are written by grids ahead of this one in the stream,
 // which this grid waits for (griddepcontrol.wait) before it reads them.
 cudaError_t launch_linear_apply_conv(const LinArgs& a, const LinPlan& p, const float* partial, const float* w,
@@ -524,9 +525,9 @@ cudaError_t launch_linear_apply_conv(const LinArgs& a, const LinPlan& p, const f
   const jv_shape& s = a.s;
   const int BH = s.B * s.H;
   CUtensorMap mq, mv, mo;
-  if (!make_map_grid(&mq, a.q, BH, s.Hg, s.Wg, kPatchW, kPatchH, true) ||
-      !make_map_grid(&mv, a.v, BH, s.Hg, s.Wg, kPatchW + 2, kPatchH + 2, false) ||
-      !make_map_grid(&mo, a.o, BH, s.Hg, s.Wg, kPatchW, kPatchH, true))
+  if (!make_map_grid(&mq, a.q, BH, s.P, s.Hg, s.Wg, kPatchW, kPatchH, true) ||
+      !make_map_grid(&mv, a.v, BH, s.P, s.Hg, s.Wg, kPatchW + 2, kPatchH + 2, false) ||
+      !make_map_grid(&mo, a.o, BH, s.P, s.Hg, s.Wg, kPatchW, kPatchH, true))
     return cudaErrorInvalidValue;
   static OncePerDevice smem_opt_in;
   cudaError_t e = smem_opt_in.run([] {

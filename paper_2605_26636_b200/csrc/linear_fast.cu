@@ -543,7 +543,8 @@ dwc_add_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ 
 constexpr int kGenTile = 1024;
 __global__ void __launch_bounds__(256)
 gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W1, const float* __restrict__ b1,
-                  float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n, int early_trigger) {
+                  float* __restrict__ hidden, int H, int R, int nchunk, int state_elems, float inv_n, int early_trigger,
+                  const __nv_bfloat16* __restrict__ v, int P, int ntok) {
   __shared__ __align__(16) float s_sm[kGenTile];
   // early_trigger: the grids behind this one each wait for their predecessor before they read its
   // output, so they may be resident (set up, prefetching inputs of the call) while this one waits.
@@ -574,6 +575,8 @@ gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W
       if (c < C) {
         const float* pv = partial + (size_t)(b * H + c / kD) * nchunk * state_elems + kOffVsum + c % kD;
         for (int k = 0; k < nchunk; ++k) m += __ldcg(pv + (size_t)k * state_elems);
+        // the v-sums run over all tokens; the pooling is over the grid: take the prefix rows out again
+        for (int t = 0; t < P; ++t) m -= __bfloat162float(v[((size_t)(b * H + c / kD) * ntok + t) * kD + c % kD]);
       }
       s_sm[threadIdx.x + 256 * i] = m * inv_n;
     }
@@ -593,12 +596,11 @@ gen_hidden_kernel(const float* __restrict__ partial, const float* __restrict__ W
 // w[b][t] = b2[t] + sum_r W2[t][r] * hidden[b][r]; 8 lanes per output t, 32 outputs per block, all
 // samples (8 at a time, their hidden vectors in shared memory).  kVec (R a multiple of 4): a lane's
 // part of the W2 row is fetched as float4, the whole row in flight at once.
-constexpr int kGenMaxR = 1024;
 template <bool kVec>
 __global__ void __launch_bounds__(256)
 gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, const float* __restrict__ b2,
                float* __restrict__ w, int B, int T, int R, int wait_first) {
-  __shared__ __align__(16) float h_sm[8 * kGenMaxR];
+  extern __shared__ __align__(16) float h_sm[];        // [min(B, 8)][R]: small, so that the grid can be resident early
   // wait_first = 0: launched behind the apply grid, which lets its dependents go only after it has
   // seen the hidden layer's grid complete: hidden is final here and this grid runs beside the apply
   // pass; it waits at its end (below).  wait_first = 1: launched directly behind the hidden layer
@@ -634,13 +636,13 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
       if (r0 == 0) {                                   // this group of samples' hidden vectors -> shared memory
         if (!waited) { griddep_wait(); waited = true; }
         __syncthreads();
-        for (int i = threadIdx.x; i < nb * R; i += 256) h_sm[(i / R) * kGenMaxR + i % R] = __ldcg(hidden + (size_t)b0 * R + i);
+        for (int i = threadIdx.x; i < nb * R; i += 256) h_sm[i] = __ldcg(hidden + (size_t)b0 * R + i);
         __syncthreads();
       }
 #pragma unroll
       for (int bb = 0; bb < 8; ++bb) {
         if (bb < nb) {
-          const float* hp = h_sm + bb * kGenMaxR + r0;
+          const float* hp = h_sm + bb * R + r0;
           if (kVec) {
 #pragma unroll
             for (int i = 0; i < kPer; ++i) {
@@ -678,20 +680,21 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
 }  // namespace
 
 bool linear_fast_supported(const LinArgs& a) {
+  if (a.dwc && a.s.P > 0 && a.dwc->k != 3) return false;   // prefix tokens + 5 x 5 kernels: the generic kernels
   return a.s.dtype == JV_BF16 && a.s.D == kD && encode_fn() != nullptr;
 }
 
 cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t st) {
   const jv_shape& s = a.s;
-  const int N = s.Hg * s.Wg, BH = s.B * s.H;
+  const int N = shape_tokens(s), BH = s.B * s.H;       // the state and the attention proper run over all tokens
   char* ws = (char*)a.ws;
   float* partial = (float*)(ws + p.off_partial);
   int* status = device_status_ptr();
   if (!status) return cudaErrorUnknown;
 
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map_tokens(&mq, a.q, BH, N, kApplyTok) || !make_map_tokens(&mk, a.k, BH, N, kTileTok) ||
-      !make_map_tokens(&mv, a.v, BH, N, kTileTok) || !make_map_tokens(&mo, a.o, BH, N, 32))
+  if (!make_map_tokens(&mq, a.q, BH, N, kApplyTok, N) || !make_map_tokens(&mk, a.k, BH, N, kTileTok, N) ||
+      !make_map_tokens(&mv, a.v, BH, N, kTileTok, N) || !make_map_tokens(&mo, a.o, BH, N, 32, N))
     return cudaErrorInvalidValue;
 
   static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
@@ -722,8 +725,39 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   // each grid waits for its predecessor (griddepcontrol.wait) before it reads what that one wrote,
   // the output layer at its very end, so that stream order still means "apply pass complete" for
   // the convolution pass that follows it.
+  // apply pass over the first ntokens tokens of every (batch, head): one wave of two CTAs per SM, spans
+  // of whole 128-token tiles; launched so that its set-up overlaps the tail of the grid before it
+  auto enqueue_apply = [&](const CUtensorMap& map_q, const CUtensorMap& map_o, int ntokens) -> cudaError_t {
+    int nspan = (2 * num_sms) / BH;
+    if (nspan < 1) nspan = 1;
+    int span = ceil_div(ceil_div(ntokens, nspan), kApplyTok) * kApplyTok;
+    if (span < 4 * kApplyTok) span = 4 * kApplyTok;
+    nspan = ceil_div(ntokens, span);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(nspan, BH);
+    cfg.blockDim = dim3(kApplyThreads);
+    cfg.dynamicSmemBytes = kApplySmem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, lin_apply_kernel, map_q, map_o, (const float*)partial, status, ntokens,
+                                               span, p.nchunk, p.state_elems, a.eps);
+    count_launch();
+    return err;
+  };
+
   float* hidden = (float*)(ws + p.off_hidden);
   const bool fused_conv = a.dwc && linear_conv_supported(a);
+  if (fused_conv && s.P > 0) {
+    // Prefix tokens: the convolution does not see them, their output is the attention output alone.
+    // The plain apply pass over the first P tokens of every (batch, head), right behind the state pass
+    // (which it waits for; the grids behind it wait for it in turn).
+    CUtensorMap mqp, mop;
+    if (!make_map_tokens(&mqp, a.q, BH, s.P, kApplyTok, N) || !make_map_tokens(&mop, a.o, BH, s.P, 32, N))
+      return cudaErrorInvalidValue;
+    e = enqueue_apply(mqp, mop, s.P);
+    if (e != cudaSuccess) return e;
+  }
   if (a.dwc && a.dwc->R > 0) {      // R == 0: static kernels, the output layer just broadcasts b2
     const jv_dwc& d = *a.dwc;
     cudaLaunchConfig_t hcfg = {};
@@ -733,7 +767,8 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     hcfg.gridDim = dim3(ceil_div(d.R, 8), s.B);
     hcfg.blockDim = dim3(256);
     e = cudaLaunchKernelEx(&hcfg, gen_hidden_kernel, (const float*)partial, d.W1, d.b1, hidden, (int)s.H, (int)d.R,
-                           p.nchunk, p.state_elems, 1.f / (float)N, fused_conv ? 1 : 0);
+                           p.nchunk, p.state_elems, 1.f / (float)(s.Hg * s.Wg), fused_conv ? 1 : 0, (const __nv_bfloat16*)a.v,
+                           (int)s.P, N);
     count_launch();
     if (e != cudaSuccess) return e;
   }
@@ -751,6 +786,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     gcfg.numAttrs = 1;
     gcfg.gridDim = dim3(ceil_div(T, 32));
     gcfg.blockDim = dim3(256);
+    gcfg.dynamicSmemBytes = (size_t)(s.B < 8 ? s.B : 8) * d.R * sizeof(float);
     e = cudaLaunchKernelEx(&gcfg, (d.R % 4 == 0) ? gen_out_kernel<true> : gen_out_kernel<false>, (const float*)hidden, d.W2,
                            d.b2, wk, (int)s.B, T, (int)d.R, 1);
     count_launch();
@@ -758,23 +794,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     return launch_linear_apply_conv(a, p, partial, wk, status, true, st);
   }
 
-  // apply pass: one wave of two CTAs per SM, spans of whole 128-token tiles; launched so that its
-  // set-up overlaps the tail of the grid before it
-  int nspan = (2 * num_sms) / BH;
-  if (nspan < 1) nspan = 1;
-  int span = ceil_div(ceil_div(N, nspan), kApplyTok) * kApplyTok;
-  if (span < 4 * kApplyTok) span = 4 * kApplyTok;
-  nspan = ceil_div(N, span);
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(nspan, BH);
-  cfg.blockDim = dim3(kApplyThreads);
-  cfg.dynamicSmemBytes = kApplySmem;
-  cfg.stream = st;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  e = cudaLaunchKernelEx(&cfg, lin_apply_kernel, mq, mo, (const float*)partial, status, N, span, p.nchunk,
-                         p.state_elems, a.eps);
-  count_launch();
+  e = enqueue_apply(mq, mo, N);
   if (e != cudaSuccess) return e;
 
   if (a.dwc) {
@@ -789,6 +809,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     gcfg.numAttrs = 1;
     gcfg.gridDim = dim3(ceil_div(T, 32));
     gcfg.blockDim = dim3(256);
+    gcfg.dynamicSmemBytes = (size_t)(s.B < 8 ? s.B : 8) * d.R * sizeof(float);
     e = cudaLaunchKernelEx(&gcfg, (d.R % 4 == 0) ? gen_out_kernel<true> : gen_out_kernel<false>, (const float*)hidden, d.W2,
                            d.b2, wk, (int)s.B, T, (int)d.R, 0);
     count_launch();

@@ -12,7 +12,7 @@ namespace jv {
 
 LinPlan lin_plan(const jv_shape& s, const jv_dwc* dwc) {
   LinPlan p{};
-  const int N = s.Hg * s.Wg, BH = s.B * s.H;
+  const int N = shape_tokens(s), BH = s.B * s.H;
   p.D1 = s.D + 1;
   p.state_elems = (p.D1 * p.D1 + 3) / 4 * 4;
   // Chunks: as many as fit one wave of two CTAs per SM over all (batch, head) pairs, each a
@@ -109,10 +109,10 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 lin_apply_generic_kernel(const T* __restrict__ q, const T* __restrict__ v, T* __restrict__ o,
                          const float* __restrict__ state, const float* __restrict__ dwc_w,
-                         int H, int Hg, int Wg, int D, int state_elems, float eps, int ksz) {
+                         int H, int P, int Hg, int Wg, int D, int state_elems, float eps, int ksz) {
   extern __shared__ float smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int N = Hg * Wg, D1 = D + 1;
+  const int N = P + Hg * Wg, D1 = D + 1;                    // P prefix tokens, then the grid
   const int bh = blockIdx.y;
   const int tok = blockIdx.x * 8 + warp;
   float* qs = smem + warp * D;
@@ -123,12 +123,12 @@ lin_apply_generic_kernel(const T* __restrict__ q, const T* __restrict__ v, T* __
   const float* S = state + (size_t)bh * state_elems;
   float den = eps;
   for (int a = 0; a < D; ++a) den = fmaf(qs[a], __ldg(&S[a * D1 + D]), den);
-  const int y = tok / Wg, x = tok % Wg, pad = (ksz - 1) / 2;
+  const int y = (tok - P) / Wg, x = (tok - P) % Wg, pad = (ksz - 1) / 2;   // (grid tokens only)
   for (int e = lane; e < D; e += 32) {
     float num = 0.f;
     for (int a = 0; a < D; ++a) num = fmaf(qs[a], __ldg(&S[a * D1 + e]), num);
     float r = num / den;
-    if (dwc_w) {
+    if (dwc_w && tok >= P) {      // the convolution sees the feature map only
       const int b = bh / H, h = bh % H;
       const float* w = dwc_w + ((size_t)b * H * D + (size_t)h * D + e) * ksz * ksz;
       float c = 0.f;
@@ -136,7 +136,7 @@ lin_apply_generic_kernel(const T* __restrict__ q, const T* __restrict__ v, T* __
         for (int dx = 0; dx < ksz; ++dx) {
           const int yy = y + dy - pad, xx = x + dx - pad;
           if (yy >= 0 && yy < Hg && xx >= 0 && xx < Wg)
-            c = fmaf(__ldg(&w[dy * ksz + dx]), to_f32(v[base + (size_t)(yy * Wg + xx) * D + e]), c);
+            c = fmaf(__ldg(&w[dy * ksz + dx]), to_f32(v[base + (size_t)(P + yy * Wg + xx) * D + e]), c);
         }
       r += c;
     }
@@ -147,10 +147,12 @@ lin_apply_generic_kernel(const T* __restrict__ q, const T* __restrict__ v, T* __
 // ---- kernel generator of the squeeze dynamic convolution ---------------------
 // hidden[b][r] = SiLU(b1[r] + sum_c W1[r][c] * mean_v[b][c]); one warp per (b, r).
 // vsum points at the v-sum of (batch 0, head 0); consecutive (batch, head) pairs are
-// bh_stride floats apart.
-__global__ void dwc_hidden_kernel(const float* __restrict__ vsum, const float* __restrict__ W1,
+// bh_stride floats apart.  The v-sums run over all tokens; the pooling is over the grid
+// tokens, so the P prefix rows of V (v: [B*H][ntok][D]) are taken out again.
+template <typename T>
+__global__ void dwc_hidden_kernel(const float* __restrict__ vsum, const T* __restrict__ v, const float* __restrict__ W1,
                                   const float* __restrict__ b1, float* __restrict__ hidden,
-                                  int H, int D, int R, int bh_stride, float inv_n) {
+                                  int H, int D, int R, int bh_stride, int P, int ntok, float inv_n) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.y;
   if (warp >= R) return;
@@ -158,7 +160,9 @@ __global__ void dwc_hidden_kernel(const float* __restrict__ vsum, const float* _
   float s = 0.f;
   for (int c = lane; c < C; c += 32) {
     const int h = c / D, e = c % D;
-    const float mean = vsum[((size_t)b * H + h) * bh_stride + e] * inv_n;
+    float sum = vsum[((size_t)b * H + h) * bh_stride + e];
+    for (int t = 0; t < P; ++t) sum -= to_f32(v[(((size_t)b * H + h) * ntok + t) * D + e]);
+    const float mean = sum * inv_n;
     s = fmaf(__ldg(&W1[(size_t)warp * C + c]), mean, s);
   }
   s = warp_sum(s);
@@ -184,7 +188,7 @@ __global__ void dwc_out_kernel(const float* __restrict__ hidden, const float* __
 template <typename T>
 cudaError_t launch_generic_t(const LinArgs& a, const LinPlan& p, cudaStream_t st) {
   const jv_shape& s = a.s;
-  const int N = s.Hg * s.Wg, BH = s.B * s.H;
+  const int N = shape_tokens(s), BH = s.B * s.H;
   char* ws = (char*)a.ws;
   float* partial = (float*)(ws + p.off_partial);
   float* state = (float*)(ws + p.off_state);
@@ -208,7 +212,7 @@ cudaError_t launch_generic_t(const LinArgs& a, const LinPlan& p, cudaStream_t st
   }
   dim3 g3(ceil_div(N, 8), BH);
   lin_apply_generic_kernel<T><<<g3, 256, 8 * s.D * sizeof(float), st>>>(
-      (const T*)a.q, (const T*)a.v, (T*)a.o, state, dw, s.H, s.Hg, s.Wg, s.D, p.state_elems, a.eps,
+      (const T*)a.q, (const T*)a.v, (T*)a.o, state, dw, s.H, s.P, s.Hg, s.Wg, s.D, p.state_elems, a.eps,
       a.dwc ? a.dwc->k : 0);
   count_launch();
   return cudaGetLastError();
@@ -230,10 +234,15 @@ cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float
   char* ws = (char*)a.ws;
   float* hidden = (float*)(ws + p.off_hidden);
   float* w = (float*)(ws + p.off_kernel);
-  const int N = s.Hg * s.Wg;
+  const int N = s.Hg * s.Wg, ntok = shape_tokens(s);   // pooling: the mean over the grid tokens
   if (d.R > 0) {   // R == 0: static kernels, the output layer just broadcasts b2
     dim3 g1(ceil_div(d.R * 32, 256), s.B);
-    dwc_hidden_kernel<<<g1, 256, 0, st>>>(vsum, d.W1, d.b1, hidden, s.H, s.D, d.R, bh_stride, 1.f / (float)N);
+    if (s.dtype == JV_F32)
+      dwc_hidden_kernel<float><<<g1, 256, 0, st>>>(vsum, (const float*)a.v, d.W1, d.b1, hidden, s.H, s.D, d.R, bh_stride,
+                                                   s.P, ntok, 1.f / (float)N);
+    else
+      dwc_hidden_kernel<__nv_bfloat16><<<g1, 256, 0, st>>>(vsum, (const __nv_bfloat16*)a.v, d.W1, d.b1, hidden, s.H, s.D, d.R,
+                                                           bh_stride, s.P, ntok, 1.f / (float)N);
     count_launch();
   }
   const int T = s.H * s.D * d.k * d.k;

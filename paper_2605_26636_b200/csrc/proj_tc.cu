@@ -287,7 +287,7 @@ bool proj_tc_available() { return encode_fn() != nullptr; }
 cudaError_t launch_proj_tc(bool qkv, const void* x, const void* w, const float* bias, void* d0, void* d1, void* d2,
                            const jv_shape& s, int* status, cudaStream_t st) {
   if (!encode_fn()) return cudaErrorNotSupported;
-  const uint64_t N = (uint64_t)s.Hg * s.Wg, C = (uint64_t)s.H * kD, BH = (uint64_t)s.B * s.H;
+  const uint64_t N = (uint64_t)shape_tokens(s), C = (uint64_t)s.H * kD, BH = (uint64_t)s.B * s.H;   // prefix and grid tokens alike
   const uint64_t features = qkv ? 3 * C : C;
   CUtensorMap ma, mb, md0, md1, md2;
   bool ok = map2(&mb, w, C, features, kBN);

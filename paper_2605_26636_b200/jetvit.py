@@ -21,7 +21,7 @@ LIB_PATH = os.environ.get("JETVIT_LIB") or os.path.join(_HERE, "libjetvit.so")
 
 class JvShape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("Hg", ctypes.c_int32),
-                ("Wg", ctypes.c_int32), ("D", ctypes.c_int32), ("dtype", ctypes.c_int32)]
+                ("Wg", ctypes.c_int32), ("D", ctypes.c_int32), ("dtype", ctypes.c_int32), ("P", ctypes.c_int32)]
 
 
 class JvDwc(ctypes.Structure):
@@ -100,11 +100,13 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"dtype {t.dtype}: the mixers take float32 or bfloat16")
 
 
-def make_shape(t: torch.Tensor, Hg: int, Wg: int) -> JvShape:
+def make_shape(t: torch.Tensor, Hg: int, Wg: int, prefix: int = 0) -> JvShape:
+    """Shape of [B, H, prefix + Hg*Wg, D] tensors: ``prefix`` tokens (class / register tokens) in
+    front of the grid tokens."""
     B, H, N, D = t.shape
-    if N != Hg * Wg:
-        raise ValueError(f"N = {N} is not Hg*Wg = {Hg}*{Wg}")
-    return JvShape(B, H, Hg, Wg, D, _dtype_code(t))
+    if prefix < 0 or N != prefix + Hg * Wg:
+        raise ValueError(f"N = {N} is not prefix + Hg*Wg = {prefix} + {Hg}*{Wg}")
+    return JvShape(B, H, Hg, Wg, D, _dtype_code(t), prefix)
 
 
 def _check_tensors(*ts: torch.Tensor):
@@ -155,11 +157,11 @@ def _raise(status: int, where: str):
 
 
 def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict] = None, out=None,
-                ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+                ws: Optional[torch.Tensor] = None, stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_linear_attn.  Allocates ``out`` / ``ws`` with torch when not given."""
     out = torch.empty_like(q) if out is None else out
     _check_tensors(q, k, v, out)
-    shape = make_shape(q, Hg, Wg)
+    shape = make_shape(q, Hg, Wg, prefix)
     d = make_dwc(dwc, q.device)
     with torch.cuda.device(q.device):
         if ws is None:
@@ -177,13 +179,13 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 
 def linear_attn_static(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict] = None, *, out,
-                       stream=None) -> torch.Tensor:
+                       stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_linear_attn_static: the linear block with the library's built-in scratch, for
     callers that must not allocate.  This wrapper allocates nothing either: ``out`` is
     required.  Problems needing more than STATIC_SCRATCH_BYTES raise JV_ERR_WORKSPACE;
     calls that can overlap on the GPU must be ordered by the caller (they share the scratch)."""
     _check_tensors(q, k, v, out)
-    shape = make_shape(q, Hg, Wg)
+    shape = make_shape(q, Hg, Wg, prefix)
     d = make_dwc(dwc, q.device)
     with torch.cuda.device(q.device):
         st = lib().jv_linear_attn_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
@@ -194,11 +196,11 @@ def linear_attn_static(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Option
 
 
 def window_attn(q, k, v, Hg: int, Wg: int, win_h: int, win_w: int, scale: float = 0.0, out=None,
-                stream=None) -> torch.Tensor:
+                stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_window_attn (scale <= 0: 1/sqrt(D))."""
     out = torch.empty_like(q) if out is None else out
     _check_tensors(q, k, v, out)
-    shape = make_shape(q, Hg, Wg)
+    shape = make_shape(q, Hg, Wg, prefix)
     with torch.cuda.device(q.device):
         st = lib().jv_window_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
                                   int(win_h), int(win_w), float(scale), None, 0, _stream(stream))
@@ -223,7 +225,8 @@ def full_attn(q, k, v, Hg: Optional[int] = None, Wg: Optional[int] = None, scale
 
 def hybrid_mixers(schedule: str, q: Sequence[torch.Tensor], k, v, Hg: int, Wg: int, win_h: int, win_w: int,
                   scale: float = 0.0, eps: float = 1e-6, dwc: Optional[Sequence[Optional[dict]]] = None,
-                  out: Optional[Sequence[torch.Tensor]] = None, ws: Optional[torch.Tensor] = None, stream=None):
+                  out: Optional[Sequence[torch.Tensor]] = None, ws: Optional[torch.Tensor] = None, stream=None,
+                  prefix: int = 0):
     """jv_hybrid_mixers: one mixer per layer, schedule[l] in 'L', 'W', 'F'."""
     n = len(schedule)
     if not (len(q) == len(k) == len(v) == n):
@@ -233,7 +236,7 @@ def hybrid_mixers(schedule: str, q: Sequence[torch.Tensor], k, v, Hg: int, Wg: i
         _check_tensors(q[l], k[l], v[l], out[l])
         if q[l].shape != q[0].shape or q[l].dtype != q[0].dtype:
             raise ValueError("all layers share one shape and dtype")
-    shape = make_shape(q[0], Hg, Wg)
+    shape = make_shape(q[0], Hg, Wg, prefix)
     arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
     dstructs = [make_dwc(d, q[0].device) for d in dwc] if dwc is not None else None
     dptr = None
@@ -268,18 +271,18 @@ def _check_proj(x, w, bias, H: int, rows: int):
         raise ValueError(f"bias must be a contiguous fp32 CUDA tensor of [{rows}]")
 
 
-def qkv_proj(x, w, bias, H: int, Hg: int, Wg: int, out=None, stream=None):
+def qkv_proj(x, w, bias, H: int, Hg: int, Wg: int, out=None, stream=None, prefix: int = 0):
     """jv_qkv_proj: x [B, N, C] bf16, w [3C, C] bf16, bias fp32 [3C] or None -> (q, k, v), each
     [B, H, N, 64] in the mixers' layout.  ``out`` is an optional (q, k, v) triple to write into."""
     B, N, C = x.shape
-    if C != 64 * H or N != Hg * Wg:
-        raise ValueError("x must be [B, Hg*Wg, 64*H]")
+    if C != 64 * H or N != prefix + Hg * Wg:
+        raise ValueError("x must be [B, prefix + Hg*Wg, 64*H]")
     _check_proj(x, w, bias, H, 3 * C)
     q, k, v = out if out is not None else (torch.empty((B, H, N, 64), dtype=x.dtype, device=x.device) for _ in range(3))
     _check_tensors(q, k, v)
     if tuple(q.shape) != (B, H, N, 64) or q.dtype != x.dtype:
         raise ValueError("q, k, v must be [B, H, N, 64] bf16")
-    shape = JvShape(B, H, Hg, Wg, 64, JV_BF16)
+    shape = JvShape(B, H, Hg, Wg, 64, JV_BF16, prefix)
     with torch.cuda.device(x.device):
         st = lib().jv_qkv_proj(x.data_ptr(), w.data_ptr(), None if bias is None else bias.data_ptr(), q.data_ptr(),
                                k.data_ptr(), v.data_ptr(), ctypes.byref(shape), _stream(stream))
@@ -287,18 +290,18 @@ def qkv_proj(x, w, bias, H: int, Hg: int, Wg: int, out=None, stream=None):
     return q, k, v
 
 
-def out_proj(o, w, bias, Hg: int, Wg: int, out=None, stream=None) -> torch.Tensor:
+def out_proj(o, w, bias, Hg: int, Wg: int, out=None, stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_out_proj: o [B, H, N, 64] bf16 (a mixer's output), w [C, C] bf16, bias fp32 [C] or None
     -> y [B, N, C]."""
     B, H, N, D = o.shape
-    if D != 64 or N != Hg * Wg:
-        raise ValueError("o must be [B, H, Hg*Wg, 64]")
+    if D != 64 or N != prefix + Hg * Wg:
+        raise ValueError("o must be [B, H, prefix + Hg*Wg, 64]")
     C = 64 * H
     _check_proj(o, w, bias, H, C)
     y = torch.empty((B, N, C), dtype=o.dtype, device=o.device) if out is None else out
     if not (y.is_cuda and y.is_contiguous() and tuple(y.shape) == (B, N, C) and y.dtype == o.dtype):
         raise ValueError("y must be a contiguous [B, N, C] bf16 CUDA tensor")
-    shape = JvShape(B, H, Hg, Wg, 64, JV_BF16)
+    shape = JvShape(B, H, Hg, Wg, 64, JV_BF16, prefix)
     with torch.cuda.device(o.device):
         st = lib().jv_out_proj(o.data_ptr(), w.data_ptr(), None if bias is None else bias.data_ptr(), y.data_ptr(),
                                ctypes.byref(shape), _stream(stream))
