@@ -40,9 +40,58 @@ METRIC = "mixer tokens/sec (L+W+F stack at ViT-L shapes)"
 UNIT = "tokens/s"
 STEP_SCHEDULE = "LWF"
 WIN = 16
-# DRAM bytes of one attn_f4_kernel launch (F at the DINOv3-L shape), from the ncu capture
-# summarised in profiles/ (None when the kernel has changed since the capture)
-ATTN_F_DRAM_BYTES = 245_050_000
+# DRAM traffic of the dominant kernel comes from an ncu capture; the record of that capture names the
+# kernel's source files and their hash, and the figure is reported only while the hash still matches
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "attn_f4_kernel_dinov3_l.traffic.json")
+
+
+TRAFFIC_SOURCES = ["paper_2605_26636_b200/csrc/attn_f4.cu", "paper_2605_26636_b200/csrc/tc_common.cuh"]
+
+
+def record_traffic(csv_path):
+    """Writes TRAFFIC_RECORD from `ncu -i <report> --page raw --csv` output of a capture of attn_f4_kernel
+    (`ncu --set full ... python bench.py --single F`): DRAM bytes per launch and the hash of the kernel's source."""
+    import csv
+    import hashlib
+    rows = list(csv.reader(open(csv_path)))
+    hdr, units = rows[0], rows[1]
+    ix = {h: i for i, h in enumerate(hdr)}
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    vals = []
+    for r in rows[2:]:
+        if "attn_f4_kernel" not in r[ix["Kernel Name"]]:
+            continue
+        tot = 0.0
+        for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+            tot += float(r[ix[key]].replace(",", "")) * scale[units[ix[key]]]
+        vals.append(tot)
+    if not vals:
+        raise SystemExit("no attn_f4_kernel launch in " + csv_path)
+    h = hashlib.sha256()
+    for rel in TRAFFIC_SOURCES:
+        h.update(open(os.path.join(ROOT, rel), "rb").read())
+    rec = {"kernel": "attn_f4_kernel", "workload": "F at dinov3_l (B=8, H=16, N=4096, D=64, bf16)", "launches": len(vals),
+           "dram_bytes_per_launch": int(sum(vals) / len(vals)), "sources": TRAFFIC_SOURCES, "sha256": h.hexdigest(),
+           "how": "ncu --set full --clock-control none -k regex:attn_f4 python bench.py --single F --steps 2 --warmup 1; "
+                  "ncu -i <report> --page raw --csv; python bench.py --record-traffic <csv>"}
+    json.dump(rec, open(TRAFFIC_RECORD, "w"), indent=1)
+    print(json.dumps(rec))
+
+
+def measured_traffic():
+    """(bytes per launch or None, note): dram__bytes_read.sum + dram__bytes_write.sum of one launch of the
+    dominant kernel, valid only for the source it was captured from."""
+    import hashlib
+    try:
+        rec = json.load(open(TRAFFIC_RECORD))
+        h = hashlib.sha256()
+        for rel in rec["sources"]:
+            h.update(open(os.path.join(ROOT, rel), "rb").read())
+        if h.hexdigest() == rec["sha256"]:
+            return int(rec["dram_bytes_per_launch"]), "ncu capture of the current source"
+        return None, "the kernel's source has changed since the ncu capture"
+    except (OSError, KeyError, ValueError):
+        return None, "no ncu record"
 
 
 def load_peaks():
@@ -61,13 +110,14 @@ def alg_bytes(B, H, N, D, esz=2, dwc=False):
     return B * H * N * D * esz * (5 if dwc else 4)
 
 
-def alg_flops_attn(B, H, Hg, Wg, D, wh, ww):
-    """2 flops per MAC over valid (query, key) pairs only, QK^T and PV."""
-    pairs = 0
+def alg_flops_attn(B, H, Hg, Wg, D, wh, ww, prefix=0):
+    """2 flops per MAC over valid (query, key) pairs only, QK^T and PV; with prefix tokens every
+    window token also attends them, and they attend everything."""
+    pairs = prefix * (prefix + Hg * Wg)
     for y0 in range(0, Hg, wh):
         for x0 in range(0, Wg, ww):
             n = min(wh, Hg - y0) * min(ww, Wg - x0)
-            pairs += n * n
+            pairs += n * (n + prefix)
     return 4 * D * pairs * B * H
 
 
@@ -212,7 +262,9 @@ def run_reference(args):
     value = step_tokens / step_s
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "extrapolated": True,
+            "extrapolated_note": "each step times a bounded sample of the workload; ms_per_step and value scale every mixer's "
+                                 "time by its sampled fraction",
             "config": {"workload": "dinov3_l 64x64 grid B=8 H=16 D=64, schedule LWF (CPU oracle, sampled)"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -286,6 +338,20 @@ def run_cuda(args):
     assert jv.device_status() == jv.JV_OK, "a kernel reported a timeout"
     step_tokens = nL * w.tokens
     value = world * step_tokens / (ms * 1e-3)
+
+    # ---- the same step for at least a second: what the clocks settle at under the power cap
+    n_sus = max(50, int(1.2e3 / max(ms, 1e-3)))
+    with ClockSampler(local) as clk_sus:
+        e0.record(stream)
+        for i in range(n_sus):
+            step()
+        e1.record(stream)
+        barrier()
+    ms_sus = max_over_ranks(e0.elapsed_time(e1) / n_sus, world, dev)
+    cs = clk_sus.summary()
+    sustained = {"steps": n_sus, "ms_per_step": ms_sus, "value": world * step_tokens / (ms_sus * 1e-3), "unit": UNIT,
+                 "clocks": cs, "ms_x_mhz": (ms_sus * cs["sm_mhz"]) if cs.get("sm_mhz") else None,
+                 "burst_ms_x_mhz": None}   # filled in below, once the burst region's clock summary exists
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region.
     # The way a user would drive the library from host data: three streams (upload, mixers, download)
@@ -381,6 +447,45 @@ def run_cuda(args):
         2 * (2 * tok * Cm + Cm * Cm), 2.0 * tok * Cm * Cm, "tensor")
     del px, py
 
+    # the same shape with the five prefix tokens of DINOv3 (class token + four registers) in front of the grid
+    P5 = 5
+    pq = [[t.to(dev) for t in inputs.custom_qkv(w.B, w.H, P5 + w.N, w.D, "bf16", seed=4100 + l)] for l in range(3)]
+    po = [torch.empty_like(pq[0][0]) for _ in range(3)]
+    tokp = w.B * (P5 + w.N)
+
+    def addp(name, fn, bytes_, flops, bound):
+        t_ms = time_calls(fn, K, W, stream)
+        per[name] = {"ms": t_ms, "tokens_per_s": tokp / (t_ms * 1e-3), "GBps": bytes_ / t_ms / 1e6, "TFLOPs": flops / t_ms / 1e9,
+                     "frac_hbm": bytes_ / t_ms / 1e6 / hbm, "frac_tensor": flops / t_ms / 1e9 / tf, "bound": bound}
+    bp = alg_bytes(w.B, w.H, P5 + w.N, w.D)
+    addp("L+dwc@prefix5", lambda i: jv.linear_attn(*pq[r(i)], w.Hg, w.Wg, dwc=dwc_dev, out=po[r(i)], ws=ws, prefix=P5),
+         alg_bytes(w.B, w.H, P5 + w.N, w.D, dwc=True), 0.0, "hbm")
+    addp("W@prefix5", lambda i: jv.window_attn(*pq[r(i)], w.Hg, w.Wg, WIN, WIN, out=po[r(i)], prefix=P5), bp,
+         alg_flops_attn(w.B, w.H, w.Hg, w.Wg, w.D, WIN, WIN, prefix=P5), "hbm")
+    del pq, po
+
+    # other model sizes at the 1024 x 2048 image of Tables 1 and 3 (64 x 128 token grid): 12 heads (ViT-B), 24 heads (Giant)
+    for tag, heads in (("vitb_64x128", 12), ("giant_64x128", 24)):
+        Bx, Hgx, Wgx = 4, 64, 128
+        xq = [[t.to(dev) for t in inputs.custom_qkv(Bx, heads, Hgx * Wgx, 64, "bf16", seed=8000 + heads + l)] for l in range(2)]
+        xo = [torch.empty_like(xq[0][0]) for _ in range(2)]
+        Cx = heads * 64
+        dx = {kk: (vv.to(dev) if hasattr(vv, "to") else vv) for kk, vv in inputs.dwc_weights(Cx, Cx // 8, 3, 8100 + heads).items()}
+        wsx = jv.alloc_workspace("L", jv.make_shape(xq[0][0], Hgx, Wgx), jv.make_dwc(dx, dev), dev)
+        rows = {"L+dwc": (lambda i: jv.linear_attn(*xq[i % 2], Hgx, Wgx, dwc=dx, out=xo[i % 2], ws=wsx),
+                          alg_bytes(Bx, heads, Hgx * Wgx, 64, dwc=True), 0.0, "hbm"),
+                "W": (lambda i: jv.window_attn(*xq[i % 2], Hgx, Wgx, WIN, WIN, out=xo[i % 2]),
+                      alg_bytes(Bx, heads, Hgx * Wgx, 64), alg_flops_attn(Bx, heads, Hgx, Wgx, 64, WIN, WIN), "hbm"),
+                "F": (lambda i: jv.full_attn(*xq[i % 2], out=xo[i % 2]),
+                      alg_bytes(Bx, heads, Hgx * Wgx, 64), alg_flops_attn(Bx, heads, Hgx, Wgx, 64, Hgx, Wgx), "tensor")}
+        for name, (fn, bytes_, flops, bound) in rows.items():
+            Kx = 5 if name == "F" else K
+            t_ms = time_calls(fn, Kx, 3, stream)
+            per[f"{name}@{tag}"] = {"ms": t_ms, "tokens_per_s": Bx * Hgx * Wgx / (t_ms * 1e-3), "GBps": bytes_ / t_ms / 1e6,
+                                    "TFLOPs": flops / t_ms / 1e9, "frac_hbm": bytes_ / t_ms / 1e6 / hbm,
+                                    "frac_tensor": flops / t_ms / 1e9 / tf, "bound": bound}
+        del xq, xo, wsx
+
     # ragged DepthAnythingV2-L grid (73x73, B=4): F and W with masked edge windows
     w4 = inputs.WORKLOADS["dav2_l"]
     q4 = [[t.to(dev) for t in inputs.qkv(w4, layer=l)] for l in range(3)]
@@ -409,6 +514,15 @@ def run_cuda(args):
                                                 out=louts, ws=ws5), 3, 2, stream)
     allf = time_calls(lambda i: jv.hybrid_mixers("F" * w5.n_layers, lq, lk, lv, w5.Hg, w5.Wg, WIN, WIN,
                                                  out=louts, ws=ws5), 2, 1, stream)
+    l5 = time_calls(lambda i: jv.linear_attn(lq[i % 4], lk[i % 4], lv[i % 4], w5.Hg, w5.Wg, out=lo[i % 4], ws=ws5), K, W, stream)
+    w5ms = time_calls(lambda i: jv.window_attn(lq[i % 4], lk[i % 4], lv[i % 4], w5.Hg, w5.Wg, WIN, WIN, out=lo[i % 4]), K, W, stream)
+    b5 = alg_bytes(*w5.shape)
+    per["L@hybrid24_layer"] = {"ms": l5, "tokens_per_s": w5.tokens / (l5 * 1e-3), "GBps": b5 / l5 / 1e6, "TFLOPs": 0.0,
+                               "frac_hbm": b5 / l5 / 1e6 / hbm, "frac_tensor": 0.0, "bound": "hbm"}
+    f5w = alg_flops_attn(w5.B, w5.H, w5.Hg, w5.Wg, w5.D, WIN, WIN)
+    per["W@hybrid24_layer"] = {"ms": w5ms, "tokens_per_s": w5.tokens / (w5ms * 1e-3), "GBps": b5 / w5ms / 1e6,
+                               "TFLOPs": f5w / w5ms / 1e9, "frac_hbm": b5 / w5ms / 1e6 / hbm,
+                               "frac_tensor": f5w / w5ms / 1e9 / tf, "bound": "hbm"}
     f5_flops = alg_flops_attn(w5.B, w5.H, w5.Hg, w5.Wg, w5.D, w5.Hg, w5.Wg)
     hybrid = {"schedule": inputs.HYBRID_SCHEDULE, "hybrid_ms": hyb, "all_full_ms": allf, "speedup": allf / hyb,
               "tokens_per_s_hybrid": w5.n_layers * w5.tokens / (hyb * 1e-3),
@@ -421,8 +535,9 @@ def run_cuda(args):
     # the timed region (events around the F layer of every step)
     f_ms = layer_ms[STEP_SCHEDULE.index("F")]
     f_tf = f_flops / f_ms / 1e9
+    traffic, traffic_note = measured_traffic()
     roofline = {"kernel": "attn_f4_kernel as jv_full_attn (one launch per step)", "bound": "tensor", "achieved": f_tf,
-                "peak": tf, "unit": "TFLOP/s", "frac": f_tf / tf, "traffic": ATTN_F_DRAM_BYTES,
+                "peak": tf, "unit": "TFLOP/s", "frac": f_tf / tf, "traffic": traffic, "traffic_note": traffic_note,
                 "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
                 "peak_source": peaks["source"] + " bf16 burst", "ms_per_launch": f_ms,
                 "flops_per_launch": f_flops, "alg_bytes_per_launch": alg_bytes(*w.shape),
@@ -441,6 +556,8 @@ def run_cuda(args):
         cpu = {"value": step_tokens / full_s, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
                "seconds_spent": spent}
 
+    cb = clk.summary()
+    sustained["burst_ms_x_mhz"] = (ms * cb["sm_mhz"]) if cb.get("sm_mhz") else None
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -448,7 +565,7 @@ def run_cuda(args):
                                    "one step = jv_hybrid_mixers('LWF'): L with squeeze dynamic DWC (k=3, R=128), "
                                    "W 16x16, F", "l2": "three layers' tensors (805 MB) exceed L2; "
                                    "per-mixer loops rotate over three tensor sets"},
-            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clk.summary(), "sustained": sustained, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu, "per_mixer": per, "hybrid24": hybrid,
             "peaks": peaks}
     print(json.dumps(line))
@@ -516,8 +633,12 @@ def main():
     ap.add_argument("--single", choices=["L", "L+dwc", "W", "F", "qkv_proj", "out_proj"], default=None,
                     help="time one mixer alone (used for profiler captures)")
     ap.add_argument("--workload", default="dinov3_l", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--record-traffic", default=None, metavar="CSV",
+                    help="write the DRAM-traffic record of the dominant kernel from an ncu raw-page CSV (no GPU needed)")
     args = ap.parse_args()
-    if args.single:
+    if args.record_traffic:
+        record_traffic(args.record_traffic)
+    elif args.single:
         run_single(args)
     elif args.impl == "reference":
         run_reference(args)
