@@ -247,21 +247,24 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           }
           if (!ok) break;
           tc_fence_after();
-          if (has_pv) {
+          if (elect_one()) {                 // one lane issues the step's MMAs back to back
+            if (has_pv) {
+              const uint64_t dv = smem_desc(vb);
 #pragma unroll
-            for (int ks = 0; ks < kSub / 16; ++ks)
-              mma_ts(tmem + kColO + t * kD, tmem + kColS + t * kSub + ks * 8, smem_desc(vb + ks * 2048), kIdescPV,
-                     (u > 1 || ks > 0) ? 1u : 0u);
-          }
-          if (has_qk) {
-            const uint32_t qa = sQ + t * kTileBytes;
+              for (int ks = 0; ks < kSub / 16; ++ks)
+                mma_ts_1(tmem + kColO + t * kD, tmem + kColS + t * kSub + ks * 8, desc_advance(dv, ks * 2048), kIdescPV,
+                         (u > 1 || ks > 0) ? 1u : 0u);
+            }
+            if (has_qk) {
+              const uint64_t dq = smem_desc(sQ + t * kTileBytes), dk = smem_desc(kb);
 #pragma unroll
-            for (int ks = 0; ks < kD / 16; ++ks)
-              mma_ss(tmem + kColS + t * kSub, smem_desc(qa + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
-            tc_commit(&bar->s_full[t]);
-          } else {
-            tc_commit(&bar->o_full[t]);
+              for (int ks = 0; ks < kD / 16; ++ks)
+                mma_ss_1(tmem + kColS + t * kSub, desc_advance(dq, ks * 32), desc_advance(dk, ks * 32), kIdescQK, ks > 0);
+            }
           }
+          __syncwarp();
+          if (has_qk) tc_commit(&bar->s_full[t]);
+          else tc_commit(&bar->o_full[t]);
         }
         if (!ok) break;
         if (has_pv && ((u - 1) & 1) == 1) { // both halves of the V tile are in flight or done

@@ -273,9 +273,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tc_fence_after();
       }
       const uint32_t kb = sK + s1 * kTileBytes + h * (kSub * kD * 2), qa = sQ + (2 * qb + t) * kTileBytes;
+      if (elect_one()) {                     // one lane issues the four MMAs back to back
+        const uint64_t dq = smem_desc(qa), dk = smem_desc(kb);
 #pragma unroll
-      for (int ks = 0; ks < kD / 16; ++ks)
-        mma_ss(tmem + kColS + (2 * t + h) * kSub, smem_desc(qa + ks * 32), smem_desc(kb + ks * 32), kIdescQK, ks > 0);
+        for (int ks = 0; ks < kD / 16; ++ks)
+          mma_ss_1(tmem + kColS + (2 * t + h) * kSub, desc_advance(dq, ks * 32), desc_advance(dk, ks * 32), kIdescQK, ks > 0);
+      }
+      __syncwarp();
       tc_commit(&bar->s_full[t][h]);
       if (h == 1) {
         tc_commit(&bar->k_empty[s1]);
@@ -302,10 +306,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           if (!ok) break;
           tc_fence_after();
           const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
+          if (elect_one()) {                 // one lane issues the four MMAs back to back
+            const uint64_t dv = smem_desc(vb);
 #pragma unroll
-          for (int ks = 0; ks < kSub / 16; ++ks)
-            mma_ts(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, smem_desc(vb + ks * 2048),
-                   kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
+            for (int ks = 0; ks < kSub / 16; ++ks)
+              mma_ts_1(tmem + kColO + t * kD, tmem + kColP + (2 * t + h) * (kSub / 2) + ks * 8, desc_advance(dv, ks * 2048),
+                       kIdescPV, (j > 0 || h > 0 || ks > 0) ? 1u : 0u);
+          }
+          __syncwarp();
           if (last && h == 1) tc_commit(&bar->o_full[t]);
           if (!last) ok = issue_qk(h, j + 1, it.nkt, n);                 // its commit also covers the P V just issued
           else if (nxt >= 0) ok = issue_qk(h, 0, itn.nkt, n + 1);        // first key tile of the next item
