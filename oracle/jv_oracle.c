@@ -413,3 +413,29 @@ void jvo_linear_attn_prefix(const double* q, const double* k, const double* v, d
   }
   free(wall);
 }
+
+/*
+ * Focused feature map (Eq. 3; the kernel function of the cited focused linear attention):
+ *   phi_p(x) = (||r|| / ||r^p||) r^p,   r = ReLU(x),  r^p element-wise,
+ * per token and head over the D features: a sharper direction with the norm of ReLU(x) kept.
+ * The paper prints the denominator as ||x||^p; the reading taken is the cited work's ||x^p||
+ * (with it the map is positively homogeneous, phi(a x) = a phi(x), and p = 1 is plain ReLU).
+ * A row whose ReLU is the zero vector maps to zero.  x, out: [rows][D].
+ */
+void jvo_focus_map(const double* x, double* out, int64_t rows, int64_t D, double p) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < rows; ++i) {
+    const double* xi = x + i * D;
+    double* oi = out + i * D;
+    double n1 = 0.0, np = 0.0;
+    for (int64_t e = 0; e < D; ++e) {
+      const double r = xi[e] > 0.0 ? xi[e] : 0.0;
+      const double rp = r > 0.0 ? pow(r, p) : 0.0;
+      oi[e] = rp;
+      n1 += r * r;
+      np += rp * rp;
+    }
+    const double scale = np > 0.0 ? sqrt(n1) / sqrt(np) : 0.0;
+    for (int64_t e = 0; e < D; ++e) oi[e] *= scale;
+  }
+}

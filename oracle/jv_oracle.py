@@ -48,6 +48,8 @@ def _load():
         lib.jvo_dwc_generate_prefix.argtypes = [_c_dp] * 2 + [_i64] * 7 + [_c_dp] * 4
         lib.jvo_linear_attn_prefix.argtypes = ([_c_dp] * 4 + [_i64] * 6 + [ctypes.c_double]
                                                + [_i64] * 2 + [_c_dp] * 4)
+        lib.jvo_focus_map.argtypes = [_c_dp] * 2 + [_i64] * 2 + [ctypes.c_double]
+        lib.jvo_focus_map.restype = None
         for f in (lib.jvo_full_attn, lib.jvo_window_attn, lib.jvo_dwc_generate,
                   lib.jvo_linear_attn, lib.jvo_window_attn_prefix, lib.jvo_dwc_generate_prefix,
                   lib.jvo_linear_attn_prefix):
@@ -157,6 +159,22 @@ def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None, prefix=0, _force_prefix_cod
     assert kk % 2 == 1
     call(kk, R, W1, b1, W2, b2)
     return o
+
+
+def focus_map(x, p) -> np.ndarray:
+    """Focused feature map of Eq. 3 over the last axis: (||r|| / ||r^p||) r^p with r = ReLU(x)."""
+    x = _f64(x)
+    out = np.empty_like(x)
+    _load().jvo_focus_map(_p(x), _p(out), x.size // x.shape[-1], x.shape[-1], float(p))
+    return out
+
+
+def linear_attn_focused(q, k, v, Hg, Wg, focus_p, eps=1e-6, dwc=None, prefix=0) -> np.ndarray:
+    """The linear-attention block with the focused feature map in place of ReLU (Table 1,
+    "+ DWC on V + Focusing Factor"): Eq. 2 with phi = phi_p of Eq. 3, the row normalisation and
+    Eq. 4's convolution as in linear_attn.  phi_p is non-negative, so the block equals the ReLU
+    block applied to phi_p(Q), phi_p(K): that is how it is evaluated."""
+    return linear_attn(focus_map(q, focus_p), focus_map(k, focus_p), v, Hg, Wg, eps=eps, dwc=dwc, prefix=prefix)
 
 
 def hybrid_mixers(schedule, q, k, v, Hg, Wg, win_h, win_w, scale=None, eps=1e-6, dwc=None, prefix=0):

@@ -542,3 +542,41 @@ def test_prefix_hybrid_schedule_layers_are_independent(oracle):
     assert np.array_equal(outs[0], oracle.linear_attn(qs[0], ks[0], vs[0], Hg, Wg, prefix=P))
     assert np.array_equal(outs[1], oracle.window_attn(qs[1], ks[1], vs[1], Hg, Wg, 2, 2, prefix=P))
     assert np.array_equal(outs[2], oracle.full_attn(qs[2], ks[2], vs[2]))
+
+
+# ------------------------------------------------------------------ focused feature map (Eq. 3)
+def test_focus_map_golden_and_closed_forms(oracle):
+    g = _golden("focus_map.txt")
+    got = oracle.focus_map(g["x"].reshape(3, 3), g["p"][0])
+    assert np.allclose(got.ravel(), g["phi"], atol=1e-14)
+    r = _rng(960)
+    x = r.standard_normal((5, 7, 16))
+    relu = np.maximum(x, 0)
+    assert np.array_equal(oracle.focus_map(x, 1.0), relu)                      # p = 1 is plain ReLU
+    for p in (2.0, 3.0, 2.5):
+        f = oracle.focus_map(x, p)
+        assert np.all(f >= 0)
+        assert np.abs(np.linalg.norm(f, axis=-1) - np.linalg.norm(relu, axis=-1)).max() < 1e-12   # the norm is kept
+        want = relu ** p                                                       # the direction is that of r^p
+        want *= (np.linalg.norm(relu, axis=-1) / np.linalg.norm(want, axis=-1))[..., None]
+        assert np.abs(f - want).max() < 1e-12
+        assert np.abs(oracle.focus_map(3.7 * x, p) - 3.7 * f).max() < 1e-11    # positively homogeneous
+    assert np.array_equal(oracle.focus_map(-np.abs(x), 3.0), np.zeros_like(x))
+
+
+def test_focused_linear_attention_is_the_naive_quadratic_form_with_phi(oracle):
+    """Eq. 2 with phi = phi_p written as the explicit N x N similarity, with the row normalisation."""
+    Hg, Wg, D, p = 5, 6, 8, 3.0
+    r = _rng(970)
+    q, k, v = (r.standard_normal((1, 2, Hg * Wg, D)) for _ in range(3))
+    got = oracle.linear_attn_focused(q, k, v, Hg, Wg, p, eps=0.25)
+
+    def phi(x):
+        a = np.maximum(x, 0) ** p
+        return a * (np.linalg.norm(np.maximum(x, 0), axis=-1) / np.linalg.norm(a, axis=-1))[..., None]
+
+    for h in range(2):
+        S = phi(q[0, h]) @ phi(k[0, h]).T
+        want = (S @ v[0, h]) / (S.sum(axis=1, keepdims=True) + 0.25)
+        assert np.abs(got[0, h] - want).max() < TOL
+    assert np.array_equal(oracle.linear_attn_focused(q, k, v, Hg, Wg, 1.0), oracle.linear_attn(q, k, v, Hg, Wg))
