@@ -102,8 +102,8 @@ typedef struct {
 } jv_dwc;
 
 /*
- * Bytes of scratch the given mixer needs for this shape.  mixer is 'L', 'W', 'F'
- * or 'S' (the maximum over the three, for jv_hybrid_mixers).  dwc may be NULL;
+ * Bytes of scratch the given mixer needs for this shape.  mixer is 'L', 'W', 'F',
+ * 'S' (the maximum over the three, for jv_hybrid_mixers) or 'f' (jv_linear_attn_focused).  dwc may be NULL;
  * pass the descriptor that the L call will get, since it enlarges the scratch.
  * Returns 0 on invalid arguments as well as when no scratch is needed.
  */
@@ -124,6 +124,19 @@ size_t jv_workspace_bytes(char mixer, const jv_shape* shape, const jv_dwc* dwc);
  */
 jv_status jv_linear_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
                          float eps, const jv_dwc* dwc, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * L with the focused feature map in place of ReLU (Eq. 3; the variant "+ DWC on V + Focusing
+ * Factor" of Table 1, which the paper measures and sets aside for its cost):
+ *   phi_p(x) = (||r|| / ||r^p||) r^p,  r = relu(x),  r^p element-wise over the D features of a token,
+ * (the denominator read as in the work Eq. 3 cites: the norm of the element-wise power), then
+ * exactly jv_linear_attn with phi_p(q), phi_p(k) in place of relu(q), relu(k).  focus_p in (0, 16];
+ * focus_p = 1 is jv_linear_attn.  phi_p(q) and phi_p(k) are formed by one extra streaming pass
+ * and kept in the caller's scratch: ws must cover jv_workspace_bytes('f', shape, dwc).
+ */
+jv_status jv_linear_attn_focused(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,
+                                 float eps, float focus_p, const jv_dwc* dwc, void* ws, size_t ws_bytes,
+                                 void* cuda_stream);
 
 /*
  * L without caller scratch.  (The paper has no counterpart: this entry point exists for

@@ -191,6 +191,8 @@ size_t jv_workspace_bytes(char mixer, const jv_shape* shape, const jv_dwc* dwc) 
     case 'L':
     case 'S':
       return lin_plan(*shape, dwc).total;   // W and F need no scratch
+    case 'f':   // the linear block with the focused feature map: two tensors for phi(q), phi(k) behind the block's own scratch
+      return align_up(lin_plan(*shape, dwc).total, 256) + 2 * align_up(tensor_bytes(shape), 256);
     case 'W':
     case 'F':
       return 0;
@@ -209,6 +211,23 @@ jv_status jv_linear_attn(const void* q, const void* k, const void* v, void* o, c
   if ((st = check_ws(ws, ws_bytes, lin_plan(*shape, dwc).total)) != JV_OK) return st;
   if ((st = check_device()) != JV_OK) return st;
   return run_linear(q, k, v, o, shape, eps, dwc, ws, (cudaStream_t)cuda_stream);
+}
+
+jv_status jv_linear_attn_focused(const void* q, const void* k, const void* v, void* o, const jv_shape* shape, float eps,
+                                 float focus_p, const jv_dwc* dwc, void* ws, size_t ws_bytes, void* cuda_stream) {
+  jv_status st = check_shape(shape);
+  if (st != JV_OK) return st;
+  if ((st = check_tensors(q, k, v, o, shape)) != JV_OK) return st;
+  if (!(eps >= 0.f) || !(focus_p > 0.f) || !(focus_p <= 16.f)) return JV_ERR_INVALID_ARG;
+  if ((st = check_dwc(dwc)) != JV_OK) return st;
+  const size_t lin = align_up(lin_plan(*shape, dwc).total, 256), tb = align_up(tensor_bytes(shape), 256);
+  if ((st = check_ws(ws, ws_bytes, lin + 2 * tb)) != JV_OK) return st;
+  if ((st = check_device()) != JV_OK) return st;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  void* qf = (char*)ws + lin;
+  void* kf = (char*)ws + lin + tb;
+  if ((st = from_cuda(launch_focus_map(q, k, qf, kf, *shape, focus_p, stream))) != JV_OK) return st;
+  return run_linear(qf, kf, v, o, shape, eps, dwc, ws, stream);
 }
 
 jv_status jv_window_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* shape,

@@ -122,6 +122,9 @@ cudaError_t launch_dwc_generator(const LinArgs& a, const LinPlan& p, const float
 cudaError_t launch_lin_reduce(const float* partial, float* state, int nchunk, int state_elems, size_t total,
                               cudaStream_t st);
 
+// Focused feature map of Eq. 3 over every token row of q and k -> qf, kf (same shape and type)
+cudaError_t launch_focus_map(const void* q, const void* k, void* qf, void* kf, const jv_shape& s, float p, cudaStream_t st);
+
 // Projections either side of a mixer (bf16, D == 64): qkv = true computes q, k, v (d0, d1, d2)
 // from x [B, N, C]; qkv = false computes y (d0) [B, N, C] from x = o [B, H, N, 64].
 bool proj_tc_available();

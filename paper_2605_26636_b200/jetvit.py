@@ -51,6 +51,8 @@ def lib() -> ctypes.CDLL:
         L.jv_workspace_bytes.argtypes = [ctypes.c_char, shp, dwc]
         L.jv_workspace_bytes.restype = sz
         L.jv_linear_attn.argtypes = [vp, vp, vp, vp, shp, f32, dwc, vp, sz, vp]
+        L.jv_linear_attn_focused.argtypes = [vp, vp, vp, vp, shp, f32, f32, dwc, vp, sz, vp]
+        L.jv_linear_attn_focused.restype = ctypes.c_int
         L.jv_linear_attn_static.argtypes = [vp, vp, vp, vp, shp, f32, dwc, vp]
         L.jv_linear_attn_static.restype = ctypes.c_int
         L.jv_window_attn.argtypes = [vp, vp, vp, vp, shp, i32, i32, f32, vp, sz, vp]
@@ -172,6 +174,26 @@ def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict
         st = lib().jv_linear_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
                                   float(eps), ctypes.byref(d) if d is not None else None, wp, wn, _stream(stream))
     _raise(st, "jv_linear_attn")
+    return out
+
+
+def linear_attn_focused(q, k, v, Hg: int, Wg: int, focus_p: float, eps: float = 1e-6, dwc: Optional[dict] = None,
+                        out=None, ws: Optional[torch.Tensor] = None, stream=None, prefix: int = 0) -> torch.Tensor:
+    """jv_linear_attn_focused: the linear block with the focused feature map of Eq. 3 (power focus_p)."""
+    out = torch.empty_like(q) if out is None else out
+    _check_tensors(q, k, v, out)
+    shape = make_shape(q, Hg, Wg, prefix)
+    d = make_dwc(dwc, q.device)
+    with torch.cuda.device(q.device):
+        if ws is None:
+            ws = alloc_workspace("f", shape, d, q.device)
+            if ws is not None and stream is not None:
+                ws.record_stream(stream)
+        wp, wn = _ws_args(ws)
+        st = lib().jv_linear_attn_focused(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), ctypes.byref(shape),
+                                          float(eps), float(focus_p), ctypes.byref(d) if d is not None else None, wp, wn,
+                                          _stream(stream))
+    _raise(st, "jv_linear_attn_focused")
     return out
 
 

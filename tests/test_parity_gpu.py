@@ -394,3 +394,29 @@ def test_runtime_errors_on_device(jv):
     with pytest.raises(jv.JetVitError):
         jv.full_attn(q, k, v, out=q)
     assert jv.device_status() == jv.JV_OK
+
+
+# ------------------------------------------------------------------ Table 1 variant: focused feature map (Eq. 3)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("p", [2.0, 3.0, 2.5])
+def test_linear_with_focused_feature_map(jv, oracle, both_paths, dtype, p):
+    B, H, Hg, Wg = 2, 2, 21, 18
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, 64, dtype, seed=int(10 * p))
+    d = inputs.dwc_weights(H * 64, 16, 3, 31)
+    dq, dk, dv = _dev((q, k, v))
+    out = jv.linear_attn_focused(dq, dk, dv, Hg, Wg, p, dwc=dwc_to_device(d, DEV))
+    assert rel_err(out, oracle.linear_attn_focused(q, k, v, Hg, Wg, p, dwc=d)) <= TOL[dtype]
+    out = jv.linear_attn_focused(dq, dk, dv, Hg, Wg, p)
+    assert rel_err(out, oracle.linear_attn_focused(q, k, v, Hg, Wg, p)) <= TOL[dtype]
+
+
+def test_focused_feature_map_full_size_and_power_one(jv, oracle):
+    w = inputs.WORKLOADS["dinov3_l"]
+    q, k, v = inputs.qkv(w)
+    dq, dk, dv = _dev((q, k, v))
+    out = jv.linear_attn_focused(dq, dk, dv, w.Hg, w.Wg, 3.0).cpu()
+    for b, h in sample_heads(w.B, w.H, 6, 33):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        assert rel_err(out[sl], oracle.linear_attn_focused(q[sl], k[sl], v[sl], w.Hg, w.Wg, 3.0)) <= TOL["bf16"], (b, h)
+    # p = 1 is the ReLU block
+    assert torch.equal(jv.linear_attn_focused(dq, dk, dv, w.Hg, w.Wg, 1.0), jv.linear_attn(dq, dk, dv, w.Hg, w.Wg))
