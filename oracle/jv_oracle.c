@@ -439,3 +439,56 @@ void jvo_focus_map(const double* x, double* out, int64_t rows, int64_t D, double
     for (int64_t e = 0; e < D; ++e) oi[e] *= scale;
   }
 }
+
+/*
+ * Token-wise dynamic depth-wise convolution (Sec. 3.2.1 "JetViT Linear Attention Block", the
+ * variant the paper tries first and drops for its cost; Table 1 "+ Token-wise Dynamic DWC"):
+ * the kernel generator, the same two-layer MLP with SiLU, is fed with each token's own value
+ * vector instead of the pooled one and emits one set of kernels per token:
+ *   for grid token i of sample b, with v_i in R^C its value vector over all heads (c = h*D + e):
+ *     hid_i = SiLU(W1 v_i + b1),   w_i = W2 hid_i + b2  viewed as [C][k][k],
+ *     DW_i[c] = sum_{dy,dx} w_i[c][dy][dx] * V[b][c][(y + dy - p, x + dx - p)]   (zero outside the grid)
+ *   O_i = LA_i + DW_i.
+ * The paper gives no formula; this is the reading: the kernels of the OUTPUT position are
+ * applied to that position's neighbourhood, everything else as in the squeeze dynamic variant
+ * (prefix tokens: attention only).  q, k, v, o: [B*H][P + Hg*Wg][D].
+ */
+void jvo_linear_attn_tokenwise(const double* q, const double* k, const double* v, double* o,
+                               int64_t B, int64_t H, int64_t P, int64_t Hg, int64_t Wg, int64_t D, double eps,
+                               int64_t dwc_k, int64_t R, const double* W1, const double* b1,
+                               const double* W2, const double* b2) {
+  const int64_t N = Hg * Wg, T = P + N, C = H * D, kk = dwc_k * dwc_k, pad = (dwc_k - 1) / 2;
+  jvo_linear_attn_prefix(q, k, v, o, B, H, P, Hg, Wg, D, eps, 0, 0, 0, 0, 0, 0);   /* LA_i for every token */
+#pragma omp parallel
+  {
+    double* vi = (double*)malloc(sizeof(double) * (size_t)C);
+    double* hid = (double*)malloc(sizeof(double) * (size_t)(R > 0 ? R : 1));
+#pragma omp for collapse(2) schedule(dynamic, 4)
+    for (int64_t b = 0; b < B; ++b)
+      for (int64_t i = 0; i < N; ++i) {
+        const int64_t y = i / Wg, x = i % Wg;
+        for (int64_t c = 0; c < C; ++c) vi[c] = v[((b * H + c / D) * T + P + i) * D + c % D];
+        for (int64_t r = 0; r < R; ++r) {
+          double acc = b1 ? b1[r] : 0.0;
+          for (int64_t c = 0; c < C; ++c) acc += W1[r * C + c] * vi[c];
+          hid[r] = silu(acc);
+        }
+        for (int64_t c = 0; c < C; ++c) {
+          const double* vg = v + ((b * H + c / D) * T + P) * D + c % D;   /* channel c of the grid, stride D */
+          double dw = 0.0;
+          for (int64_t dy = 0; dy < dwc_k; ++dy)
+            for (int64_t dx = 0; dx < dwc_k; ++dx) {
+              const int64_t yy = y + dy - pad, xx = x + dx - pad;
+              if (yy < 0 || yy >= Hg || xx < 0 || xx >= Wg) continue;
+              const int64_t t = c * kk + dy * dwc_k + dx;
+              double w = b2 ? b2[t] : 0.0;
+              for (int64_t r = 0; r < R; ++r) w += W2[t * R + r] * hid[r];
+              dw += w * vg[(yy * Wg + xx) * D];
+            }
+          o[((b * H + c / D) * T + P + i) * D + c % D] += dw;
+        }
+      }
+    free(vi);
+    free(hid);
+  }
+}

@@ -48,6 +48,8 @@ def _load():
         lib.jvo_dwc_generate_prefix.argtypes = [_c_dp] * 2 + [_i64] * 7 + [_c_dp] * 4
         lib.jvo_linear_attn_prefix.argtypes = ([_c_dp] * 4 + [_i64] * 6 + [ctypes.c_double]
                                                + [_i64] * 2 + [_c_dp] * 4)
+        lib.jvo_linear_attn_tokenwise.argtypes = lib.jvo_linear_attn_prefix.argtypes
+        lib.jvo_linear_attn_tokenwise.restype = None
         lib.jvo_focus_map.argtypes = [_c_dp] * 2 + [_i64] * 2 + [ctypes.c_double]
         lib.jvo_focus_map.restype = None
         for f in (lib.jvo_full_attn, lib.jvo_window_attn, lib.jvo_dwc_generate,
@@ -145,6 +147,15 @@ def linear_attn(q, k, v, Hg, Wg, eps=1e-6, dwc=None, prefix=0, _force_prefix_cod
 
     if dwc is None:
         call(0, 0, None, None, None, None)
+        return o
+    if dwc.get("token_wise"):     # one set of kernels per token (Table 1 "+ Token-wise Dynamic DWC")
+        kk, R = int(dwc["k"]), int(dwc["R"])
+        W1, W2 = _f64(dwc["W1"]), _f64(dwc["W2"])
+        b1 = None if dwc.get("b1") is None else _f64(dwc["b1"])
+        b2 = None if dwc.get("b2") is None else _f64(dwc["b2"])
+        assert R > 0 and W1.shape == (R, H * D) and W2.shape == (H * D * kk * kk, R)
+        _load().jvo_linear_attn_tokenwise(_p(q), _p(k), _p(v), _p(o), B, H, prefix, Hg, Wg, D, float(eps),
+                                          kk, R, _p(W1), _p(b1), _p(W2), _p(b2))
         return o
     kk, R = int(dwc["k"]), int(dwc["R"])
     C = H * D

@@ -580,3 +580,50 @@ def test_focused_linear_attention_is_the_naive_quadratic_form_with_phi(oracle):
         want = (S @ v[0, h]) / (S.sum(axis=1, keepdims=True) + 0.25)
         assert np.abs(got[0, h] - want).max() < TOL
     assert np.array_equal(oracle.linear_attn_focused(q, k, v, Hg, Wg, 1.0), oracle.linear_attn(q, k, v, Hg, Wg))
+
+
+# ------------------------------------------------------------------ token-wise dynamic convolution (Table 1)
+def _tokenwise_dwc(ksz, R, C, seed):
+    r = _rng(seed)
+    return {"k": ksz, "R": R, "W1": 0.3 * r.standard_normal((R, C)), "b1": 0.1 * r.standard_normal(R),
+            "W2": 0.3 * r.standard_normal((C * ksz * ksz, R)), "b2": 0.1 * r.standard_normal(C * ksz * ksz),
+            "token_wise": 1}
+
+
+@pytest.mark.parametrize("ksz", [3, 5])
+def test_tokenwise_dwc_against_library_unfold(oracle, ksz):
+    """Kernels per token from torch's linear + silu + linear on the token's value vector; the
+    neighbourhoods from torch's unfold (zero padding); the product summed over the taps."""
+    B, H, P, Hg, Wg, D, R = 2, 2, 3, 5, 4, 4, 3
+    C, N = H * D, Hg * Wg
+    r = _rng(980 + ksz)
+    q, k, v = (r.standard_normal((B, H, P + N, D)) for _ in range(3))
+    d = _tokenwise_dwc(ksz, R, C, 981)
+    got = oracle.linear_attn(q, k, v, Hg, Wg, dwc=d, prefix=P)
+    la = oracle.linear_attn(q, k, v, Hg, Wg, prefix=P)
+    vt = torch.from_numpy(v[:, :, P:, :]).permute(0, 2, 1, 3).reshape(B, N, C)                 # token vectors, c = h*D + e
+    hid = torch.nn.functional.silu(torch.nn.functional.linear(vt, torch.from_numpy(d["W1"]), torch.from_numpy(d["b1"])))
+    w = torch.nn.functional.linear(hid, torch.from_numpy(d["W2"]), torch.from_numpy(d["b2"])).reshape(B, N, C, ksz * ksz)
+    img = vt.permute(0, 2, 1).reshape(B, C, Hg, Wg)
+    nb = torch.nn.functional.unfold(img, ksz, padding=ksz // 2).reshape(B, C, ksz * ksz, N).permute(0, 3, 1, 2)   # [B, N, C, taps]
+    dw = (w * nb).sum(-1)                                                                      # [B, N, C]
+    dw = dw.reshape(B, N, H, D).permute(0, 2, 1, 3).numpy()
+    assert np.abs(got[:, :, P:] - (la[:, :, P:] + dw)).max() < 1e-10
+    assert np.array_equal(got[:, :, :P], la[:, :, :P])                                         # prefix tokens: attention only
+
+
+def test_tokenwise_dwc_reduces_to_the_pooled_and_static_variants(oracle):
+    """When every grid token carries the same value vector, each token's kernels are the kernels the
+    pooled (squeeze) generator gives; with W2 = 0 the kernels are b2, the static convolution."""
+    B, H, Hg, Wg, D, R = 1, 2, 4, 5, 4, 3
+    C, N = H * D, Hg * Wg
+    r = _rng(990)
+    q, k = (r.standard_normal((B, H, N, D)) for _ in range(2))
+    v = np.broadcast_to(r.standard_normal((B, H, 1, D)), (B, H, N, D)).copy()
+    d = _tokenwise_dwc(3, R, C, 991)
+    squeeze = dict(d, token_wise=0)
+    assert np.abs(oracle.linear_attn(q, k, v, Hg, Wg, dwc=d) - oracle.linear_attn(q, k, v, Hg, Wg, dwc=squeeze)).max() < 1e-11
+    v2 = r.standard_normal((B, H, N, D))
+    d0 = dict(d, W2=np.zeros_like(d["W2"]))
+    static = {"k": 3, "R": 0, "b2": d["b2"]}
+    assert np.abs(oracle.linear_attn(q, k, v2, Hg, Wg, dwc=d0) - oracle.linear_attn(q, k, v2, Hg, Wg, dwc=static)).max() < 1e-11
