@@ -91,6 +91,14 @@ typedef struct {
  * (Sec. 3.2.1, Table 1 "DWC"): no generator, b2 holds the kernels themselves
  * ([C, k, k], shared by every sample and required); W1, b1 and W2 are ignored
  * and may be NULL.
+ *
+ * token_wise = 1 selects the token-wise dynamic convolution the paper tries first and sets
+ * aside for its cost (Sec. 3.2.1, Table 1 "+ Token-wise Dynamic DWC"): the same generator
+ * (R > 0) is fed with every grid token's own value vector instead of the pooled one and
+ * gives that token its own kernels, which are applied to the token's neighbourhood:
+ *   w_i = W2 SiLU(W1 v_i + b1) + b2,   o_i += sum_taps w_i[c][dy][dx] V[(y+dy-p, x+dx-p)][c].
+ * The kernels of all tokens pass through the caller's scratch: jv_workspace_bytes() grows by
+ * about 2 * B * N * C * k * k bytes.
  */
 typedef struct {
   int32_t k;       /* odd kernel edge: 3 or 5 */
@@ -99,6 +107,7 @@ typedef struct {
   const float* b1; /* [R] or NULL */
   const float* W2; /* [C*k*k, R] */
   const float* b2; /* [C*k*k] or NULL */
+  int32_t token_wise; /* 0: one set of kernels per sample from the pooled V; 1: one set per token */
 } jv_dwc;
 
 /*

@@ -52,6 +52,8 @@ jv_status check_dwc(const jv_dwc* d) {
   if (!d) return JV_OK;
   if (d->k != 3 && d->k != 5) return JV_ERR_INVALID_ARG;
   if (d->R < 0 || d->R > 1024) return JV_ERR_INVALID_ARG;
+  if (d->token_wise != 0 && d->token_wise != 1) return JV_ERR_INVALID_ARG;
+  if (d->token_wise && d->R == 0) return JV_ERR_INVALID_ARG;  // per-token kernels need the generator
   if (d->R == 0) return d->b2 ? JV_OK : JV_ERR_INVALID_ARG;   // static kernels live in b2
   if (!d->W1 || !d->W2) return JV_ERR_INVALID_ARG;
   return JV_OK;

@@ -78,6 +78,9 @@ struct LinPlan {
   int chunk_tokens;  // tokens per phase-1 chunk
   int nchunk;        // chunks per (batch, head)
   size_t off_partial, off_state, off_hidden, off_kernel, total;  // byte offsets into ws
+  // token-wise dynamic convolution on the tensor-core path: bf16 copies of W1, W2, the hidden layer
+  // [B, ntok, R] and the kernels of all tokens as planes [B, C*k*k/64, ntok, 64] (bf16)
+  size_t off_tok_w1, off_tok_w2, off_tok_hidden, off_tok_kernel;
 };
 LinPlan lin_plan(const jv_shape& s, const jv_dwc* dwc);
 
@@ -124,6 +127,21 @@ cudaError_t launch_lin_reduce(const float* partial, float* state, int nchunk, in
 
 // Focused feature map of Eq. 3 over every token row of q and k -> qf, kf (same shape and type)
 cudaError_t launch_focus_map(const void* q, const void* k, void* qf, void* kf, const jv_shape& s, float p, cudaStream_t st);
+
+// Token-wise dynamic convolution (Table 1): o (which holds the attention output) += the convolution
+// of V with every grid token's own kernels.  Generic: everything per token on the fly, any type.
+cudaError_t launch_dwc_tokenwise_generic(const LinArgs& a, cudaStream_t st);
+// bf16, head_dim 64, 3 x 3, R a multiple of 64: generator as two tensor-core GEMMs, then the convolution
+bool dwc_tokenwise_fast_supported(const LinArgs& a);
+cudaError_t launch_dwc_tokenwise_fast(const LinArgs& a, const LinPlan& p, int* status, cudaStream_t st);
+// the projection GEMM kernel on its own terms: D = act(A W^T + bias), bf16, fp32 accumulation.
+//   planes_in:  A is [B, a_planes, N, 64] (K block kb = plane kb % a_planes), else A is [B, N, 64 * kblocks]
+//   planes_out: D is [B, F / 64, N, 64] (feature block fb = plane fb), else D is [B, N, F]
+//   W: [F, 64 * kblocks], bias fp32 [F] or null, silu: apply x / (1 + exp(-x)) to the result;
+//   f16_in: A and W hold fp16 instead of bf16; f16_out: D is stored as fp16 instead of bf16
+cudaError_t launch_proj_gemm(bool planes_in, bool planes_out, const void* A, const void* W, const float* bias, void* D, int B,
+                             int N, int kblocks, int a_planes, int F, bool silu, bool f16_in, bool f16_out, int* status,
+                             cudaStream_t st);
 
 // Projections either side of a mixer (bf16, D == 64): qkv = true computes q, k, v (d0, d1, d2)
 // from x [B, N, C]; qkv = false computes y (d0) [B, N, C] from x = o [B, H, N, 64].

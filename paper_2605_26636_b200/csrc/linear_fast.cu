@@ -680,6 +680,7 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
 }  // namespace
 
 bool linear_fast_supported(const LinArgs& a) {
+  if (a.dwc && a.dwc->token_wise && !dwc_tokenwise_fast_supported(a)) return false;
   if (a.dwc && a.s.P > 0 && a.dwc->k != 3) return false;   // prefix tokens + 5 x 5 kernels: the generic kernels
   return a.s.dtype == JV_BF16 && a.s.D == kD && encode_fn() != nullptr;
 }
@@ -691,6 +692,15 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   float* partial = (float*)(ws + p.off_partial);
   int* status = device_status_ptr();
   if (!status) return cudaErrorUnknown;
+  if (a.dwc && a.dwc->token_wise) {
+    // token-wise dynamic convolution: the attention proper as without a convolution, then o += the
+    // convolution of V with every token's own kernels (generator as two tensor-core GEMMs)
+    LinArgs plain = a;
+    plain.dwc = nullptr;
+    const cudaError_t e0 = launch_linear_fast(plain, p, st);
+    if (e0 != cudaSuccess) return e0;
+    return launch_dwc_tokenwise_fast(a, p, status, st);
+  }
 
   CUtensorMap mq, mk, mv, mo;
   if (!make_map_tokens(&mq, a.q, BH, N, kApplyTok, N) || !make_map_tokens(&mk, a.k, BH, N, kTileTok, N) ||

@@ -29,7 +29,14 @@ LinPlan lin_plan(const jv_shape& s, const jv_dwc* dwc) {
   p.off_state = off;   off += align_up((size_t)BH * p.state_elems * sizeof(float), 256);
   p.off_hidden = off;
   p.off_kernel = off;
-  if (dwc) {
+  p.off_tok_w1 = p.off_tok_w2 = p.off_tok_hidden = p.off_tok_kernel = off;
+  if (dwc && dwc->token_wise) {
+    const size_t C = (size_t)s.H * s.D, F = C * dwc->k * dwc->k;
+    p.off_tok_w1 = off;     off += align_up((size_t)dwc->R * C * 2 * 2, 256);   // bf16 pair (hi | lo) per value
+    p.off_tok_w2 = off;     off += align_up(F * dwc->R * 2, 256);
+    p.off_tok_hidden = off; off += align_up((size_t)s.B * N * dwc->R * 2, 256);
+    p.off_tok_kernel = off; off += align_up((size_t)s.B * N * F * 2, 256);
+  } else if (dwc) {
     off += align_up((size_t)s.B * dwc->R * sizeof(float), 256);
     p.off_kernel = off;
     off += align_up((size_t)s.B * s.H * s.D * dwc->k * dwc->k * sizeof(float), 256);
@@ -205,7 +212,8 @@ cudaError_t launch_generic_t(const LinArgs& a, const LinPlan& p, cudaStream_t st
   lin_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(partial, state, p.nchunk, p.state_elems, total);
   count_launch();
   const float* dw = nullptr;
-  if (a.dwc) {
+  const bool token_wise = a.dwc && a.dwc->token_wise;
+  if (a.dwc && !token_wise) {
     cudaError_t e = launch_dwc_generator(a, p, state + s.D * p.D1, p.state_elems, st);
     if (e != cudaSuccess) return e;
     dw = (const float*)(ws + p.off_kernel);
@@ -215,6 +223,7 @@ cudaError_t launch_generic_t(const LinArgs& a, const LinPlan& p, cudaStream_t st
       (const T*)a.q, (const T*)a.v, (T*)a.o, state, dw, s.H, s.P, s.Hg, s.Wg, s.D, p.state_elems, a.eps,
       a.dwc ? a.dwc->k : 0);
   count_launch();
+  if (token_wise) return launch_dwc_tokenwise_generic(a, st);   // o += per-token kernels applied to V
   return cudaGetLastError();
 }
 

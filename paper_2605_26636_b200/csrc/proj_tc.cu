@@ -58,10 +58,19 @@ struct ProjParams {
   int H;                   // heads
   int fblocks;             // features / 64
   int N;                   // tokens per batch element
+  int silu;                // 1: x / (1 + exp(-x)) on the result (the kernel generator's hidden layer)
+  int out_f16;             // 1: the result is stored as fp16 instead of bf16 (same size; the generator's intermediates)
+  uint32_t idesc;          // instruction descriptor: M128 N256, both operands K-major, bf16 or fp16 operands
 };
 
-// Instruction descriptor: M128 N256, both operands K-major
+// Instruction descriptor: M128 N256, both operands K-major; bf16 operands, or fp16 ones (format 0 in both fields)
 constexpr uint32_t kIdesc = idesc(kBM, kBN, 0);
+constexpr uint32_t kIdescF16 = kIdesc & ~((1u << 7) | (1u << 10));
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
 
 struct Tile {
   int b, tok0, f0;   // batch element, first token, first feature
@@ -134,7 +143,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           const uint32_t dst = sRing + s * kStageBytes;
           mbar_expect_tx(&bar->full[s], kStageBytes);
           if (kQKV) tma_load_3d(dst, &mapA, &bar->full[s], kb * kD, t.tok0, t.b);
-          else tma_load_3d(dst, &mapA, &bar->full[s], 0, t.tok0, t.b * p.H + kb);
+          else tma_load_3d(dst, &mapA, &bar->full[s], 0, t.tok0, t.b * p.H + kb % p.H);   // (more K blocks than planes: A repeats)
           tma_load_2d(dst + kABytes, &mapB, &bar->full[s], kb * kD, t.f0);
         }
         __syncwarp();
@@ -166,7 +175,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         const uint32_t sa = sRing + s * kStageBytes, sb = sa + kABytes;
 #pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks)
-          mma_ss(d, smem_desc(sa + ks * 32), smem_desc(sb + ks * 32), kIdesc, (kb > 0 || ks > 0) ? 1u : 0u);
+          mma_ss(d, smem_desc(sa + ks * 32), smem_desc(sb + ks * 32), p.idesc, (kb > 0 || ks > 0) ? 1u : 0u);
         tc_commit(&bar->empty[s]);
         if (++s == kStages) { s = 0; ph ^= 1; }
       }
@@ -204,7 +213,24 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
           uint32_t v[32];
           tmem_ld32(tmem + lane_base + a * kBN + j * kD + c * 32, v);
           tmem_wait_ld(v);
-          if (p.bias) {
+          if (p.silu) {
+#pragma unroll
+            for (int i2 = 0; i2 < 32; ++i2) {
+              const float z = __uint_as_float(v[i2]) + (p.bias ? __ldg(p.bias + fb * kD + c * 32 + i2) : 0.f);
+              v[i2] = __float_as_uint(z / (1.f + __expf(-z)));
+            }
+#pragma unroll
+            for (int i2 = 0; i2 < 16; ++i2)
+              ob[16 * c + i2] = p.out_f16 ? pack_f16(__uint_as_float(v[2 * i2]), __uint_as_float(v[2 * i2 + 1]))
+                                          : pack_bf16(__uint_as_float(v[2 * i2]), __uint_as_float(v[2 * i2 + 1]));
+          } else if (p.out_f16) {
+#pragma unroll
+            for (int i2 = 0; i2 < 16; ++i2) {
+              const float b0 = p.bias ? __ldg(p.bias + fb * kD + c * 32 + 2 * i2) : 0.f;
+              const float b1 = p.bias ? __ldg(p.bias + fb * kD + c * 32 + 2 * i2 + 1) : 0.f;
+              ob[16 * c + i2] = pack_f16(__uint_as_float(v[2 * i2]) + b0, __uint_as_float(v[2 * i2 + 1]) + b1);
+            }
+          } else if (p.bias) {
             const float4* b4 = reinterpret_cast<const float4*>(p.bias + fb * kD + c * 32);
 #pragma unroll
             for (int i4 = 0; i4 < 8; ++i4) {
@@ -284,6 +310,56 @@ bool map2(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t rows, uint32
 
 bool proj_tc_available() { return encode_fn() != nullptr; }
 
+static cudaError_t proj_opt_in() {   // > 48 KB of dynamic shared memory: a per-device function attribute
+  static OncePerDevice once;
+  return once.run([] {
+    cudaError_t r = cudaFuncSetAttribute(proj_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (r == cudaSuccess)
+      r = cudaFuncSetAttribute(proj_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    return r;
+  });
+}
+
+// The kernel on its own terms (see common.cuh).  kQKV of the kernel means "A is [B, N, K]" for the loads
+// and "D is planes" for the stores, which go together in the two projections; the other two
+// combinations are reached through the plane count: with one K block per "head" ... the generator's
+// GEMMs need A planes -> D rows (the out form, as it is) and A rows -> D planes (the qkv form with
+// every feature block a plane of its own: H := F / 64, so that "which" is always 0).
+cudaError_t launch_proj_gemm(bool planes_in, bool planes_out, const void* A, const void* W, const float* bias, void* D, int B,
+                             int N, int kblocks, int a_planes, int F, bool silu, bool f16_in, bool f16_out, int* status,
+                             cudaStream_t st) {
+  if (!encode_fn() || planes_in == planes_out || F % kD != 0) return cudaErrorNotSupported;
+  const uint64_t K = (uint64_t)kblocks * kD;
+  CUtensorMap ma, mb, md;
+  bool ok = map2(&mb, W, K, (uint64_t)F, kBN);
+  if (planes_in) ok = ok && map3(&ma, A, kD, (uint64_t)N, (uint64_t)B * a_planes, kBM) && map3(&md, D, (uint64_t)F, (uint64_t)N, (uint64_t)B, 32);
+  else ok = ok && map3(&ma, A, K, (uint64_t)N, (uint64_t)B, kBM) && map3(&md, D, kD, (uint64_t)N, (uint64_t)B * (F / kD), 32);
+  if (!ok) return cudaErrorInvalidValue;
+  cudaError_t e = proj_opt_in();
+  if (e != cudaSuccess) return e;
+  const int num_sms = device_sm_count();
+  ProjParams p;
+  p.bias = bias;
+  p.status = status;
+  p.tiles_m_per_batch = ceil_div(N, kBM);
+  p.tiles_n = ceil_div(F, kBN);
+  const int64_t total = (int64_t)B * p.tiles_m_per_batch * p.tiles_n;
+  if (total > 0x7fffffffll) return cudaErrorInvalidValue;
+  p.total_tiles = (int)total;
+  p.kblocks = kblocks;
+  p.H = planes_in ? a_planes : F / kD;
+  p.fblocks = F / kD;
+  p.N = N;
+  p.silu = silu ? 1 : 0;
+  p.out_f16 = f16_out ? 1 : 0;
+  p.idesc = f16_in ? kIdescF16 : kIdesc;
+  const int grid = p.total_tiles < num_sms ? p.total_tiles : num_sms;
+  if (planes_in) proj_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, md, md, md, p);
+  else proj_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, md, md, md, p);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_proj_tc(bool qkv, const void* x, const void* w, const float* bias, void* d0, void* d1, void* d2,
                            const jv_shape& s, int* status, cudaStream_t st) {
   if (!encode_fn()) return cudaErrorNotSupported;
@@ -301,13 +377,7 @@ cudaError_t launch_proj_tc(bool qkv, const void* x, const void* w, const float* 
   }
   if (!ok) return cudaErrorInvalidValue;
 
-  static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
-  cudaError_t e = smem_opt_in.run([] {
-    cudaError_t r = cudaFuncSetAttribute(proj_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (r == cudaSuccess)
-      r = cudaFuncSetAttribute(proj_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    return r;
-  });
+  cudaError_t e = proj_opt_in();
   if (e != cudaSuccess) return e;
   const int num_sms = device_sm_count();
   ProjParams p;
@@ -322,6 +392,9 @@ cudaError_t launch_proj_tc(bool qkv, const void* x, const void* w, const float* 
   p.H = s.H;
   p.fblocks = (int)(features / kD);
   p.N = (int)N;
+  p.silu = 0;
+  p.out_f16 = 0;
+  p.idesc = kIdesc;
   const int grid = p.total_tiles < num_sms ? p.total_tiles : num_sms;
   if (qkv) proj_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, md0, md1, md2, p);
   else proj_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(ma, mb, md0, md1, md2, p);

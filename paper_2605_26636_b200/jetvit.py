@@ -26,7 +26,8 @@ class JvShape(ctypes.Structure):
 
 class JvDwc(ctypes.Structure):
     _fields_ = [("k", ctypes.c_int32), ("R", ctypes.c_int32), ("W1", ctypes.c_void_p),
-                ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p)]
+                ("b1", ctypes.c_void_p), ("W2", ctypes.c_void_p), ("b2", ctypes.c_void_p),
+                ("token_wise", ctypes.c_int32)]
 
 
 class JetVitError(RuntimeError):
@@ -131,7 +132,8 @@ def make_dwc(d: Optional[dict], device) -> Optional[JvDwc]:
         if t is None or not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
             raise ValueError(f"dwc[{key!r}] must be a contiguous fp32 CUDA tensor")
     ptr = lambda t: None if t is None else t.data_ptr()
-    return JvDwc(int(d["k"]), int(d["R"]), ptr(d.get("W1")), ptr(d.get("b1")), ptr(d.get("W2")), ptr(d.get("b2")))
+    return JvDwc(int(d["k"]), int(d["R"]), ptr(d.get("W1")), ptr(d.get("b1")), ptr(d.get("W2")), ptr(d.get("b2")),
+                 int(d.get("token_wise", 0)))
 
 
 def _stream(stream) -> int:

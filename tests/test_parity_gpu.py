@@ -420,3 +420,32 @@ def test_focused_feature_map_full_size_and_power_one(jv, oracle):
         assert rel_err(out[sl], oracle.linear_attn_focused(q[sl], k[sl], v[sl], w.Hg, w.Wg, 3.0)) <= TOL["bf16"], (b, h)
     # p = 1 is the ReLU block
     assert torch.equal(jv.linear_attn_focused(dq, dk, dv, w.Hg, w.Wg, 1.0), jv.linear_attn(dq, dk, dv, w.Hg, w.Wg))
+
+
+# ------------------------------------------------------------------ Table 1 variant: token-wise dynamic convolution
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("case", [(2, 2, 0, 21, 18, 3, 64), (1, 2, 5, 13, 16, 3, 64), (1, 2, 0, 9, 10, 5, 16), (1, 3, 2, 8, 8, 3, 24)],
+                         ids=lambda c: "x".join(map(str, c)))
+def test_linear_with_tokenwise_dynamic_dwc(jv, oracle, both_paths, dtype, case):
+    """R = 64 with 3 x 3 kernels runs on the tensor-core generator (bf16); the other cases, fp32 and
+    the forced-generic runs on the per-token kernels."""
+    B, H, P, Hg, Wg, ksz, R = case
+    q, k, v = inputs.custom_qkv(B, H, P + Hg * Wg, 64, dtype, seed=300 + Hg + R)
+    d = dict(inputs.dwc_weights(H * 64, R, ksz, 301), token_wise=1)
+    out, check = guarded_empty(q.shape, _dev((q,))[0].dtype, DEV)
+    jv.linear_attn(*_dev((q, k, v)), Hg, Wg, dwc=dwc_to_device(d, DEV), out=out, prefix=P)
+    check()
+    # This variant stores the attention output, reads it back and stores the sum: two bf16 roundings,
+    # sqrt(2) x 2.26e-3 rms from the stores alone, hence its own rms bar (the max-norm bar is the usual one).
+    assert rel_err(out, oracle.linear_attn(q, k, v, Hg, Wg, dwc=d, prefix=P), rms_tol=4.5e-3) <= TOL[dtype]
+
+
+def test_tokenwise_dynamic_dwc_larger_grid_sampled(jv, oracle):
+    """64 x 64 grid, 4 heads, R = 128: the GEMM tiles of the generator run over several token and
+    feature tiles; whole samples against the oracle (the generator mixes the heads of a sample)."""
+    B, H, Hg, Wg, R = 2, 4, 64, 64, 128
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, 64, "bf16", seed=310)
+    d = dict(inputs.dwc_weights(H * 64, R, 3, 311), token_wise=1)
+    out = jv.linear_attn(*_dev((q, k, v)), Hg, Wg, dwc=dwc_to_device(d, DEV)).cpu()
+    ref = oracle.linear_attn(q[1:], k[1:], v[1:], Hg, Wg, dwc=d)
+    assert rel_err(out[1:], ref, rms_tol=4.5e-3) <= TOL["bf16"]
