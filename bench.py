@@ -434,6 +434,27 @@ def run_cuda(args):
     add("F", lambda i: jv.full_attn(dq[r(i)], dk[r(i)], dv[r(i)], out=outs[r(i)]),
         alg_bytes(*w.shape), f_flops, "tensor")
 
+    # Table 1's variants of the linear block at mixer level, same shape, same inputs: ReLU linear attention,
+    # + static DWC, + DWC + focusing factor (p = 3), + token-wise dynamic DWC, + squeeze dynamic DWC
+    dwc_static = {"k": 3, "R": 0, "b2": dwc_dev["b2"]}
+    dwc_token = dict(dwc_dev, token_wise=1)
+    shape_l = jv.make_shape(dq[0], w.Hg, w.Wg)
+    ws_f = jv.alloc_workspace("f", shape_l, jv.make_dwc(dwc_static, dev), dev)
+    ws_t = jv.alloc_workspace("L", shape_l, jv.make_dwc(dwc_token, dev), dev)
+    table1 = {}
+    for name, fn in (
+            ("relu_la", lambda i: jv.linear_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, out=outs[r(i)], ws=ws)),
+            ("static_dwc", lambda i: jv.linear_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, dwc=dwc_static, out=outs[r(i)], ws=ws)),
+            ("static_dwc_focus_p3", lambda i: jv.linear_attn_focused(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, 3.0, dwc=dwc_static,
+                                                                     out=outs[r(i)], ws=ws_f)),
+            ("tokenwise_dyn_dwc", lambda i: jv.linear_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, dwc=dwc_token, out=outs[r(i)], ws=ws_t)),
+            ("squeeze_dyn_dwc", lambda i: jv.linear_attn(dq[r(i)], dk[r(i)], dv[r(i)], w.Hg, w.Wg, dwc=dwc_dev, out=outs[r(i)], ws=ws))):
+        t_ms = time_calls(fn, min(K, 30), 3, stream)
+        table1[name] = {"ms": t_ms, "tokens_per_s": w.tokens / (t_ms * 1e-3)}
+    table1["note"] = ("mixer-level times of the rows of the paper's Table 1 (whole-model H100 latencies there: 5.33 / 5.72 / 6.00 / "
+                      "8.94 / 5.88 ms); only the ordering is comparable")
+    del ws_f, ws_t
+
     # the projections either side of a mixer (outside the step: the metric counts mixers only)
     Cm = w.H * w.D
     px = inputs.normal((w.B, w.N, Cm), inputs.seed_for(w.cfg, 0, 5), "bf16").to(dev)
@@ -566,7 +587,7 @@ def run_cuda(args):
                                    "W 16x16, F", "l2": "three layers' tensors (805 MB) exceed L2; "
                                    "per-mixer loops rotate over three tensor sets"},
             "clocks": clk.summary(), "sustained": sustained, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": cpu, "per_mixer": per, "hybrid24": hybrid,
+            "roofline": roofline, "cpu_baseline": cpu, "per_mixer": per, "table1_variants": table1, "hybrid24": hybrid,
             "peaks": peaks}
     print(json.dumps(line))
     if world > 1:
