@@ -99,6 +99,9 @@ cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, bool prefix_
 // windows whose width ww is a power of two <= 128 (a tile is a box of ww x 128/ww tokens).
 bool attn_tc_supported(const AttnArgs& a, bool full);
 cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream_t st);
+// tcgen05 path for windows of one or two 128-token tiles (bf16, D == 64, no prefix): two windows per CTA
+bool attn_w4_supported(const AttnArgs& a);
+cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st);
 // tcgen05 path for full attention over long sequences (bf16, D == 64, N >= 1024): four query tiles per CTA
 bool attn_f4_supported(const AttnArgs& a);
 cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st);
