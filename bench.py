@@ -485,6 +485,20 @@ def run_cuda(args):
          alg_flops_attn(w.B, w.H, w.Hg, w.Wg, w.D, WIN, WIN, prefix=P5), "hbm")
     del pq, po
 
+    # the same shape with q, k, v as slices of a fused [B, N, 3, H, D] activation (token stride 3 H D), the form in
+    # which a model's QKV projection leaves them; the mixers read them in place through strided tensor maps
+    fq = []
+    for l in range(3):
+        qkv3 = torch.stack([t.permute(0, 2, 1, 3) for t in (dq[l], dk[l], dv[l])], dim=2).contiguous()
+        fq.append((qkv3, [qkv3[:, :, i].permute(0, 2, 1, 3) for i in range(3)]))
+    add("L+dwc@fused_qkv", lambda i: jv.linear_attn(*fq[r(i)][1], w.Hg, w.Wg, dwc=dwc_dev, out=outs[r(i)], ws=ws),
+        alg_bytes(*w.shape, dwc=True), 0.0, "hbm")
+    add("W@fused_qkv", lambda i: jv.window_attn(*fq[r(i)][1], w.Hg, w.Wg, WIN, WIN, out=outs[r(i)]),
+        alg_bytes(*w.shape), alg_flops_attn(w.B, w.H, w.Hg, w.Wg, w.D, WIN, WIN), "hbm")
+    add("F@fused_qkv", lambda i: jv.full_attn(*fq[r(i)][1], out=outs[r(i)]),
+        alg_bytes(*w.shape), f_flops, "tensor")
+    del fq
+
     # other model sizes at the 1024 x 2048 image of Tables 1 and 3 (64 x 128 token grid): 12 heads (ViT-B), 24 heads (Giant)
     for tag, heads in (("vitb_64x128", 12), ("giant_64x128", 24)):
         Bx, Hgx, Wgx = 4, 64, 128

@@ -75,11 +75,24 @@ typedef enum { JV_F32 = 0, JV_BF16 = 1 } jv_dtype;
  * tokens; in W a grid token attends its window and the P prefix tokens, a prefix token attends
  * all N tokens; the convolution and the pooling that feeds its kernel generator see the grid only
  * (a prefix token's L output is its linear-attention output alone).
+ *
+ * in_layout describes q, k and v only (o is always [B, H, N, D] contiguous).  With JV_LAYOUT_BNHD
+ * they are [B, N, H, D] arrays whose token rows (H * D elements each, heads side by side) are
+ * in_tok_stride elements apart: H * D for a contiguous array (0 selects that), 3 * H * D for the
+ * three slices of a fused [B, N, 3, H, D] activation, the form in which a model's QKV projection
+ * leaves them (the blocks take their inputs from the inherited projections, Sec. 3.2.4).  Batch
+ * element b starts N * in_tok_stride elements after b - 1.  The layout is served by the tensor-core
+ * paths only: bf16, D = 64, P = 0 where a convolution is asked for, 3 x 3 pooled or static kernels;
+ * everything else returns JV_ERR_UNSUPPORTED.  in_tok_stride * element size must be a multiple of 16.
  */
+typedef enum { JV_LAYOUT_BHND = 0, JV_LAYOUT_BNHD = 1 } jv_layout;
+
 typedef struct {
   int32_t B, H, Hg, Wg, D;
-  int32_t dtype; /* jv_dtype */
-  int32_t P;     /* prefix tokens in front of the grid tokens, >= 0 */
+  int32_t dtype;         /* jv_dtype */
+  int32_t P;             /* prefix tokens in front of the grid tokens, >= 0 */
+  int32_t in_layout;     /* jv_layout of q, k, v; 0 = [B, H, N, D] contiguous like o */
+  int64_t in_tok_stride; /* JV_LAYOUT_BNHD: elements between token rows; 0 = H * D */
 } jv_shape;
 
 /*

@@ -37,14 +37,31 @@ jv_status check_shape(const jv_shape* s) {
   // rows must keep 16-byte alignment for the vector loads
   const int esz = s->dtype == JV_F32 ? 4 : 2;
   if ((s->D * esz) % 16 != 0) return JV_ERR_UNSUPPORTED;
+  if (s->in_layout != JV_LAYOUT_BHND && s->in_layout != JV_LAYOUT_BNHD) return JV_ERR_INVALID_ARG;
+  if (s->in_layout == JV_LAYOUT_BNHD) {
+    const int64_t row = (int64_t)s->H * s->D;
+    if (s->in_tok_stride != 0 && s->in_tok_stride < row) return JV_ERR_INVALID_ARG;   // token rows would overlap
+    if ((s->in_tok_stride * esz) % 16 != 0) return JV_ERR_INVALID_ARG;
+    if (s->in_tok_stride > ((int64_t)1 << 31)) return JV_ERR_UNSUPPORTED;
+  } else if (s->in_tok_stride != 0) {
+    return JV_ERR_INVALID_ARG;
+  }
   return JV_OK;
+}
+
+// bytes from the first to one past the last element of an input tensor (q, k or v)
+size_t input_bytes(const jv_shape* s) {
+  if (!in_strided(*s)) return tensor_bytes(s);
+  const InStrides in = in_strides(*s);
+  const size_t esz = s->dtype == JV_F32 ? 4 : 2;
+  return (size_t)((int64_t)(s->B - 1) * in.batch + (int64_t)(shape_tokens(*s) - 1) * in.tok + (int64_t)s->H * s->D) * esz;
 }
 
 jv_status check_tensors(const void* q, const void* k, const void* v, const void* o, const jv_shape* s) {
   if (!q || !k || !v || !o) return JV_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return JV_ERR_INVALID_ARG;
-  const size_t n = tensor_bytes(s);      // o may not share a byte with an input
-  if (overlaps(o, n, q, n) || overlaps(o, n, k, n) || overlaps(o, n, v, n)) return JV_ERR_INVALID_ARG;
+  const size_t n = tensor_bytes(s), ni = input_bytes(s);      // o may not share a byte with an input
+  if (overlaps(o, n, q, ni) || overlaps(o, n, k, ni) || overlaps(o, n, v, ni)) return JV_ERR_INVALID_ARG;
   return JV_OK;
 }
 
@@ -90,6 +107,7 @@ jv_status check_proj(const jv_shape* s, const void* const* ptrs, const size_t* b
   for (int i = 0; i < nptr; ++i)
     if (!ptrs[i] || !aligned(ptrs[i], 16)) return JV_ERR_INVALID_ARG;
   if (s->dtype != JV_BF16 || s->D != 64) return JV_ERR_UNSUPPORTED;   // (the extents below assume both)
+  if (in_strided(*s)) return JV_ERR_UNSUPPORTED;                        // the projections have layouts of their own
   for (int i = nin; i < nptr; ++i)           // outputs overlap neither an input nor each other
     for (int j = 0; j < i; ++j)
       if (overlaps(ptrs[i], bytes[i], ptrs[j], bytes[j])) return JV_ERR_INVALID_ARG;
@@ -107,7 +125,8 @@ float pick_scale(float scale, int D) { return scale > 0.f ? scale : 1.f / sqrtf(
 // ---- enqueue helpers (arguments already validated) ---------------------------
 jv_status run_attn(const void* q, const void* k, const void* v, void* o, const jv_shape* s, int wh, int ww,
                    float scale, bool full, cudaStream_t st) {
-  AttnArgs a{q, k, v, o, s->B * s->H, s->Hg, s->Wg, s->D, s->P, wh, ww, pick_scale(scale, s->D), s->dtype};
+  AttnArgs a{q, k, v, o, s->B * s->H, s->Hg, s->Wg, s->D, s->H, in_strides(*s), in_strided(*s),
+             s->P, wh, ww, pick_scale(scale, s->D), s->dtype};
   const bool one_window = full || (wh >= s->Hg && ww >= s->Wg);
   if (one_window) {      // every token attends all P + N tokens: where a token sits does not matter
     a.Hg = 1;
@@ -129,10 +148,12 @@ jv_status run_attn(const void* q, const void* k, const void* v, void* o, const j
   if (!g_force_generic.load() && attn_tc_supported(a, full)) {
     int* status = device_status_ptr();
     if (!status) return JV_ERR_CUDA;
+    if (a.strided && a.P > 0) return JV_ERR_UNSUPPORTED;  // the prefix queries' kernel reads contiguous tensors
     const jv_status r = from_cuda(launch_attn_tc(a, full, status, st));
     if (r != JV_OK || a.P == 0) return r;
     return from_cuda(launch_attn_generic(a, st, true));   // the P prefix queries, which attend everything
   }
+  if (a.strided) return JV_ERR_UNSUPPORTED;               // the generic kernels read contiguous tensors
   return from_cuda(launch_attn_generic(a, st));
 }
 
@@ -146,6 +167,7 @@ jv_status run_linear(const void* q, const void* k, const void* v, void* o, const
   }
   const LinPlan p = lin_plan(*s, dwc);
   if (!g_force_generic.load() && linear_fast_supported(a)) return from_cuda(launch_linear_fast(a, p, st));
+  if (in_strided(*s)) return JV_ERR_UNSUPPORTED;          // the generic kernels read contiguous tensors
   return from_cuda(launch_linear_generic(a, p, st));
 }
 
@@ -227,6 +249,7 @@ jv_status jv_linear_attn_focused(const void* q, const void* k, const void* v, vo
   if ((st = check_tensors(q, k, v, o, shape)) != JV_OK) return st;
   if (!(eps >= 0.f) || !(focus_p > 0.f) || !(focus_p <= 16.f)) return JV_ERR_INVALID_ARG;
   if ((st = check_dwc(dwc)) != JV_OK) return st;
+  if (in_strided(*shape)) return JV_ERR_UNSUPPORTED;      // the feature-map pass reads contiguous q and k
   const size_t lin = align_up(lin_plan(*shape, dwc).total, 256), tb = align_up(tensor_bytes(shape), 256);
   if ((st = check_ws(ws, ws_bytes, lin + 2 * tb)) != JV_OK) return st;
   if ((st = check_device()) != JV_OK) return st;

@@ -57,6 +57,8 @@ struct F4Params {
   int n_full;            // items [0, n_full) are whole groups, (batch*head, group) with the group fastest;
   int total_items;       // items [n_full, total_items) are half groups (two query tiles), see launch_attn_f4
   FastDiv div_qgroups;
+  int H;                 // heads per batch element: the inputs are addressed by (head, batch)
+  FastDiv div_H;
   float scale_log2;      // softmax scale * log2(e)
 };
 
@@ -169,12 +171,13 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     for (int i = item0; i < p.total_items && ok; i += item_step) {
       const Item it = decode_item<kHalves>(p, i);
       if (kHalves && !tile_exists<kHalves>(it, 0, ntiles)) continue;
+      const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
       for (int t = 0; t < kQT && ok; ++t) {
         ok = warp_wait(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
         if (!ok) break;
         if (tile_exists<kHalves>(it, t, ntiles) && elect_one()) {
           mbar_expect_tx(&bar->q_full[t], kTileBytes);
-          tma_load_3d(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], 0, (it.qt0 + t) * kTile, it.bh);
+          tma_load_4d(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], 0, (it.qt0 + t) * kTile, h, b);
         }
         __syncwarp();
       }
@@ -183,14 +186,14 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s], kTileBytes);
-          tma_load_3d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, j * kTile, it.bh);
+          tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, j * kTile, h, b);
         }
         __syncwarp();
         ok = warp_wait(&bar->v_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s], kTileBytes);
-          tma_load_3d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, j * kTile, it.bh);
+          tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, j * kTile, h, b);
         }
         __syncwarp();
         ++issued_v;
@@ -460,13 +463,20 @@ cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st) {
   const void* ptrs[4] = {a.q, a.k, a.v, a.o};
   const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)a.BH};
   const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)N * kD * 2};
-  const cuuint32_t box[3] = {(cuuint32_t)kD, (cuuint32_t)kTile, 1};
   const cuuint32_t qbox[3] = {(cuuint32_t)kD, 32, 1};          // the output is stored per warp: 32 tokens
   const cuuint32_t estr[3] = {1, 1, 1};
+  // the inputs as (d, token, head, batch) with the caller's strides; the output as (d, token, batch*head)
+  const cuuint64_t idims[4] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
+  const cuuint64_t istrides[3] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)a.in.head * 2, (cuuint64_t)a.in.batch * 2};
+  const cuuint32_t ibox[4] = {(cuuint32_t)kD, (cuuint32_t)kTile, 1, 1};
+  const cuuint32_t iestr[4] = {1, 1, 1, 1};
   for (int i = 0; i < 4; ++i) {
-    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptrs[i]), dims, strides,
-                     i == 3 ? qbox : box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = i < 3 ? enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), idims, istrides, ibox,
+                             iestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE)
+                       : enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptrs[i]), dims, strides, qbox,
+                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
@@ -492,6 +502,8 @@ cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st) {
   p.n_full = groups - split;
   p.total_items = groups + split;
   p.div_qgroups = make_fastdiv((uint32_t)p.qgroups);
+  p.H = a.H;
+  p.div_H = make_fastdiv((uint32_t)a.H);
   p.scale_log2 = a.scale * 1.4426950408889634f;
   const int grid = p.total_items < num_sms ? p.total_items : num_sms;
   if (split) attn_f4_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);

@@ -71,6 +71,8 @@ struct TcParams {
   int lg_box_h;          // log2(box_h)
   int P;                 // prefix keys behind every window's own key tiles (0: none)
   FastDiv div_qpairs, div_nwin, div_nwx;
+  int H;                 // heads per batch element: the inputs are addressed by (head, batch)
+  FastDiv div_H;
   float scale_log2;      // softmax scale * log2(e)
 };
 
@@ -196,13 +198,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const Item it = decode_item(p, i);
       if (it.qt0 >= it.ntiles) continue;
       const int qb = n & 1;
+      const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
       ok = warp_wait(&bar->q_empty[qb], ((n >> 1) & 1) ^ 1, &bar->abort_flag, p.status);
       if (!ok) break;
       if (elect_one()) {
         mbar_expect_tx(&bar->q_full[qb], 2 * kTileBytes);
         for (int t = 0; t < 2; ++t)
-          tma_load_4d(sQ + (2 * qb + t) * kTileBytes, &mapQ, &bar->q_full[qb], 0, it.x0 + (it.qt0 + t) * p.step_x,
-                      it.y0 + (it.qt0 + t) * p.step_y, it.bh);
+          tma_load_5d(sQ + (2 * qb + t) * kTileBytes, &mapQ, &bar->q_full[qb], 0, it.x0 + (it.qt0 + t) * p.step_x,
+                      it.y0 + (it.qt0 + t) * p.step_y, h, b);
       }
       __syncwarp();
       for (int j = 0; j < it.nkt; ++j) {
@@ -212,7 +215,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s], kTileBytes);
           if (pre) tma_load_4d(sK + s * kTileBytes, &mapKp, &bar->k_full[s], 0, 0, 0, it.bh);
-          else tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
+          else tma_load_5d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, h, b);
         }
         __syncwarp();
         ok = warp_wait(&bar->v_empty[s], par, &bar->abort_flag, p.status);
@@ -220,7 +223,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s], kTileBytes);
           if (pre) tma_load_4d(sV + s * kTileBytes, &mapVp, &bar->v_full[s], 0, 0, 0, it.bh);
-          else tma_load_4d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, it.bh);
+          else tma_load_5d(sV + s * kTileBytes, &mapV, &bar->v_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, h, b);
         }
         __syncwarp();
         ++issued_v;
@@ -703,8 +706,9 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   if (!enc) return cudaErrorNotSupported;
   const int N = a.P + a.Hg * a.Wg;                     // tokens per (batch, head): prefix tokens, then the grid
   CUtensorMap maps[6];
-  const size_t grid0 = (size_t)a.P * kD * 2;           // the grid tokens start behind the prefix rows
-  const void* ptrs[4] = {(const char*)a.q + grid0, (const char*)a.k + grid0, (const char*)a.v + grid0, (char*)a.o + grid0};
+  // the grid tokens start behind the prefix rows
+  const size_t grid0 = (size_t)a.P * kD * 2, igrid0 = (size_t)a.P * (size_t)a.in.tok * 2;
+  const void* ptrs[4] = {(const char*)a.q + igrid0, (const char*)a.k + igrid0, (const char*)a.v + igrid0, (char*)a.o + grid0};
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.gridW, (cuuint64_t)g.gridH, (cuuint64_t)a.BH};
   const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)g.gridW * kD * 2, (cuuint64_t)N * kD * 2};
   const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1};
@@ -712,17 +716,26 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   // the output is stored per warp: a quarter of the tile's box (32 tokens)
   const cuuint32_t qbox[4] = {(cuuint32_t)kD, (cuuint32_t)(g.box_h >= 4 ? g.box_w : 32),
                               (cuuint32_t)(g.box_h >= 4 ? g.box_h / 4 : 1), 1};
+  // the inputs as (d, x, y, head, batch) with the caller's strides; the output as (d, x, y, batch*head)
+  const cuuint64_t idims[5] = {(cuuint64_t)kD, (cuuint64_t)g.gridW, (cuuint64_t)g.gridH, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
+  const cuuint64_t istrides[4] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)g.gridW * a.in.tok * 2, (cuuint64_t)a.in.head * 2,
+                                  (cuuint64_t)a.in.batch * 2};
+  const cuuint32_t ibox[5] = {(cuuint32_t)kD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1, 1};
+  const cuuint32_t iestr[5] = {1, 1, 1, 1, 1};
   for (int i = 0; i < 4; ++i) {
-    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides,
-                     i == 3 ? qbox : box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = i < 3 ? enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptrs[i]), idims, istrides, ibox,
+                             iestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE)
+                       : enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides, qbox,
+                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   // The prefix rows of K and V in the shape of a key box: prefix token r at box position
   // (r % box_w, r / box_w).  Positions past P inside the last box row read grid tokens (they exist:
   // a grid holds at least one box row of tokens) and are masked by the softmax; rows past that are
   // outside the map and arrive as zeros.
+  // (prefix tokens come with contiguous inputs only: the caller has checked)
   maps[4] = maps[1];
   maps[5] = maps[2];
   if (a.P > 0) {
@@ -763,6 +776,8 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
   p.div_qpairs = make_fastdiv((uint32_t)p.qpairs);
   p.div_nwin = make_fastdiv((uint32_t)p.nwin);
   p.div_nwx = make_fastdiv((uint32_t)p.nwx);
+  p.H = a.H;
+  p.div_H = make_fastdiv((uint32_t)a.H);
   p.scale_log2 = a.scale * 1.4426950408889634f;
   // persistent: one CTA per SM (shared memory and the 512 tensor-memory columns allow no more)
   const int num_sms = device_sm_count();

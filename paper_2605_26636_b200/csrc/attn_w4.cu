@@ -58,6 +58,8 @@ struct W4Params {
   int nwx, nwin;         // windows per grid row, per (batch, head)
   int total;             // windows of the whole call: (batch*head, window), window fastest
   FastDiv div_nwin, div_nwx;
+  int H;                 // heads per batch element: the inputs are addressed by (head, batch)
+  FastDiv div_H;
   float scale_log2;      // softmax scale * log2(e)
 };
 
@@ -167,13 +169,14 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     int issued_v = 0;                // for the abort path: V copies issued so far
     for (int r = kSlots * blockIdx.x + s; r < p.total && ok; r += item_step) {
       const Item it = decode_item(p, r);
+      const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
       for (int x = 0; x < 2 && ok; ++x) {
         const int t = 2 * s + x;
         ok = warp_wait(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
         if (!ok) break;
         if (x < it.ntiles && elect_one()) {
           mbar_expect_tx(&bar->q_full[t], kTileBytes);
-          tma_load_4d(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], 0, it.x0, it.y0 + x * p.box_h, it.bh);
+          tma_load_5d(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], 0, it.x0, it.y0 + x * p.box_h, h, b);
         }
         __syncwarp();
       }
@@ -182,7 +185,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s][ks], kTileBytes);
-          tma_load_4d(sK + (s * kKS + ks) * kTileBytes, &mapK, &bar->k_full[s][ks], 0, it.x0, it.y0 + j * p.box_h, it.bh);
+          tma_load_5d(sK + (s * kKS + ks) * kTileBytes, &mapK, &bar->k_full[s][ks], 0, it.x0, it.y0 + j * p.box_h, h, b);
         }
         __syncwarp();
         if (++ks == kKS) { ks = 0; kpar ^= 1; }
@@ -190,7 +193,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s][vs], kTileBytes);
-          tma_load_4d(sV + (s * kVS + vs) * kTileBytes, &mapV, &bar->v_full[s][vs], 0, it.x0, it.y0 + j * p.box_h, it.bh);
+          tma_load_5d(sV + (s * kVS + vs) * kTileBytes, &mapV, &bar->v_full[s][vs], 0, it.x0, it.y0 + j * p.box_h, h, b);
         }
         __syncwarp();
         ++issued_v;
@@ -494,14 +497,22 @@ cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st) {
   const void* ptrs[4] = {a.q, a.k, a.v, a.o};
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)a.Wg, (cuuint64_t)a.Hg, (cuuint64_t)a.BH};
   const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)a.Wg * kD * 2, (cuuint64_t)N * kD * 2};
-  const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
   // the output is stored per warp: a quarter of the tile's box (32 tokens)
   const cuuint32_t qbox[4] = {(cuuint32_t)kD, (cuuint32_t)box_w, (cuuint32_t)(box_h / 4), 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
+  // the inputs as (d, x, y, head, batch) with the caller's strides; the output as (d, x, y, batch*head)
+  const cuuint64_t idims[5] = {(cuuint64_t)kD, (cuuint64_t)a.Wg, (cuuint64_t)a.Hg, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
+  const cuuint64_t istrides[4] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)a.Wg * a.in.tok * 2, (cuuint64_t)a.in.head * 2,
+                                  (cuuint64_t)a.in.batch * 2};
+  const cuuint32_t ibox[5] = {(cuuint32_t)kD, (cuuint32_t)box_w, (cuuint32_t)box_h, 1, 1};
+  const cuuint32_t iestr[5] = {1, 1, 1, 1, 1};
   for (int i = 0; i < 4; ++i) {
-    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides,
-                     i == 3 ? qbox : box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = i < 3 ? enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptrs[i]), idims, istrides, ibox,
+                             iestr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE)
+                       : enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), dims, strides, qbox,
+                             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
   static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
@@ -524,6 +535,8 @@ cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st) {
   p.total = p.nwin * a.BH;
   p.div_nwin = make_fastdiv((uint32_t)p.nwin);
   p.div_nwx = make_fastdiv((uint32_t)p.nwx);
+  p.H = a.H;
+  p.div_H = make_fastdiv((uint32_t)a.H);
   p.scale_log2 = a.scale * 1.4426950408889634f;
   const int num_sms = device_sm_count();
   const int want = ceil_div(p.total, kSlots);

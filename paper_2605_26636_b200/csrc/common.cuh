@@ -68,6 +68,20 @@ static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline int shape_tokens(const jv_shape& s) { return s.P + s.Hg * s.Wg; }
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Element strides of the inputs q, k, v over (token, head, batch); o is always [B, H, N, D] contiguous.
+struct InStrides {
+  int64_t tok, head, batch;
+};
+static inline InStrides in_strides(const jv_shape& s) {
+  const int64_t n = shape_tokens(s);
+  if (s.in_layout == JV_LAYOUT_BNHD) {
+    const int64_t ts = s.in_tok_stride ? s.in_tok_stride : (int64_t)s.H * s.D;
+    return InStrides{ts, (int64_t)s.D, n * ts};
+  }
+  return InStrides{(int64_t)s.D, n * s.D, (int64_t)s.H * n * s.D};
+}
+static inline bool in_strided(const jv_shape& s) { return s.in_layout != JV_LAYOUT_BHND; }
+
 // ---- plan of the linear-attention workspace --------------------------------
 // State per (batch, head): (D+1) x (D+1) fp32, S[a][e] = sum_j pk[j][a] * pv[j][e]
 // with pk = [relu(k) | 1], pv = [v | 1]:  S[a<D][e<D] = KV, S[a][D] = z (k-sum),
@@ -89,6 +103,9 @@ struct AttnArgs {
   const void *q, *k, *v;
   void* o;
   int BH, Hg, Wg, D;
+  int H;           // heads: (batch, head) index bh = b * H + h
+  InStrides in;    // element strides of q, k, v (the tensor-core paths honour them; the others need the default)
+  bool strided;    // in differs from the contiguous [B, H, N, D] strides
   int P;       // prefix tokens in front of the Hg x Wg grid tokens (full attention: folded into the "grid")
   int wh, ww;  // window size (wh >= Hg and ww >= Wg: one window = full attention)
   float scale;

@@ -56,6 +56,13 @@ __device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(map), "r"(tc::smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                                 int c2, int c3, int c4, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6, %7}], [%2], %8;"
+      ::"r"(dst), "l"(map), "r"(tc::smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(policy) : "memory");
+}
+
 // ---- host side: tensor maps ---------------------------------------------------------------
 // The first N tokens of every (batch, head) of a [BH, ntok, 64] bf16 tensor as (channel, token,
 // batch*head); boxes of box_tok tokens, 128-byte swizzle; tokens past N arrive as zeros.
@@ -69,6 +76,37 @@ inline bool make_map_tokens(CUtensorMap* m, const void* ptr, int BH, int N, int 
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// An input tensor (q, k or v) with the caller's strides: the first N tokens of every (batch, head)
+// as (channel, token, head, batch); boxes of box_tok tokens, 128-byte swizzle; tokens past N arrive as zeros.
+inline bool make_map_tokens_in(CUtensorMap* m, const void* ptr, int B, int H, int N, int box_tok, const InStrides& in) {
+  tc::EncodeFn enc = tc::encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)H, (cuuint64_t)B};
+  const cuuint64_t strides[3] = {(cuuint64_t)in.tok * 2, (cuuint64_t)in.head * 2, (cuuint64_t)in.batch * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)kD, (cuuint32_t)box_tok, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The Hg x Wg grid tokens (behind P prefix tokens) of an input tensor with the caller's strides as a 5-D
+// tensor (channel, x, y, head, batch); boxes of box_x x box_y tokens; positions outside the grid arrive as zeros.
+inline bool make_map_grid_in(CUtensorMap* m, const void* ptr, int B, int H, int P, int Hg, int Wg, int box_x, int box_y,
+                             bool swizzle128, const InStrides& in) {
+  tc::EncodeFn enc = tc::encode_fn();
+  if (!enc) return false;
+  ptr = (const char*)ptr + (size_t)P * (size_t)in.tok * 2;   // token strides are multiples of 16 bytes
+  const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)Wg, (cuuint64_t)Hg, (cuuint64_t)H, (cuuint64_t)B};
+  const cuuint64_t strides[4] = {(cuuint64_t)in.tok * 2, (cuuint64_t)Wg * in.tok * 2, (cuuint64_t)in.head * 2,
+                                 (cuuint64_t)in.batch * 2};
+  const cuuint32_t box[5] = {(cuuint32_t)kD, (cuuint32_t)box_x, (cuuint32_t)box_y, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // The Hg x Wg grid tokens of a [BH, P + Hg*Wg, 64] bf16 tensor (P prefix tokens in front of the

@@ -182,7 +182,9 @@ lin_apply_conv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
       }
       if (elect_one()) {
         mbar_expect_tx(&bars->q_full[sq], kTileBytes);
-        tma_load_4d_hint(smem + sq * kTileBytes, &mapQ, &bars->q_full[sq], 0, ti.px * kPatchW, ti.py * kPatchH, ti.bh, pol_first);
+        const int in_b = ti.bh / p.H;              // the inputs are addressed by (head, batch)
+        tma_load_5d_hint(smem + sq * kTileBytes, &mapQ, &bars->q_full[sq], 0, ti.px * kPatchW, ti.py * kPatchH,
+                         ti.bh - in_b * p.H, in_b, pol_first);
       }
       __syncwarp();
       ++issued_q;
@@ -192,8 +194,9 @@ lin_apply_conv_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_con
       }
       if (elect_one()) {
         mbar_expect_tx(&bars->v_full[sv], kHaloBytes);
-        tma_load_4d(smem + (uint32_t)kOffHalo + sv * kHaloSlot, &mapV, &bars->v_full[sv], 0, ti.px * kPatchW - 1,
-                    ti.py * kPatchH - 1, ti.bh);
+        const int in_b = ti.bh / p.H;
+        tma_load_5d(smem + (uint32_t)kOffHalo + sv * kHaloSlot, &mapV, &bars->v_full[sv], 0, ti.px * kPatchW - 1,
+                    ti.py * kPatchH - 1, ti.bh - in_b * p.H, in_b);
       }
       __syncwarp();
       ++issued_v;
@@ -525,8 +528,9 @@ cudaError_t launch_linear_apply_conv(const LinArgs& a, const LinPlan& p, const f
   const jv_shape& s = a.s;
   const int BH = s.B * s.H;
   CUtensorMap mq, mv, mo;
-  if (!make_map_grid(&mq, a.q, BH, s.P, s.Hg, s.Wg, kPatchW, kPatchH, true) ||
-      !make_map_grid(&mv, a.v, BH, s.P, s.Hg, s.Wg, kPatchW + 2, kPatchH + 2, false) ||
+  const InStrides in = in_strides(s);
+  if (!make_map_grid_in(&mq, a.q, s.B, s.H, s.P, s.Hg, s.Wg, kPatchW, kPatchH, true, in) ||
+      !make_map_grid_in(&mv, a.v, s.B, s.H, s.P, s.Hg, s.Wg, kPatchW + 2, kPatchH + 2, false, in) ||
       !make_map_grid(&mo, a.o, BH, s.P, s.Hg, s.Wg, kPatchW, kPatchH, true))
     return cudaErrorInvalidValue;
   static OncePerDevice smem_opt_in;

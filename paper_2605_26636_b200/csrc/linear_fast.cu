@@ -42,12 +42,10 @@ constexpr int kTileBytes = kTileTok * kD * 2; // 8 KB
 constexpr int kConsumers = 128;               // 4 MMA warps
 constexpr int kThreads = kConsumers + 32;     // + 1 producer warp
 
-// 64 tokens x 64 channels of a [B*H, N, 64] tensor -> shared memory (128-byte swizzle);
-// tokens past N arrive as zeros.
-__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int tok, int bh) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(0), "r"(tok), "r"(bh) : "memory");
+// A box of tokens x 64 channels of an input tensor (channel, token, head, batch) -> shared memory
+// (128-byte swizzle); tokens past N arrive as zeros.
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int tok, int h, int b) {
+  tma_load_4d(dst, map, bar, 0, tok, h, b);
 }
 
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
@@ -71,7 +69,7 @@ constexpr size_t kStateSmem = (size_t)kStateStages * 2 * kTileBytes + 1024 + siz
 template <bool kVsum>
 __global__ void __launch_bounds__(kThreads)
 lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
-                 float* __restrict__ partial, int* status, int N, int chunk_tokens, int state_elems) {
+                 float* __restrict__ partial, int* status, int N, int chunk_tokens, int state_elems, int H) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
   unsigned char* smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -79,6 +77,7 @@ lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant
   Ring* ring = reinterpret_cast<Ring*>(smem_al + (size_t)kStateStages * 2 * kTileBytes);
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
   const int bh = blockIdx.y, chunk = blockIdx.x;
+  const int in_b = bh / H, in_h = bh - in_b * H;      // coordinates of the input tensor maps
   const int t_begin = chunk * chunk_tokens, t_end = min(N, t_begin + chunk_tokens);
   const int ntiles = (t_end - t_begin + kTileTok - 1) / kTileTok;
 
@@ -112,9 +111,9 @@ lin_state_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant
       if (elect_one()) {
         mbar_expect_tx(&ring->full[s], 2 * kTileBytes);
         const int tok = t_begin + it * kTileTok;     // a chunk's last tile may run past t_end: only by whole
-        tma_load_3d_hint(smem + s * 2 * kTileBytes, &mapK, &ring->full[s], 0, tok, bh, pol_k);   // zero rows past N
-        if (kVsum) tma_load_3d_hint(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], 0, tok, bh, pol_v);
-        else tma_load_tile(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], tok, bh);
+        tma_load_4d_hint(smem + s * 2 * kTileBytes, &mapK, &ring->full[s], 0, tok, in_h, in_b, pol_k);   // zero rows past N
+        if (kVsum) tma_load_4d_hint(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], 0, tok, in_h, in_b, pol_v);
+        else tma_load_tile(smem + s * 2 * kTileBytes + kTileBytes, &mapV, &ring->full[s], tok, in_h, in_b);
       }
       __syncwarp();
       ++issued;
@@ -232,7 +231,7 @@ constexpr uint32_t kIdescApply = idesc(128, 64, 1);
 __global__ void __launch_bounds__(kApplyThreads, 2)
 lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapO,
                  const float* __restrict__ partial, int* status, int N, int span_tokens, int nchunk, int state_elems,
-                 float eps) {
+                 float eps, int H) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
   unsigned char* smem_al = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -292,7 +291,7 @@ lin_apply_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       if (elect_one()) {
         const int s = it % kApplyStages;
         mbar_expect_tx(&bars->full[s], kApplyTileBytes);
-        tma_load_tile(smem + s * kApplyTileBytes, &mapQ, &bars->full[s], t_begin + it * kApplyTok, bh);
+        tma_load_tile(smem + s * kApplyTileBytes, &mapQ, &bars->full[s], t_begin + it * kApplyTok, bh % H, bh / H);
       }
       __syncwarp();
       ++issued;
@@ -682,6 +681,9 @@ gen_out_kernel(const float* __restrict__ hidden, const float* __restrict__ W2, c
 bool linear_fast_supported(const LinArgs& a) {
   if (a.dwc && a.dwc->token_wise && !dwc_tokenwise_fast_supported(a)) return false;
   if (a.dwc && a.s.P > 0 && a.dwc->k != 3) return false;   // prefix tokens + 5 x 5 kernels: the generic kernels
+  // inputs with the caller's strides: only what reads them through tensor maps (the passes of the
+  // attention proper and the fused 3 x 3 convolution; the pooling's prefix correction reads V directly)
+  if (in_strided(a.s) && a.dwc && (a.dwc->token_wise || a.dwc->k != 3 || a.s.P > 0)) return false;
   return a.s.dtype == JV_BF16 && a.s.D == kD && encode_fn() != nullptr;
 }
 
@@ -703,8 +705,9 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   }
 
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map_tokens(&mq, a.q, BH, N, kApplyTok, N) || !make_map_tokens(&mk, a.k, BH, N, kTileTok, N) ||
-      !make_map_tokens(&mv, a.v, BH, N, kTileTok, N) || !make_map_tokens(&mo, a.o, BH, N, 32, N))
+  const InStrides in = in_strides(s);
+  if (!make_map_tokens_in(&mq, a.q, s.B, s.H, N, kApplyTok, in) || !make_map_tokens_in(&mk, a.k, s.B, s.H, N, kTileTok, in) ||
+      !make_map_tokens_in(&mv, a.v, s.B, s.H, N, kTileTok, in) || !make_map_tokens(&mo, a.o, BH, N, 32, N))
     return cudaErrorInvalidValue;
 
   static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
@@ -718,9 +721,9 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
   const int num_sms = device_sm_count();
   dim3 g1(p.nchunk, BH);
   if (a.dwc)
-    lin_state_kernel<true><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems);
+    lin_state_kernel<true><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems, (int)s.H);
   else
-    lin_state_kernel<false><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems);
+    lin_state_kernel<false><<<g1, kThreads, kStateSmem, st>>>(mk, mv, partial, status, N, p.chunk_tokens, p.state_elems, (int)s.H);
   count_launch();
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -751,7 +754,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, lin_apply_kernel, map_q, map_o, (const float*)partial, status, ntokens,
-                                               span, p.nchunk, p.state_elems, a.eps);
+                                               span, p.nchunk, p.state_elems, a.eps, (int)s.H);
     count_launch();
     return err;
   };
@@ -763,7 +766,7 @@ cudaError_t launch_linear_fast(const LinArgs& a, const LinPlan& p, cudaStream_t 
     // The plain apply pass over the first P tokens of every (batch, head), right behind the state pass
     // (which it waits for; the grids behind it wait for it in turn).
     CUtensorMap mqp, mop;
-    if (!make_map_tokens(&mqp, a.q, BH, s.P, kApplyTok, N) || !make_map_tokens(&mop, a.o, BH, s.P, 32, N))
+    if (!make_map_tokens_in(&mqp, a.q, s.B, s.H, s.P, kApplyTok, in) || !make_map_tokens(&mop, a.o, BH, s.P, 32, N))
       return cudaErrorInvalidValue;
     e = enqueue_apply(mqp, mop, s.P);
     if (e != cudaSuccess) return e;

@@ -21,7 +21,8 @@ LIB_PATH = os.environ.get("JETVIT_LIB") or os.path.join(_HERE, "libjetvit.so")
 
 class JvShape(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("Hg", ctypes.c_int32),
-                ("Wg", ctypes.c_int32), ("D", ctypes.c_int32), ("dtype", ctypes.c_int32), ("P", ctypes.c_int32)]
+                ("Wg", ctypes.c_int32), ("D", ctypes.c_int32), ("dtype", ctypes.c_int32), ("P", ctypes.c_int32),
+                ("in_layout", ctypes.c_int32), ("in_tok_stride", ctypes.c_int64)]
 
 
 class JvDwc(ctypes.Structure):
@@ -103,22 +104,48 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise TypeError(f"dtype {t.dtype}: the mixers take float32 or bfloat16")
 
 
+JV_LAYOUT_BHND, JV_LAYOUT_BNHD = 0, 1
+
+
+def _in_layout(t: torch.Tensor):
+    """(jv_layout, token stride) of an input tensor of logical shape [B, H, N, D]: contiguous, or a
+    [B, N, H, D] array seen through ``permute(0, 2, 1, 3)`` whose token rows are ``stride(2)`` elements
+    apart, e.g. ``qkv[:, :, i].permute(0, 2, 1, 3)`` of a fused [B, N, 3, H, D] activation."""
+    if t.is_contiguous():
+        return JV_LAYOUT_BHND, 0
+    B, H, N, D = t.shape
+    sb, sh, sn, sd = t.stride()
+    if sd == 1 and sh == D and sn >= H * D and (sb == N * sn or B == 1):
+        return JV_LAYOUT_BNHD, sn
+    raise ValueError("inputs must be contiguous [B,H,N,D] tensors or permuted views of [B,N,H,D] token rows")
+
+
 def make_shape(t: torch.Tensor, Hg: int, Wg: int, prefix: int = 0) -> JvShape:
     """Shape of [B, H, prefix + Hg*Wg, D] tensors: ``prefix`` tokens (class / register tokens) in
-    front of the grid tokens."""
+    front of the grid tokens.  The layout of the inputs is taken from ``t`` (see ``_in_layout``)."""
     B, H, N, D = t.shape
     if prefix < 0 or N != prefix + Hg * Wg:
         raise ValueError(f"N = {N} is not prefix + Hg*Wg = {prefix} + {Hg}*{Wg}")
-    return JvShape(B, H, Hg, Wg, D, _dtype_code(t), prefix)
+    layout, tok_stride = _in_layout(t)
+    return JvShape(B, H, Hg, Wg, D, _dtype_code(t), prefix, layout, tok_stride)
 
 
 def _check_tensors(*ts: torch.Tensor):
+    """q, k, v[, o]: one shape, dtype and device; q, k, v in one layout; o (a fourth tensor) contiguous."""
     ref = ts[0]
-    for t in ts:
+    for i, t in enumerate(ts):
         if not t.is_cuda:
             raise ValueError("tensors must live on a CUDA device (there is no CPU path)")
-        if not t.is_contiguous() or t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device:
-            raise ValueError("q, k, v, o must be contiguous [B,H,N,D] tensors of one shape, dtype and device")
+        if t.shape != ref.shape or t.dtype != ref.dtype or t.device != ref.device:
+            raise ValueError("q, k, v, o must be [B,H,N,D] tensors of one shape, dtype and device")
+        if i < 3 and _in_layout(t) != _in_layout(ref):
+            raise ValueError("q, k and v must share one layout (all contiguous, or all views with the same token stride)")
+        if i >= 3 and not t.is_contiguous():
+            raise ValueError("o must be a contiguous [B,H,N,D] tensor")
+
+
+def _empty_out(q: torch.Tensor) -> torch.Tensor:
+    return torch.empty(q.shape, dtype=q.dtype, device=q.device)
 
 
 def make_dwc(d: Optional[dict], device) -> Optional[JvDwc]:
@@ -163,7 +190,7 @@ def _raise(status: int, where: str):
 def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict] = None, out=None,
                 ws: Optional[torch.Tensor] = None, stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_linear_attn.  Allocates ``out`` / ``ws`` with torch when not given."""
-    out = torch.empty_like(q) if out is None else out
+    out = _empty_out(q) if out is None else out
     _check_tensors(q, k, v, out)
     shape = make_shape(q, Hg, Wg, prefix)
     d = make_dwc(dwc, q.device)
@@ -182,7 +209,7 @@ def linear_attn(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Optional[dict
 def linear_attn_focused(q, k, v, Hg: int, Wg: int, focus_p: float, eps: float = 1e-6, dwc: Optional[dict] = None,
                         out=None, ws: Optional[torch.Tensor] = None, stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_linear_attn_focused: the linear block with the focused feature map of Eq. 3 (power focus_p)."""
-    out = torch.empty_like(q) if out is None else out
+    out = _empty_out(q) if out is None else out
     _check_tensors(q, k, v, out)
     shape = make_shape(q, Hg, Wg, prefix)
     d = make_dwc(dwc, q.device)
@@ -222,7 +249,7 @@ def linear_attn_static(q, k, v, Hg: int, Wg: int, eps: float = 1e-6, dwc: Option
 def window_attn(q, k, v, Hg: int, Wg: int, win_h: int, win_w: int, scale: float = 0.0, out=None,
                 stream=None, prefix: int = 0) -> torch.Tensor:
     """jv_window_attn (scale <= 0: 1/sqrt(D))."""
-    out = torch.empty_like(q) if out is None else out
+    out = _empty_out(q) if out is None else out
     _check_tensors(q, k, v, out)
     shape = make_shape(q, Hg, Wg, prefix)
     with torch.cuda.device(q.device):
@@ -235,7 +262,7 @@ def window_attn(q, k, v, Hg: int, Wg: int, win_h: int, win_w: int, scale: float 
 def full_attn(q, k, v, Hg: Optional[int] = None, Wg: Optional[int] = None, scale: float = 0.0, out=None,
               stream=None) -> torch.Tensor:
     """jv_full_attn (scale <= 0: 1/sqrt(D)).  The grid split of N is irrelevant to F."""
-    out = torch.empty_like(q) if out is None else out
+    out = _empty_out(q) if out is None else out
     _check_tensors(q, k, v, out)
     if Hg is None or Wg is None:
         Hg, Wg = 1, q.shape[2]
@@ -255,11 +282,11 @@ def hybrid_mixers(schedule: str, q: Sequence[torch.Tensor], k, v, Hg: int, Wg: i
     n = len(schedule)
     if not (len(q) == len(k) == len(v) == n):
         raise ValueError("need one q, k, v per schedule entry")
-    out = [torch.empty_like(t) for t in q] if out is None else list(out)
+    out = [_empty_out(t) for t in q] if out is None else list(out)
     for l in range(n):
         _check_tensors(q[l], k[l], v[l], out[l])
-        if q[l].shape != q[0].shape or q[l].dtype != q[0].dtype:
-            raise ValueError("all layers share one shape and dtype")
+        if q[l].shape != q[0].shape or q[l].dtype != q[0].dtype or _in_layout(q[l]) != _in_layout(q[0]):
+            raise ValueError("all layers share one shape, dtype and input layout")
     shape = make_shape(q[0], Hg, Wg, prefix)
     arr = lambda ts: (ctypes.c_void_p * n)(*[t.data_ptr() for t in ts])
     dstructs = [make_dwc(d, q[0].device) for d in dwc] if dwc is not None else None

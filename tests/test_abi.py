@@ -85,6 +85,17 @@ def test_argument_errors_are_found_before_any_launch(L):
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 0, jv.JV_F32)) == jv.JV_ERR_INVALID_ARG
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 512, jv.JV_F32)) == jv.JV_ERR_UNSUPPORTED
     assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 30, jv.JV_BF16)) == jv.JV_ERR_UNSUPPORTED
+    # input layout: unknown code, token rows that would overlap, a stride that breaks 16-byte alignment,
+    # a stride without the layout that uses it; and an output inside the span of a strided input
+    assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 64, jv.JV_BF16, 0, 2, 0)) == jv.JV_ERR_INVALID_ARG
+    assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 64, jv.JV_BF16, 0, jv.JV_LAYOUT_BNHD, 64)) == jv.JV_ERR_INVALID_ARG
+    assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 64, jv.JV_BF16, 0, jv.JV_LAYOUT_BNHD, 3 * 128 + 4)) == jv.JV_ERR_INVALID_ARG
+    assert _call_linear(L, jv.JvShape(1, 2, 8, 8, 64, jv.JV_BF16, 0, jv.JV_LAYOUT_BHND, 384)) == jv.JV_ERR_INVALID_ARG
+    fused = jv.JvShape(1, 2, 8, 8, 64, jv.JV_BF16, 0, jv.JV_LAYOUT_BNHD, 384)
+    span = (63 * 384 + 128) * 2                   # bytes from the first to one past the last element of a slice
+    assert _call_linear(L, fused, o=FQ + span - 16) == jv.JV_ERR_INVALID_ARG
+    if not torch.cuda.is_available():
+        assert _call_linear(L, fused, o=FQ + span) in (jv.JV_ERR_CUDA, jv.JV_ERR_UNSUPPORTED)
     assert L.jv_window_attn(FQ, FK, FV, FO, ctypes.byref(shp), 0, 4, 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
     assert L.jv_full_attn(FQ, FK, FV, None, ctypes.byref(shp), 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
     assert L.jv_full_attn(FQ, FK, FV, FO, None, 0.0, None, 0, None) == jv.JV_ERR_INVALID_ARG
