@@ -562,6 +562,8 @@ def run_cuda(args):
     hybrid = {"schedule": inputs.HYBRID_SCHEDULE, "hybrid_ms": hyb, "all_full_ms": allf, "speedup": allf / hyb,
               "tokens_per_s_hybrid": w5.n_layers * w5.tokens / (hyb * 1e-3),
               "all_full_TFLOPs": w5.n_layers * f5_flops / allf / 1e9,
+              "all_full_frac_tensor_sustained": w5.n_layers * f5_flops / allf / 1e9 / peaks["bf16_tflops_sustained"],
+              "peak_note": "24 F layers back to back run under the power cap: the fraction is of the measured sustained bf16 peak",
               "note": "4 distinct layer inputs reused round-robin over the 24 layers (134 MB each: larger than L2)"}
     del q5, lo, base
     assert jv.device_status() == jv.JV_OK, "a kernel reported a timeout"

@@ -32,6 +32,10 @@ namespace {
 
 using namespace tc;
 
+#ifndef JV_ATTN_SUSPEND_NS
+#define JV_ATTN_SUSPEND_NS 4000
+#endif
+constexpr uint32_t kSuspendNs = JV_ATTN_SUSPEND_NS;   // suspend-time hint of this kernel's barrier waits (tc_common.cuh)
 constexpr int kD = 64;
 constexpr int kTile = 128;                  // tokens per tile (MMA M and key-tile rows)
 constexpr int kTileBytes = kTile * kD * 2;  // 16 KB
@@ -173,7 +177,7 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (kHalves && !tile_exists<kHalves>(it, 0, ntiles)) continue;
       const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
       for (int t = 0; t < kQT && ok; ++t) {
-        ok = warp_wait(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
         if (!ok) break;
         if (tile_exists<kHalves>(it, t, ntiles) && elect_one()) {
           mbar_expect_tx(&bar->q_full[t], kTileBytes);
@@ -182,14 +186,14 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         __syncwarp();
       }
       for (int j = 0; j < ntiles && ok; ++j) {
-        ok = warp_wait(&bar->k_empty[s], par, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->k_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s], kTileBytes);
           tma_load_4d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, j * kTile, h, b);
         }
         __syncwarp();
-        ok = warp_wait(&bar->v_empty[s], par, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->v_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s], kTileBytes);
@@ -228,11 +232,11 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int u = 0; u <= nsteps && ok; ++u) {
         const bool has_qk = u < nsteps, has_pv = u > 0;
         if (has_qk && (u & 1) == 0) {       // first half of a key tile: its K must have landed
-          ok = warp_wait(&bar->k_full[sk], phk, &bar->abort_flag, p.status);
+          ok = warp_wait<kSuspendNs>(&bar->k_full[sk], phk, &bar->abort_flag, p.status);
           if (!ok) break;
         }
         if (has_pv && ((u - 1) & 1) == 0) { // P V of a first half: its V must have landed
-          ok = warp_wait(&bar->v_full[sv], phv, &bar->abort_flag, p.status);
+          ok = warp_wait<kSuspendNs>(&bar->v_full[sv], phv, &bar->abort_flag, p.status);
           if (!ok) break;
         }
         const uint32_t kb = sK + sk * kTileBytes + (u & 1) * (kSub * kD * 2);
@@ -242,10 +246,10 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           if (!ex[x]) continue;
           const int t = tb + x;
           if (u == 0) {
-            ok = warp_wait(&bar->q_full[t], qcnt[x] & 1, &bar->abort_flag, p.status);
+            ok = warp_wait<kSuspendNs>(&bar->q_full[t], qcnt[x] & 1, &bar->abort_flag, p.status);
             ++qcnt[x];
           } else {
-            ok = warp_wait(&bar->p_full[t], pcnt[x] & 1, &bar->abort_flag, p.status);
+            ok = warp_wait<kSuspendNs>(&bar->p_full[t], pcnt[x] & 1, &bar->abort_flag, p.status);
             ++pcnt[x];
           }
           if (!ok) break;
@@ -314,7 +318,7 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (!tile_exists<kHalves>(it, t, ntiles)) continue;   // this query tile does not exist
       float m = -INFINITY, l = 0.f;
       for (int u = 0; u < nsteps; ++u) {
-        ok = warp_wait(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
         if (!ok) break;
         ++scnt;
         tc_fence_after();
@@ -391,7 +395,7 @@ attn_f4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       if (!ok) break;
       // ---- epilogue: O / l -> bf16 -> this warp's quarter of the staging tile -> one TMA store
-      ok = warp_wait(&bar->o_full[t], ocnt & 1, &bar->abort_flag, p.status);
+      ok = warp_wait<kSuspendNs>(&bar->o_full[t], ocnt & 1, &bar->abort_flag, p.status);
       if (!ok) break;
       ++ocnt;
       tc_fence_after();

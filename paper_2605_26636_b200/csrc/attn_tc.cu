@@ -42,6 +42,10 @@ namespace {
 
 using namespace tc;
 
+#ifndef JV_ATTN_SUSPEND_NS
+#define JV_ATTN_SUSPEND_NS 4000
+#endif
+constexpr uint32_t kSuspendNs = JV_ATTN_SUSPEND_NS;   // suspend-time hint of this kernel's barrier waits (tc_common.cuh)
 constexpr int kD = 64;
 constexpr int kTile = 128;                 // tokens per tile (MMA M and key-tile N)
 constexpr int kTileBytes = kTile * kD * 2; // 16 KB
@@ -199,7 +203,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (it.qt0 >= it.ntiles) continue;
       const int qb = n & 1;
       const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
-      ok = warp_wait(&bar->q_empty[qb], ((n >> 1) & 1) ^ 1, &bar->abort_flag, p.status);
+      ok = warp_wait<kSuspendNs>(&bar->q_empty[qb], ((n >> 1) & 1) ^ 1, &bar->abort_flag, p.status);
       if (!ok) break;
       if (elect_one()) {
         mbar_expect_tx(&bar->q_full[qb], 2 * kTileBytes);
@@ -210,7 +214,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       __syncwarp();
       for (int j = 0; j < it.nkt; ++j) {
         const bool pre = j == it.ntiles;               // the tile of prefix keys
-        ok = warp_wait(&bar->k_empty[s], par, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->k_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s], kTileBytes);
@@ -218,7 +222,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           else tma_load_5d(sK + s * kTileBytes, &mapK, &bar->k_full[s], 0, it.x0 + j * p.step_x, it.y0 + j * p.step_y, h, b);
         }
         __syncwarp();
-        ok = warp_wait(&bar->v_empty[s], par, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->v_empty[s], par, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s], kTileBytes);
@@ -271,8 +275,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     auto issue_qk = [&](int h, int jq, int ntiles_q, int n_q) -> bool {
       const int qb = n_q & 1;
       if (h == 0) {
-        if (jq == 0 && !warp_wait(&bar->q_full[qb], (n_q >> 1) & 1, &bar->abort_flag, p.status)) return false;
-        if (!warp_wait(&bar->k_full[s1], ph1, &bar->abort_flag, p.status)) return false;
+        if (jq == 0 && !warp_wait<kSuspendNs>(&bar->q_full[qb], (n_q >> 1) & 1, &bar->abort_flag, p.status)) return false;
+        if (!warp_wait<kSuspendNs>(&bar->k_full[s1], ph1, &bar->abort_flag, p.status)) return false;
         tc_fence_after();
       }
       const uint32_t kb = sK + s1 * kTileBytes + h * (kSub * kD * 2), qa = sQ + (2 * qb + t) * kTileBytes;
@@ -302,10 +306,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       Item itn{};
       if (nxt >= 0) itn = decode_item(p, nxt);
       for (int j = 0; j < it.nkt && ok; ++j) {
-        ok = warp_wait(&bar->v_full[s], ph, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->v_full[s], ph, &bar->abort_flag, p.status);
         const bool last = j + 1 == it.nkt;
         for (int h = 0; h < 2 && ok; ++h) {
-          ok = warp_wait(&bar->p_full[t][h], g_par, &bar->abort_flag, p.status);
+          ok = warp_wait<kSuspendNs>(&bar->p_full[t][h], g_par, &bar->abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t vb = sV + s * kTileBytes + h * (kSub * kD * 2);
@@ -457,7 +461,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const uint32_t sOt = sO + t * kTileBytes;
     unsigned char* sOt_ptr = smem + (size_t)(4 + 2 * kStages + t) * kTileBytes;
     auto epi_load = [&](uint32_t (&ob)[32]) -> bool {
-      if (!__all_sync(0xffffffffu, mbar_wait(&bar->o_full[t], done.par, &bar->abort_flag, p.status))) return false;
+      if (!__all_sync(0xffffffffu, mbar_wait<kSuspendNs>(&bar->o_full[t], done.par, &bar->abort_flag, p.status))) return false;
       tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
@@ -532,7 +536,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int j = u >> 1, h = u & 1;
         // warp-uniform outcome: the tensor-memory accesses below are warp-collective
         if (!__all_sync(0xffffffffu, next_ready)) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&bar->s_full[t][h], g_par, &bar->abort_flag, p.status));
+          ok = __all_sync(0xffffffffu, mbar_wait<kSuspendNs>(&bar->s_full[t][h], g_par, &bar->abort_flag, p.status));
           if (!ok) return false;
         }
         tc_fence_after();
@@ -596,9 +600,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           // tells us; after the last step of the run there are no further scores, and pv_done
           // (committed after each P V of the run's last key tile) does.
           if (has_next)
-            ok = __all_sync(0xffffffffu, mbar_wait(next_bar, next_parity, &bar->abort_flag, p.status));
+            ok = __all_sync(0xffffffffu, mbar_wait<kSuspendNs>(next_bar, next_parity, &bar->abort_flag, p.status));
           else
-            ok = __all_sync(0xffffffffu, mbar_wait(&bar->pv_done[t], 0, &bar->abort_flag, p.status));
+            ok = __all_sync(0xffffffffu, mbar_wait<kSuspendNs>(&bar->pv_done[t], 0, &bar->abort_flag, p.status));
           if (!ok) return false;
           tc_fence_after();
 #pragma unroll

@@ -34,6 +34,10 @@ namespace {
 
 using namespace tc;
 
+#ifndef JV_ATTN_SUSPEND_NS
+#define JV_ATTN_SUSPEND_NS 4000
+#endif
+constexpr uint32_t kSuspendNs = JV_ATTN_SUSPEND_NS;   // suspend-time hint of this kernel's barrier waits (tc_common.cuh)
 constexpr int kD = 64;
 constexpr int kTile = 128;                  // tokens per tile (MMA M and key-tile rows)
 constexpr int kTileBytes = kTile * kD * 2;  // 16 KB
@@ -172,7 +176,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
       for (int x = 0; x < 2 && ok; ++x) {
         const int t = 2 * s + x;
-        ok = warp_wait(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
         if (!ok) break;
         if (x < it.ntiles && elect_one()) {
           mbar_expect_tx(&bar->q_full[t], kTileBytes);
@@ -181,7 +185,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         __syncwarp();
       }
       for (int j = 0; j < it.ntiles && ok; ++j) {      // in the order the issuer needs them: K0, V0, K1, V1
-        ok = warp_wait(&bar->k_empty[s][ks], kpar, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->k_empty[s][ks], kpar, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->k_full[s][ks], kTileBytes);
@@ -189,7 +193,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         __syncwarp();
         if (++ks == kKS) { ks = 0; kpar ^= 1; }
-        ok = warp_wait(&bar->v_empty[s][vs], vpar, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->v_empty[s][vs], vpar, &bar->abort_flag, p.status);
         if (!ok) break;
         if (elect_one()) {
           mbar_expect_tx(&bar->v_full[s][vs], kTileBytes);
@@ -227,11 +231,11 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       for (int u = 0; u <= nsteps && ok; ++u) {
         const bool has_qk = u < nsteps, has_pv = u > 0;
         if (has_qk && (u & 1) == 0) {       // first half of a key tile: its K must have landed
-          ok = warp_wait(&bar->k_full[s][sk], phk, &bar->abort_flag, p.status);
+          ok = warp_wait<kSuspendNs>(&bar->k_full[s][sk], phk, &bar->abort_flag, p.status);
           if (!ok) break;
         }
         if (has_pv && ((u - 1) & 1) == 0) { // P V of a first half: its V must have landed
-          ok = warp_wait(&bar->v_full[s][sv], phv, &bar->abort_flag, p.status);
+          ok = warp_wait<kSuspendNs>(&bar->v_full[s][sv], phv, &bar->abort_flag, p.status);
           if (!ok) break;
         }
         const uint32_t kb = sK + (s * kKS + sk) * kTileBytes + (u & 1) * (kSub * kD * 2);
@@ -241,10 +245,10 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           if (x >= it.ntiles) continue;
           const int t = tb + x;
           if (u == 0) {
-            ok = warp_wait(&bar->q_full[t], qcnt[x] & 1, &bar->abort_flag, p.status);
+            ok = warp_wait<kSuspendNs>(&bar->q_full[t], qcnt[x] & 1, &bar->abort_flag, p.status);
             ++qcnt[x];
           } else {
-            ok = warp_wait(&bar->p_full[t], pcnt[x] & 1, &bar->abort_flag, p.status);
+            ok = warp_wait<kSuspendNs>(&bar->p_full[t], pcnt[x] & 1, &bar->abort_flag, p.status);
             ++pcnt[x];
           }
           if (!ok) break;
@@ -333,7 +337,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const int vx = it.x_end - it.x0;                   // valid columns of every box of this window
       float m = -INFINITY, l = 0.f;
       for (int u = 0; u < nsteps; ++u) {
-        ok = warp_wait(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
+        ok = warp_wait<kSuspendNs>(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
         if (!ok) break;
         ++scnt;
         tc_fence_after();
@@ -424,8 +428,8 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (!ok) break;
       // ---- epilogue: O / l -> bf16 -> this warp's quarter of the V tile x of this window -> one TMA store.
       // Both query tiles' last P V read that V tile: both must have retired.
-      ok = warp_wait(&bar->o_full[t], par_own, &bar->abort_flag, p.status);
-      if (ok && it.ntiles == 2) ok = warp_wait(&bar->o_full[t ^ 1], par_other, &bar->abort_flag, p.status);
+      ok = warp_wait<kSuspendNs>(&bar->o_full[t], par_own, &bar->abort_flag, p.status);
+      if (ok && it.ntiles == 2) ok = warp_wait<kSuspendNs>(&bar->o_full[t ^ 1], par_other, &bar->abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;

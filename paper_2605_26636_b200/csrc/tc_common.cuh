@@ -62,15 +62,34 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same test with a suspend-time hint: the thread may sleep in the barrier unit for up to that many
+// nanoseconds and is woken when the phase completes, instead of coming back after the (short) default
+// limit to spin through the loop around it.  A waiting warp then costs the sub-core it shares with
+// working warps fewer issue slots: worth 2.4 % on full attention, whose softmax warps are bound by
+// issue slots; the linear block's short kernels lost 1 % to it and wait without the hint.
+template <uint32_t kHintNs>
+__device__ __forceinline__ bool mbar_try_hint(uint64_t* bar, uint32_t parity) {
+  if (kHintNs == 0) return mbar_try(bar, parity);
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(kHintNs) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false (after flagging the status word and the CTA abort flag)
 // if the phase did not complete within limit_ns or another role already aborted.
+// kHintNs > 0: every try may suspend the thread for up to that long (see mbar_try_hint).
+template <uint32_t kHintNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status,
                                           unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try(bar, parity)) return true;
+  constexpr uint32_t kCheckMask = kHintNs >= 1000 ? 15u : 63u;   // tries between looks at the clock and the abort flag
   unsigned long long t0 = 0;
   for (uint32_t spin = 0;; ++spin) {
-    if (mbar_try(bar, parity)) return true;
-    if ((spin & 63u) == 63u) {
+    if (mbar_try_hint<kHintNs>(bar, parity)) return true;
+    if ((spin & kCheckMask) == kCheckMask) {
       if (*abort_flag) return false;
       const unsigned long long now = globaltimer();
       if (t0 == 0) t0 = now;
@@ -84,12 +103,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 }
 
 // The same for a whole converged warp, with a warp-uniform outcome.
+template <uint32_t kHintNs = 0>
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+  return __all_sync(0xffffffffu, mbar_wait<kHintNs>(bar, parity, abort_flag, status));
 }
 __device__ __forceinline__ bool warp_wait_limit(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, int* status,
                                                 unsigned long long limit_ns) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, limit_ns));
+  return __all_sync(0xffffffffu, mbar_wait<0>(bar, parity, abort_flag, status, limit_ns));
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
