@@ -521,6 +521,16 @@ def run_cuda(args):
                                     "frac_tensor": flops / t_ms / 1e9 / tf, "bound": bound}
         del xq, xo, wsx
 
+    # head_dim 128 (a 7B-class model: 32 heads of 128 channels; here 8 of them, B = 8, 64 x 64 grid): F on its own kernel
+    dq8 = [[t.to(dev) for t in inputs.custom_qkv(8, 8, w.N, 128, "bf16", seed=8300 + l)] for l in range(3)]
+    do8 = [torch.empty_like(dq8[0][0]) for _ in range(3)]
+    t_ms = time_calls(lambda i: jv.full_attn(*dq8[r(i)], out=do8[r(i)]), min(K, 50), 3, stream)
+    fl8 = 4.0 * 8 * 8 * w.N * w.N * 128
+    by8 = alg_bytes(8, 8, w.N, 128)
+    per["F@d128_64x64"] = {"ms": t_ms, "tokens_per_s": 8 * w.N / (t_ms * 1e-3), "GBps": by8 / t_ms / 1e6, "TFLOPs": fl8 / t_ms / 1e9,
+                           "frac_hbm": by8 / t_ms / 1e6 / hbm, "frac_tensor": fl8 / t_ms / 1e9 / tf, "bound": "tensor"}
+    del dq8, do8
+
     # ragged DepthAnythingV2-L grid (73x73, B=4): F and W with masked edge windows
     w4 = inputs.WORKLOADS["dav2_l"]
     q4 = [[t.to(dev) for t in inputs.qkv(w4, layer=l)] for l in range(3)]

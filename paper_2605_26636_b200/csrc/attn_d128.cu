@@ -1,0 +1,444 @@
+// Full softmax attention (Eq. 1) at head_dim 128 on the 5th-generation tensor cores: two 128-row
+// query tiles per CTA.  bf16 tensors.
+//
+// The four-tile kernel of head_dim 64 (attn_f4.cu) does not carry over: a 128-column fp32 accumulator
+// per query tile leaves tensor memory (512 columns) room for two tiles: per tile one 64-column score
+// buffer (the bf16 probabilities written over the scores they came from) and one 128-column
+// accumulator.  At this head_dim there are twice the tensor-core flops per exponential, so the two
+// tiles' serial chains  scores -> softmax -> P V  alternate on the tensor pipe instead of being
+// hidden behind more softmax warps.
+//
+// A tile of 128 tokens x 128 channels lies in shared memory as two 128-byte-swizzled halves of 64
+// channels (16 KB each, one TMA box each): Q K^T runs over both halves (8 MMAs of K = 16), P V
+// writes the two 64-column halves of the accumulator from the two halves of V (2 x 4 MMAs).
+//
+// Persistent CTAs (one per SM) loop over work items; an item is two consecutive query tiles of one
+// (batch, head) against all key tiles.  Warp roles (10 warps):
+//   warp 0        TMA producer: two Q tiles per item, K tiles through a ring of three, V tiles through a ring of two
+//   warp 1        MMA issuer, in steps of 64 keys, both tiles: O_t += P_t V of the previous step, then S_t = Q_t K^T
+//   warps 2-9     softmax, one thread per query row (warp w: tile (w - 2) / 4, tensor-memory quadrant w % 4):
+//                 exact two-pass softmax per step against a lazily raised reference, P as bf16 back into
+//                 tensor memory, final 1/l scaling, rows written straight to global memory (256 contiguous
+//                 bytes per row and thread)
+//
+// Every mbarrier wait is bounded: a wait that runs out sets the device status word, raises a
+// CTA-wide abort flag, and every role falls through to the common teardown (tensor memory is
+// always released).
+#include "tc_common.cuh"
+
+namespace jv {
+namespace {
+
+using namespace tc;
+
+constexpr uint32_t kSuspendNs = 4000;       // suspend-time hint of this kernel's barrier waits (tc_common.cuh)
+constexpr int kD = 128;
+constexpr int kHalfD = 64;                  // channels per swizzled half tile
+constexpr int kTile = 128;                  // tokens per tile (MMA M and key-tile rows)
+constexpr int kHalfBytes = kTile * kHalfD * 2;   // 16 KB
+constexpr int kTileBytes = 2 * kHalfBytes;       // 32 KB
+constexpr int kQT = 2;                      // query tiles per work item
+constexpr int kKS = 3, kVS = 2;             // K and V ring depths
+constexpr int kWarps = 10;
+constexpr int kThreads = kWarps * 32;
+constexpr int kFirstSoftmaxWarp = 2;
+constexpr uint32_t kTmemCols = 512;
+constexpr int kSub = 64;                    // keys per step
+constexpr int kPolyOf8 = 0;                 // the tensor pipe, not MUFU, is the tighter unit at this head_dim
+// Tensor-memory columns: S_t (and P_t over its first 32 columns) at 64 t, O_t at 128 + 128 t
+constexpr uint32_t kColS = 0, kColO = 128;
+
+struct D128Params {
+  __nv_bfloat16* o;      // [B*H, N, 128]
+  int* status;
+  int N;                 // tokens per (batch, head)
+  int ntiles;            // key (and query) tiles per head: ceil(N / 128)
+  int qgroups;           // pairs of query tiles per head
+  int total_items;       // (batch*head, pair), pair fastest
+  FastDiv div_qgroups;
+  int H;                 // heads per batch element: the inputs are addressed by (head, batch)
+  FastDiv div_H;
+  float scale_log2;      // softmax scale * log2(e)
+};
+
+struct __align__(8) Barriers {
+  uint64_t q_full[kQT], q_empty[kQT];
+  uint64_t k_full[kKS], k_empty[kKS], v_full[kVS], v_empty[kVS];
+  uint64_t s_full[kQT], p_full[kQT], o_full[kQT];
+  uint64_t drain;
+  uint32_t tmem_base;
+  volatile uint32_t abort_flag;
+};
+constexpr size_t kSmemTiles = (kQT + kKS + kVS) * (size_t)kTileBytes;          // Q[2] K[3] V[2] = 224 KB
+constexpr size_t kSmemBytes = kSmemTiles + sizeof(Barriers) + 1024;            // + alignment slack
+
+constexpr uint32_t kIdescQK = idesc(kTile, kSub, 0);       // S = Q K^T: M128 N64, both operands K-major
+constexpr uint32_t kIdescPV = idesc(kTile, kHalfD, 1);     // O half = P V half: M128 N64, V MN-major
+
+// ---- the kernel ------------------------------------------------------------------
+// CTA c works on items c, c + gridDim.x, ...  Every role walks the same item sequence on its own;
+// ring stages and barrier parities follow running counters.  The second query tile of a head's last
+// item does not exist when the head has an odd number of tiles: its softmax warps skip the item, the
+// issuer still frees its Q buffer so that arrival counts hold.
+__global__ void __launch_bounds__(kThreads, 1)
+attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                 const __grid_constant__ CUtensorMap mapV, const D128Params p) {
+  extern __shared__ unsigned char smem_raw[];
+  // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
+  const uint32_t sQ = smem_u32(smem), sK = sQ + kQT * kTileBytes, sV = sK + kKS * kTileBytes;
+
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
+
+  // a timeout flagged earlier (by any CTA or launch) makes the rest leave at once
+  if (threadIdx.x == 0) bar->tmem_base = *reinterpret_cast<volatile int*>(p.status);
+  __syncthreads();
+  if (bar->tmem_base != 0) return;
+  __syncthreads();
+
+  if (threadIdx.x == 0) {
+    for (int t = 0; t < kQT; ++t) {
+      mbar_init(&bar->q_full[t], 1);
+      mbar_init(&bar->q_empty[t], 1);
+      mbar_init(&bar->s_full[t], 1);
+      mbar_init(&bar->p_full[t], 128);
+      mbar_init(&bar->o_full[t], 1);
+    }
+    for (int s = 0; s < kKS; ++s) {
+      mbar_init(&bar->k_full[s], 1);
+      mbar_init(&bar->k_empty[s], 1);
+    }
+    for (int s = 0; s < kVS; ++s) {
+      mbar_init(&bar->v_full[s], 1);
+      mbar_init(&bar->v_empty[s], 1);
+    }
+    mbar_init(&bar->drain, 1);
+    bar->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bar->tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
+
+  const int item0 = blockIdx.x, item_step = gridDim.x;
+  const int ntiles = p.ntiles, nsteps = 2 * p.ntiles;
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    // a tile = two boxes of 64 channels x 128 tokens, one per swizzled half
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* map, uint64_t* full, int tok, int h, int b) {
+      mbar_expect_tx(full, kTileBytes);
+      tma_load_4d(dst, map, full, 0, tok, h, b);
+      tma_load_4d(dst + kHalfBytes, map, full, kHalfD, tok, h, b);
+    };
+    bool ok = true;
+    int n = 0;                 // items seen
+    int ks = 0, vs = 0;        // ring stages of the next K and V tile
+    uint32_t kpar = 1, vpar = 1;   // parity of the "empty" phase this pass over each ring waits for
+    int issued_v = 0;          // for the abort path: V copies issued so far
+    for (int i = item0; i < p.total_items && ok; i += item_step) {
+      const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
+      const int b = fdiv(bh, p.div_H), h = bh - b * p.H;   // coordinates of the input tensor maps
+      for (int t = 0; t < kQT && ok; ++t) {
+        ok = warp_wait<kSuspendNs>(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
+        if (!ok) break;
+        if (qt0 + t < ntiles && elect_one()) load_tile(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], (qt0 + t) * kTile, h, b);
+        __syncwarp();
+      }
+      for (int j = 0; j < ntiles && ok; ++j) {
+        ok = warp_wait<kSuspendNs>(&bar->k_empty[ks], kpar, &bar->abort_flag, p.status);
+        if (!ok) break;
+        if (elect_one()) load_tile(sK + ks * kTileBytes, &mapK, &bar->k_full[ks], j * kTile, h, b);
+        __syncwarp();
+        if (++ks == kKS) { ks = 0; kpar ^= 1; }
+        ok = warp_wait<kSuspendNs>(&bar->v_empty[vs], vpar, &bar->abort_flag, p.status);
+        if (!ok) break;
+        if (elect_one()) load_tile(sV + vs * kTileBytes, &mapV, &bar->v_full[vs], j * kTile, h, b);
+        __syncwarp();
+        ++issued_v;
+        if (++vs == kVS) { vs = 0; vpar ^= 1; }
+      }
+      ++n;
+    }
+    if (!ok && lane == 0) {
+      // let the copies still in flight land before the CTA leaves (bounded by the same limit)
+      const unsigned long long t0 = globaltimer();
+      for (int g = max(0, issued_v - kVS); g < issued_v; ++g)
+        while (!mbar_try(&bar->v_full[g % kVS], (g / kVS) & 1) && globaltimer() - t0 < kWaitLimitNs) {}
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer, both query tiles =================
+    // Per item and query tile t the work is a chain over 64-key steps u (key tile u / 2, half u % 2):
+    //   S_t(u) = Q_t K(u)^T          8 MMAs, M128 N64 K16, operands in shared memory (two channel halves)
+    //   O_t   += P_t(u) V(u)         2 x 4 MMAs, M128 N64 K16, A = P in tensor memory, one per channel half of V
+    // P_t(u) lies over S_t(u), so S_t(u + 1) is issued behind P_t(u) V(u): the tensor pipe executes one
+    // thread's MMAs in issue order.  The commit that publishes S_t(u + 1) therefore also tells the
+    // softmax warps that P_t(u) V(u) has retired and O_t is quiescent.
+    bool ok = true;
+    int sk = 0, sv = 0;                     // ring stages of the score key tile and of the P V key tile
+    uint32_t phk = 0, phv = 0;              // and their "full" parities
+    uint32_t pcnt[2] = {0, 0};              // steps published so far per tile: parity of p_full
+    uint32_t qcnt[2] = {0, 0};              // items in which the tile existed: parity of q_full
+    for (int i = item0; i < p.total_items && ok; i += item_step) {
+      const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
+      const bool ex[2] = {true, qt0 + 1 < ntiles};
+      for (int u = 0; u <= nsteps && ok; ++u) {
+        const bool has_qk = u < nsteps, has_pv = u > 0;
+        if (has_qk && (u & 1) == 0) {       // first half of a key tile: its K must have landed
+          ok = warp_wait<kSuspendNs>(&bar->k_full[sk], phk, &bar->abort_flag, p.status);
+          if (!ok) break;
+        }
+        if (has_pv && ((u - 1) & 1) == 0) { // P V of a first half: its V must have landed
+          ok = warp_wait<kSuspendNs>(&bar->v_full[sv], phv, &bar->abort_flag, p.status);
+          if (!ok) break;
+        }
+        // 64 keys = rows 64 (u % 2) .. of each 128-row half tile: 8 KB into the half
+        const uint32_t kb = sK + sk * kTileBytes + (u & 1) * (kSub * kHalfD * 2);
+        const uint32_t vb = sV + sv * kTileBytes + ((u - 1) & 1) * (kSub * kHalfD * 2);
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          if (!ex[x]) continue;
+          if (u == 0) {
+            ok = warp_wait<kSuspendNs>(&bar->q_full[x], qcnt[x] & 1, &bar->abort_flag, p.status);
+            ++qcnt[x];
+          } else {
+            ok = warp_wait<kSuspendNs>(&bar->p_full[x], pcnt[x] & 1, &bar->abort_flag, p.status);
+            ++pcnt[x];
+          }
+          if (!ok) break;
+          tc_fence_after();
+          if (elect_one()) {                 // one lane issues the step's MMAs back to back
+            if (has_pv) {
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                const uint64_t dv = smem_desc(vb + half * kHalfBytes);
+#pragma unroll
+                for (int c = 0; c < kSub / 16; ++c)
+                  mma_ts_1(tmem + kColO + x * kD + half * kHalfD, tmem + kColS + x * kSub + c * 8, desc_advance(dv, c * 2048),
+                           kIdescPV, (u > 1 || c > 0) ? 1u : 0u);
+              }
+            }
+            if (has_qk) {
+#pragma unroll
+              for (int half = 0; half < 2; ++half) {
+                const uint64_t dq = smem_desc(sQ + x * kTileBytes + half * kHalfBytes), dk = smem_desc(kb + half * kHalfBytes);
+#pragma unroll
+                for (int c = 0; c < kHalfD / 16; ++c)
+                  mma_ss_1(tmem + kColS + x * kSub, desc_advance(dq, c * 32), desc_advance(dk, c * 32), kIdescQK,
+                           (half > 0 || c > 0) ? 1u : 0u);
+              }
+            }
+          }
+          __syncwarp();
+          if (has_qk) tc_commit(&bar->s_full[x]);
+          else tc_commit(&bar->o_full[x]);
+        }
+        if (!ok) break;
+        if (has_pv && ((u - 1) & 1) == 1) { // both halves of the V tile are in flight or done
+          tc_commit(&bar->v_empty[sv]);
+          if (++sv == kVS) { sv = 0; phv ^= 1; }
+        }
+        if (has_qk && (u & 1) == 1) {
+          tc_commit(&bar->k_empty[sk]);
+          if (u == nsteps - 1) {            // the item's last scores: its query tiles may be replaced
+            tc_commit(&bar->q_empty[0]);
+            tc_commit(&bar->q_empty[1]);
+          }
+          if (++sk == kKS) { sk = 0; phk ^= 1; }
+        }
+      }
+    }
+    // Teardown: every MMA issued so far must have retired before tensor memory is released.
+    tc_commit(&bar->drain);
+    if (lane == 0) {
+      const unsigned long long t0 = globaltimer();
+      while (!mbar_try(&bar->drain, 0) && globaltimer() - t0 < kWaitLimitNs) {}
+    }
+    __syncwarp();
+  } else {
+    // ================= softmax + epilogue: one thread per query row =================
+    const int t = (warp - kFirstSoftmaxWarp) >> 2;  // query tile of this warp
+    const int q4 = warp & 3;                        // tensor-memory quadrant a warp may touch: warp % 4
+    const uint32_t lane_base = (uint32_t)(q4 << 5) << 16;
+    const uint32_t tS = tmem + lane_base + kColS + t * kSub;   // scores; probabilities over their first 32 columns
+    const uint32_t tO = tmem + lane_base + kColO + t * kD;
+    const float sl2 = p.scale_log2;
+    const float kLazy = 8.f / sl2;                 // the reference maximum moves only when it grew by > 2^8
+    const uint64_t sl2x2 = pack2(sl2, sl2);
+    const int last_valid = p.N - (ntiles - 1) * kTile;         // keys that exist in the last key tile
+    bool ok = true;
+    uint32_t scnt = 0;                // steps seen by this tile: parity of s_full
+    uint32_t ocnt = 0;                // items seen by this tile: parity of o_full
+
+    for (int i = item0; i < p.total_items && ok; i += item_step) {
+      const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
+      if (qt0 + t >= ntiles) continue;              // this query tile does not exist
+      float m = -INFINITY, l = 0.f;
+      for (int u = 0; u < nsteps; ++u) {
+        ok = warp_wait<kSuspendNs>(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
+        if (!ok) break;
+        ++scnt;
+        tc_fence_after();
+        uint32_t va[32], vb2[32];
+        if ((u >> 1) == ntiles - 1 && last_valid < kTile) {
+          // Last key tile of a sequence that is not a multiple of 128: overwrite the scores of keys
+          // that do not exist with -inf in tensor memory, then treat the step like any other.
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            const int nv = last_valid - (64 * (u & 1) + 32 * c);      // valid keys among these 32
+            if (nv < 32) {                                             // warp-uniform
+              tmem_ld32(tS + 32 * c, va);
+              tmem_wait_ld(va);
+#pragma unroll
+              for (int x = 0; x < 32; ++x)
+                if (x >= nv) va[x] = kNegInf;     // exp2(-inf) = 0 and -inf never wins the maximum
+              tmem_st32(tS + 32 * c, va);
+            }
+          }
+          tmem_wait_st();
+        }
+        // ---- pass 1: the step's maximum; both halves of the scores stay in registers for pass 2
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        tmem_ld32(tS, va);
+        tmem_ld32(tS + 32, vb2);
+        tmem_wait_ld(va);
+        tmem_wait_ld(vb2);
+        max32(va, mx4);
+        max32(vb2, mx4);
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        float o_scale = 1.f;
+        if (mx > m + kLazy) {          // always true on the first step (m = -inf, mx finite)
+          o_scale = ex2((m - mx) * sl2);            // first step: exp2(-inf) = 0
+          l *= o_scale;
+          m = mx;
+        }
+        if (u > 0 && __any_sync(0xffffffffu, o_scale != 1.f)) {
+          // Rare: the reference moved.  O_t may be touched: the scores just waited for were committed
+          // behind the previous step's P V, and the next P V waits for this step's P.
+#pragma unroll 1
+          for (int c = 0; c < kD / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(tO + 32 * c, v);
+            tmem_wait_ld(v);
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(__uint_as_float(v[x]) * o_scale);
+            tmem_st32(tO + 32 * c, v);
+          }
+          tmem_wait_st();
+        }
+        // ---- pass 2: exponentials against the reference, P over the scores just consumed
+        const float mneg = -m * sl2;
+        const uint64_t mnegx2 = pack2(mneg, mneg);
+        uint64_t lsum[4] = {0ull, 0ull, 0ull, 0ull};
+        uint32_t pk[16];
+        exp32<false, kPolyOf8>(va, sl2x2, mnegx2, lsum, pk, mx4);
+        tmem_st16(tS, pk);
+        exp32<false, kPolyOf8>(vb2, sl2x2, mnegx2, lsum, pk, mx4);
+        tmem_st16(tS + 16, pk);
+        float a0, a1, b0, b1;
+        unpack2(add2(lsum[0], lsum[1]), a0, a1);
+        unpack2(add2(lsum[2], lsum[3]), b0, b1);
+        l += (a0 + a1) + (b0 + b1);
+        // publish P
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bar->p_full[t]);
+      }
+      if (!ok) break;
+      // ---- epilogue: O / l -> bf16 -> this thread's row, 256 contiguous bytes of global memory
+      ok = warp_wait<kSuspendNs>(&bar->o_full[t], ocnt & 1, &bar->abort_flag, p.status);
+      if (!ok) break;
+      ++ocnt;
+      tc_fence_after();
+      const float inv = 1.f / l;
+      const int tok = (qt0 + t) * kTile + 32 * q4 + lane;       // this thread's token
+      __nv_bfloat16* dst = p.o + ((size_t)bh * p.N + (size_t)tok) * kD;
+#pragma unroll 1
+      for (int c = 0; c < kD / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld32(tO + 32 * c, v);
+        tmem_wait_ld(v);
+        if (tok < p.N) {
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+            *reinterpret_cast<uint4*>(dst + 32 * c + 8 * x) =
+                make_uint4(pack_bf16(__uint_as_float(v[8 * x]) * inv, __uint_as_float(v[8 * x + 1]) * inv),
+                           pack_bf16(__uint_as_float(v[8 * x + 2]) * inv, __uint_as_float(v[8 * x + 3]) * inv),
+                           pack_bf16(__uint_as_float(v[8 * x + 4]) * inv, __uint_as_float(v[8 * x + 5]) * inv),
+                           pack_bf16(__uint_as_float(v[8 * x + 6]) * inv, __uint_as_float(v[8 * x + 7]) * inv));
+        }
+      }
+      tc_fence_before();
+    }
+  }
+
+  // ================= common teardown =================
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+}
+
+}  // namespace
+
+bool attn_d128_supported(const AttnArgs& a) {
+  if (a.dtype != JV_BF16 || a.D != kD) return false;
+  const int64_t N = (int64_t)a.Hg * a.Wg;
+  if (N < kTile) return false;                              // shorter sequences: the generic kernel
+  const int64_t ntiles = (N + kTile - 1) / kTile;
+  if ((ntiles + kQT - 1) / kQT * a.BH > 0x7fffffffll) return false;
+  return encode_fn() != nullptr;
+}
+
+cudaError_t launch_attn_d128(const AttnArgs& a, int* status, cudaStream_t st) {
+  EncodeFn enc = encode_fn();
+  if (!enc) return cudaErrorNotSupported;
+  const int N = a.Hg * a.Wg;
+  CUtensorMap maps[3];
+  const void* ptrs[3] = {a.q, a.k, a.v};
+  // the inputs as (d, token, head, batch) with the caller's strides; a box is one 64-channel half of a tile
+  const cuuint64_t idims[4] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
+  const cuuint64_t istrides[3] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)a.in.head * 2, (cuuint64_t)a.in.batch * 2};
+  const cuuint32_t ibox[4] = {(cuuint32_t)kHalfD, (cuuint32_t)kTile, 1, 1};
+  const cuuint32_t iestr[4] = {1, 1, 1, 1};
+  for (int i = 0; i < 3; ++i) {
+    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), idims, istrides, ibox, iestr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  }
+  static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
+  cudaError_t e = smem_opt_in.run([] {
+    return cudaFuncSetAttribute(attn_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  });
+  if (e != cudaSuccess) return e;
+  D128Params p;
+  p.o = (__nv_bfloat16*)a.o;
+  p.status = status;
+  p.N = N;
+  p.ntiles = ceil_div(N, kTile);
+  p.qgroups = ceil_div(p.ntiles, kQT);
+  p.total_items = p.qgroups * a.BH;
+  p.div_qgroups = make_fastdiv((uint32_t)p.qgroups);
+  p.H = a.H;
+  p.div_H = make_fastdiv((uint32_t)a.H);
+  p.scale_log2 = a.scale * 1.4426950408889634f;
+  const int num_sms = device_sm_count();
+  const int grid = p.total_items < num_sms ? p.total_items : num_sms;
+  attn_d128_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], p);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace jv
