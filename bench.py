@@ -629,7 +629,10 @@ def run_single(args):
     dev = torch.device("cuda:0")
     w = inputs.WORKLOADS[args.workload]
     stream = torch.cuda.current_stream()
-    sets = [[t.to(dev) for t in inputs.qkv(w, layer=l)] for l in range(3)]
+    if args.single == "F@d128":     # the workload's token count with half the heads at twice the channels
+        sets = [[t.to(dev) for t in inputs.custom_qkv(w.B, max(1, w.H // 2), w.N, 128, "bf16", seed=8300 + l)] for l in range(3)]
+    else:
+        sets = [[t.to(dev) for t in inputs.qkv(w, layer=l)] for l in range(3)]
     outs = [torch.empty_like(s[0]) for s in sets]
     C = w.H * w.D
     dwc = None
@@ -677,7 +680,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--single", choices=["L", "L+dwc", "W", "F", "qkv_proj", "out_proj"], default=None,
+    ap.add_argument("--single", choices=["L", "L+dwc", "W", "F", "F@d128", "qkv_proj", "out_proj"], default=None,
                     help="time one mixer alone (used for profiler captures)")
     ap.add_argument("--workload", default="dinov3_l", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--record-traffic", default=None, metavar="CSV",
