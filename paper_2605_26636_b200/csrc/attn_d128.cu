@@ -2,11 +2,11 @@
 // query tiles per CTA.  bf16 tensors.
 //
 // The four-tile kernel of head_dim 64 (attn_f4.cu) does not carry over: a 128-column fp32 accumulator
-// per query tile leaves tensor memory (512 columns) room for two tiles: per tile one 64-column score
-// buffer (the bf16 probabilities written over the scores they came from) and one 128-column
-// accumulator.  At this head_dim there are twice the tensor-core flops per exponential, so the two
-// tiles' serial chains  scores -> softmax -> P V  alternate on the tensor pipe instead of being
-// hidden behind more softmax warps.
+// per query tile leaves tensor memory (512 columns) room for two tiles: per tile two 64-column score
+// buffers (the bf16 probabilities written over the scores they came from) and one 128-column
+// accumulator.  With two buffers the scores of the next step are computed while the softmax works on
+// this one, so a tile's chain is  softmax -> P V  only; at this head_dim there are twice the
+// tensor-core flops per exponential, and the tensor pipe and MUFU are about equally loaded.
 //
 // A tile of 128 tokens x 128 channels lies in shared memory as two 128-byte-swizzled halves of 64
 // channels (16 KB each, one TMA box each): Q K^T runs over both halves (8 MMAs of K = 16), P V
@@ -15,7 +15,8 @@
 // Persistent CTAs (one per SM) loop over work items; an item is two consecutive query tiles of one
 // (batch, head) against all key tiles.  Warp roles (10 warps):
 //   warp 0        TMA producer: two Q tiles per item, K tiles through a ring of three, V tiles through a ring of two
-//   warp 1        MMA issuer, in steps of 64 keys, both tiles: O_t += P_t V of the previous step, then S_t = Q_t K^T
+//   warp 1        MMA issuer, in steps of 64 keys, both tiles: O_t += P_t V of step u, then S_t = Q_t K^T of step u + 2
+//                 into the score buffer that P V has just read
 //   warps 2-9     softmax, one thread per query row (warp w: tile (w - 2) / 4, tensor-memory quadrant w % 4):
 //                 exact two-pass softmax per step against a lazily raised reference, P as bf16 back into
 //                 tensor memory, final 1/l scaling, rows written straight to global memory (256 contiguous
@@ -44,9 +45,13 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kFirstSoftmaxWarp = 2;
 constexpr uint32_t kTmemCols = 512;
 constexpr int kSub = 64;                    // keys per step
-constexpr int kPolyOf8 = 1;                 // of every 8 score pairs, this many take the polynomial exponential (measured: 0 -1.5 %, 2 same, 3 -3.5 %)
-// Tensor-memory columns: S_t (and P_t over its first 32 columns) at 64 t, O_t at 128 + 128 t
-constexpr uint32_t kColS = 0, kColO = 128;
+#ifndef JV_D128_POLY
+#define JV_D128_POLY 1
+#endif
+constexpr int kPolyOf8 = JV_D128_POLY;      // of every 8 score pairs, this many take the polynomial exponential
+// Tensor-memory columns: score buffer h of tile t (and its P over the first 32 columns) at 128 t + 64 h,
+// O_t at 256 + 128 t
+constexpr uint32_t kColS = 0, kColO = 256;
 
 struct D128Params {
   __nv_bfloat16* o;      // [B*H, N, 128]
@@ -64,7 +69,8 @@ struct D128Params {
 struct __align__(8) Barriers {
   uint64_t q_full[kQT], q_empty[kQT];
   uint64_t k_full[kKS], k_empty[kKS], v_full[kVS], v_empty[kVS];
-  uint64_t s_full[kQT], p_full[kQT], o_full[kQT];
+  uint64_t s_full[kQT][2], p_full[kQT][2];   // per query tile and score buffer
+  uint64_t pv_done[kQT];                     // one phase per step: its P V has retired
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
@@ -101,9 +107,11 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     for (int t = 0; t < kQT; ++t) {
       mbar_init(&bar->q_full[t], 1);
       mbar_init(&bar->q_empty[t], 1);
-      mbar_init(&bar->s_full[t], 1);
-      mbar_init(&bar->p_full[t], 128);
-      mbar_init(&bar->o_full[t], 1);
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(&bar->s_full[t][h], 1);
+        mbar_init(&bar->p_full[t][h], 128);
+      }
+      mbar_init(&bar->pv_done[t], 1);
     }
     for (int s = 0; s < kKS; ++s) {
       mbar_init(&bar->k_full[s], 1);
@@ -180,81 +188,102 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     // Per item and query tile t the work is a chain over 64-key steps u (key tile u / 2, half u % 2):
     //   S_t(u) = Q_t K(u)^T          8 MMAs, M128 N64 K16, operands in shared memory (two channel halves)
     //   O_t   += P_t(u) V(u)         2 x 4 MMAs, M128 N64 K16, A = P in tensor memory, one per channel half of V
-    // P_t(u) lies over S_t(u), so S_t(u + 1) is issued behind P_t(u) V(u): the tensor pipe executes one
-    // thread's MMAs in issue order.  The commit that publishes S_t(u + 1) therefore also tells the
-    // softmax warps that P_t(u) V(u) has retired and O_t is quiescent.
+    // Two score buffers per tile: the scores of steps u and u + 1 are in flight or done while the softmax
+    // works on step u, so it never waits for Q K^T in steady state.  P_t(u) lies over S_t(u) in buffer u % 2,
+    // and S_t(u + 2) is issued into that buffer behind P_t(u) V(u): the tensor pipe executes one thread's
+    // MMAs in issue order.  pv_done tells the softmax warps that a step's P V has retired (O_t quiescent).
     bool ok = true;
     int sk = 0, sv = 0;                     // ring stages of the score key tile and of the P V key tile
     uint32_t phk = 0, phv = 0;              // and their "full" parities
-    uint32_t pcnt[2] = {0, 0};              // steps published so far per tile: parity of p_full
+    uint32_t pcnt[2][2] = {{0, 0}, {0, 0}}; // publications seen so far per tile and buffer: parity of p_full
     uint32_t qcnt[2] = {0, 0};              // items in which the tile existed: parity of q_full
     for (int i = item0; i < p.total_items && ok; i += item_step) {
       const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
       const bool ex[2] = {true, qt0 + 1 < ntiles};
-      for (int u = 0; u <= nsteps && ok; ++u) {
-        const bool has_qk = u < nsteps, has_pv = u > 0;
-        if (has_qk && (u & 1) == 0) {       // first half of a key tile: its K must have landed
-          ok = warp_wait<kSuspendNs>(&bar->k_full[sk], phk, &bar->abort_flag, p.status);
-          if (!ok) break;
+      // Scores of step u: scores_begin waits for the key tile, scores_tile issues tile x's MMAs into buffer
+      // u % 2 (the caller has made sure that the buffer is free: its previous P V has been issued, and one
+      // thread's MMAs execute in issue order), scores_end hands the key tile and the query tiles back.
+      auto scores_begin = [&](int u) -> bool {
+        if ((u & 1) == 0 && !warp_wait<kSuspendNs>(&bar->k_full[sk], phk, &bar->abort_flag, p.status)) return false;
+        tc_fence_after();
+        return true;
+      };
+      auto scores_tile = [&](int u, int x) {
+        const uint32_t kb = sK + sk * kTileBytes + (u & 1) * (kSub * kHalfD * 2);   // 64 keys = 8 KB into each half tile
+        if (elect_one()) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const uint64_t dq = smem_desc(sQ + x * kTileBytes + half * kHalfBytes), dk = smem_desc(kb + half * kHalfBytes);
+#pragma unroll
+            for (int c = 0; c < kHalfD / 16; ++c)
+              mma_ss_1(tmem + kColS + x * 128 + (u & 1) * kSub, desc_advance(dq, c * 32), desc_advance(dk, c * 32), kIdescQK,
+                       (half > 0 || c > 0) ? 1u : 0u);
+          }
         }
-        if (has_pv && ((u - 1) & 1) == 0) { // P V of a first half: its V must have landed
+        __syncwarp();
+        tc_commit(&bar->s_full[x][u & 1]);
+      };
+      auto scores_end = [&](int u) {
+        if ((u & 1) == 1) {
+          tc_commit(&bar->k_empty[sk]);
+          if (++sk == kKS) { sk = 0; phk ^= 1; }
+        }
+        if (u == nsteps - 1) {              // the item's last scores: its query tiles may be replaced
+          tc_commit(&bar->q_empty[0]);
+          tc_commit(&bar->q_empty[1]);
+        }
+      };
+      for (int x = 0; x < 2 && ok; ++x) {
+        if (!ex[x]) continue;
+        ok = warp_wait<kSuspendNs>(&bar->q_full[x], qcnt[x] & 1, &bar->abort_flag, p.status);
+        ++qcnt[x];
+      }
+      for (int u = 0; u < 2 && ok; ++u) {   // (a key tile is two steps: nsteps >= 2)
+        ok = scores_begin(u);
+        if (!ok) break;
+        for (int x = 0; x < 2; ++x)
+          if (ex[x]) scores_tile(u, x);
+        scores_end(u);
+      }
+      for (int u = 0; u < nsteps && ok; ++u) {
+        const int hb = u & 1;
+        const bool more = u + 2 < nsteps;   // the buffer of step u is free behind its P V: the scores of step u + 2 go there
+        if (hb == 0) {                      // P V of a first half: its V must have landed
           ok = warp_wait<kSuspendNs>(&bar->v_full[sv], phv, &bar->abort_flag, p.status);
           if (!ok) break;
         }
-        // 64 keys = rows 64 (u % 2) .. of each 128-row half tile: 8 KB into the half
-        const uint32_t kb = sK + sk * kTileBytes + (u & 1) * (kSub * kHalfD * 2);
-        const uint32_t vb = sV + sv * kTileBytes + ((u - 1) & 1) * (kSub * kHalfD * 2);
+        if (more) {
+          ok = scores_begin(u + 2);
+          if (!ok) break;
+        }
+        const uint32_t vb = sV + sv * kTileBytes + hb * (kSub * kHalfD * 2);
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           if (!ex[x]) continue;
-          if (u == 0) {
-            ok = warp_wait<kSuspendNs>(&bar->q_full[x], qcnt[x] & 1, &bar->abort_flag, p.status);
-            ++qcnt[x];
-          } else {
-            ok = warp_wait<kSuspendNs>(&bar->p_full[x], pcnt[x] & 1, &bar->abort_flag, p.status);
-            ++pcnt[x];
-          }
+          ok = warp_wait<kSuspendNs>(&bar->p_full[x][hb], pcnt[x][hb] & 1, &bar->abort_flag, p.status);
+          ++pcnt[x][hb];
           if (!ok) break;
           tc_fence_after();
           if (elect_one()) {                 // one lane issues the step's MMAs back to back
-            if (has_pv) {
 #pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                const uint64_t dv = smem_desc(vb + half * kHalfBytes);
+            for (int half = 0; half < 2; ++half) {
+              const uint64_t dv = smem_desc(vb + half * kHalfBytes);
 #pragma unroll
-                for (int c = 0; c < kSub / 16; ++c)
-                  mma_ts_1(tmem + kColO + x * kD + half * kHalfD, tmem + kColS + x * kSub + c * 8, desc_advance(dv, c * 2048),
-                           kIdescPV, (u > 1 || c > 0) ? 1u : 0u);
-              }
-            }
-            if (has_qk) {
-#pragma unroll
-              for (int half = 0; half < 2; ++half) {
-                const uint64_t dq = smem_desc(sQ + x * kTileBytes + half * kHalfBytes), dk = smem_desc(kb + half * kHalfBytes);
-#pragma unroll
-                for (int c = 0; c < kHalfD / 16; ++c)
-                  mma_ss_1(tmem + kColS + x * kSub, desc_advance(dq, c * 32), desc_advance(dk, c * 32), kIdescQK,
-                           (half > 0 || c > 0) ? 1u : 0u);
-              }
+              for (int c = 0; c < kSub / 16; ++c)
+                mma_ts_1(tmem + kColO + x * kD + half * kHalfD, tmem + kColS + x * 128 + hb * kSub + c * 8, desc_advance(dv, c * 2048),
+                         kIdescPV, (u > 0 || c > 0) ? 1u : 0u);
             }
           }
           __syncwarp();
-          if (has_qk) tc_commit(&bar->s_full[x]);
-          else tc_commit(&bar->o_full[x]);
+          tc_commit(&bar->pv_done[x]);
+          if (more) scores_tile(u + 2, x);
         }
         if (!ok) break;
-        if (has_pv && ((u - 1) & 1) == 1) { // both halves of the V tile are in flight or done
+        if (hb == 1) {                      // both halves of the V tile are in flight or done
           tc_commit(&bar->v_empty[sv]);
           if (++sv == kVS) { sv = 0; phv ^= 1; }
         }
-        if (has_qk && (u & 1) == 1) {
-          tc_commit(&bar->k_empty[sk]);
-          if (u == nsteps - 1) {            // the item's last scores: its query tiles may be replaced
-            tc_commit(&bar->q_empty[0]);
-            tc_commit(&bar->q_empty[1]);
-          }
-          if (++sk == kKS) { sk = 0; phk ^= 1; }
-        }
+        if (more) scores_end(u + 2);
       }
     }
     // Teardown: every MMA issued so far must have retired before tensor memory is released.
@@ -269,24 +298,25 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const int t = (warp - kFirstSoftmaxWarp) >> 2;  // query tile of this warp
     const int q4 = warp & 3;                        // tensor-memory quadrant a warp may touch: warp % 4
     const uint32_t lane_base = (uint32_t)(q4 << 5) << 16;
-    const uint32_t tS = tmem + lane_base + kColS + t * kSub;   // scores; probabilities over their first 32 columns
+    const uint32_t tS0 = tmem + lane_base + kColS + t * 128;   // score buffer 0 (buffer 1: + 64); probabilities over a buffer's first 32 columns
     const uint32_t tO = tmem + lane_base + kColO + t * kD;
     const float sl2 = p.scale_log2;
     const float kLazy = 8.f / sl2;                 // the reference maximum moves only when it grew by > 2^8
     const uint64_t sl2x2 = pack2(sl2, sl2);
     const int last_valid = p.N - (ntiles - 1) * kTile;         // keys that exist in the last key tile
     bool ok = true;
-    uint32_t scnt = 0;                // steps seen by this tile: parity of s_full
-    uint32_t ocnt = 0;                // items seen by this tile: parity of o_full
+    uint32_t scnt[2] = {0, 0};        // steps seen by this tile per score buffer: parity of s_full
+    uint32_t g = 0;                   // steps seen by this tile in all: phase of pv_done
 
     for (int i = item0; i < p.total_items && ok; i += item_step) {
       const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
       if (qt0 + t >= ntiles) continue;              // this query tile does not exist
       float m = -INFINITY, l = 0.f;
       for (int u = 0; u < nsteps; ++u) {
-        ok = warp_wait<kSuspendNs>(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
+        const uint32_t tS = tS0 + (u & 1) * kSub;
+        ok = warp_wait<kSuspendNs>(&bar->s_full[t][u & 1], scnt[u & 1] & 1, &bar->abort_flag, p.status);
         if (!ok) break;
-        ++scnt;
+        ++scnt[u & 1];
         tc_fence_after();
         uint32_t va[32], vb2[32];
         if ((u >> 1) == ntiles - 1 && last_valid < kTile) {
@@ -315,6 +345,7 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         max32(va, mx4);
         max32(vb2, mx4);
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        bool pv_seen = u == 0;         // every step looks at the phase of the previous step's P V exactly once
         float o_scale = 1.f;
         if (mx > m + kLazy) {          // always true on the first step (m = -inf, mx finite)
           o_scale = ex2((m - mx) * sl2);            // first step: exp2(-inf) = 0
@@ -322,8 +353,12 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
           m = mx;
         }
         if (u > 0 && __any_sync(0xffffffffu, o_scale != 1.f)) {
-          // Rare: the reference moved.  O_t may be touched: the scores just waited for were committed
-          // behind the previous step's P V, and the next P V waits for this step's P.
+          // Rare: the reference moved.  O_t may be touched once the previous step's P V has retired
+          // (phase g - 1 of pv_done); the next P V waits for this step's P.
+          ok = warp_wait<kSuspendNs>(&bar->pv_done[t], (g - 1) & 1, &bar->abort_flag, p.status);
+          if (!ok) break;
+          pv_seen = true;
+          tc_fence_after();
 #pragma unroll 1
           for (int c = 0; c < kD / 32; ++c) {
             uint32_t v[32];
@@ -348,16 +383,22 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         unpack2(add2(lsum[0], lsum[1]), a0, a1);
         unpack2(add2(lsum[2], lsum[3]), b0, b1);
         l += (a0 + a1) + (b0 + b1);
+        // A parity wait must not skip a phase: the previous step's P V is waited for here at the latest
+        // (it retired long ago), before this step's P can set the next one going.
+        if (!pv_seen) {
+          ok = warp_wait<kSuspendNs>(&bar->pv_done[t], (g - 1) & 1, &bar->abort_flag, p.status);
+          if (!ok) break;
+        }
         // publish P
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&bar->p_full[t]);
+        mbar_arrive(&bar->p_full[t][u & 1]);
+        ++g;
       }
       if (!ok) break;
       // ---- epilogue: O / l -> bf16 -> this thread's row, 256 contiguous bytes of global memory
-      ok = warp_wait<kSuspendNs>(&bar->o_full[t], ocnt & 1, &bar->abort_flag, p.status);
+      ok = warp_wait<kSuspendNs>(&bar->pv_done[t], (g - 1) & 1, &bar->abort_flag, p.status);   // the item's last P V
       if (!ok) break;
-      ++ocnt;
       tc_fence_after();
       const float inv = 1.f / l;
       const int tok = (qt0 + t) * kTile + 32 * q4 + lane;       // this thread's token
