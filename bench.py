@@ -529,6 +529,10 @@ def run_cuda(args):
     by8 = alg_bytes(8, 8, w.N, 128)
     per["F@d128_64x64"] = {"ms": t_ms, "tokens_per_s": 8 * w.N / (t_ms * 1e-3), "GBps": by8 / t_ms / 1e6, "TFLOPs": fl8 / t_ms / 1e9,
                            "frac_hbm": by8 / t_ms / 1e6 / hbm, "frac_tensor": fl8 / t_ms / 1e9 / tf, "bound": "tensor"}
+    t_ms = time_calls(lambda i: jv.window_attn(*dq8[r(i)], w.Hg, w.Wg, WIN, WIN, out=do8[r(i)]), K, W, stream)
+    fw8 = alg_flops_attn(8, 8, w.Hg, w.Wg, 128, WIN, WIN)
+    per["W@d128_64x64"] = {"ms": t_ms, "tokens_per_s": 8 * w.N / (t_ms * 1e-3), "GBps": by8 / t_ms / 1e6, "TFLOPs": fw8 / t_ms / 1e9,
+                           "frac_hbm": by8 / t_ms / 1e6 / hbm, "frac_tensor": fw8 / t_ms / 1e9 / tf, "bound": "hbm"}
     del dq8, do8
 
     # ragged DepthAnythingV2-L grid (73x73, B=4): F and W with masked edge windows

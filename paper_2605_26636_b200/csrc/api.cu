@@ -140,10 +140,10 @@ jv_status run_attn(const void* q, const void* k, const void* v, void* o, const j
     if (!status) return JV_ERR_CUDA;
     return from_cuda(launch_attn_f4(a, status, st));
   }
-  if (!g_force_generic.load() && one_window && attn_d128_supported(a)) {
+  if (!g_force_generic.load() && attn_d128_supported(a, full)) {
     int* status = device_status_ptr();
     if (!status) return JV_ERR_CUDA;
-    return from_cuda(launch_attn_d128(a, status, st));
+    return from_cuda(launch_attn_d128(a, full, status, st));
   }
   if (!g_force_generic.load() && !one_window && attn_w4_supported(a)) {
     int* status = device_status_ptr();

@@ -1,5 +1,5 @@
-// Full softmax attention (Eq. 1) at head_dim 128 on the 5th-generation tensor cores: two 128-row
-// query tiles per CTA.  bf16 tensors.
+// Full softmax attention (Eq. 1) and 2-D window attention (Sec. 3.2.3) at head_dim 128 on the
+// 5th-generation tensor cores: two 128-row query tiles per CTA.  bf16 tensors, no prefix tokens in W.
 //
 // The four-tile kernel of head_dim 64 (attn_f4.cu) does not carry over: a 128-column fp32 accumulator
 // per query tile leaves tensor memory (512 columns) room for two tiles: per tile two 64-column score
@@ -12,8 +12,12 @@
 // channels (16 KB each, one TMA box each): Q K^T runs over both halves (8 MMAs of K = 16), P V
 // writes the two 64-column halves of the accumulator from the two halves of V (2 x 4 MMAs).
 //
+// The token grid is a 5-D TMA tensor (d, x, y, head, batch); a tile is a box of 128 tokens (F: 128
+// consecutive tokens of the sequence seen as an N x 1 grid; W: ww x 128 / ww tokens of a window).
 // Persistent CTAs (one per SM) loop over work items; an item is two consecutive query tiles of one
-// (batch, head) against all key tiles.  Warp roles (10 warps):
+// window of one (batch, head) against all key tiles of that window.  Keys outside the grid or the
+// window arrive as zeros or as a neighbour's tokens and are overwritten with -inf in tensor memory
+// before the softmax; query rows outside are not written.  Warp roles (10 warps):
 //   warp 0        TMA producer: two Q tiles per item, K tiles through a ring of three, V tiles through a ring of two
 //   warp 1        MMA issuer, in steps of 64 keys, both tiles: O_t += P_t V of step u, then S_t = Q_t K^T of step u + 2
 //                 into the score buffer that P V has just read
@@ -57,14 +61,41 @@ struct D128Params {
   __nv_bfloat16* o;      // [B*H, N, 128]
   int* status;
   int N;                 // tokens per (batch, head)
-  int ntiles;            // key (and query) tiles per head: ceil(N / 128)
-  int qgroups;           // pairs of query tiles per head
-  int total_items;       // (batch*head, pair), pair fastest
-  FastDiv div_qgroups;
+  int gridW, gridH;      // token grid as TMA sees it (F: N x 1)
+  int win_w, win_h;      // window extent in (x, y) (F: N x 1)
+  int box_w, box_h;      // tile box: box_w * box_h == 128
+  int lg_box_w;
+  int step_x, step_y;    // origin step from one tile of a window to the next
+  int nwx, nwin;         // windows per grid row, per (batch, head)
+  int qpairs;            // pairs of query tiles per window (by the full window extent)
+  int total_items;       // (batch*head, window, pair), pair fastest
+  FastDiv div_qpairs, div_nwin, div_nwx;
   int H;                 // heads per batch element: the inputs are addressed by (head, batch)
   FastDiv div_H;
   float scale_log2;      // softmax scale * log2(e)
 };
+
+// One work item: two query tiles of one window of one (batch, head).  F is one window per head: the
+// token sequence as an N x 1 grid with boxes of 128 x 1 tokens.
+struct Item {
+  int bh, x0, y0, x_end, y_end;   // window origin and valid end (exclusive) in the token grid
+  int ntiles;                     // tiles of the window: query tiles, and key tiles
+  int qt0;                        // first of the item's two query tiles (an item with qt0 >= ntiles is empty)
+};
+__device__ __forceinline__ Item decode_item(const D128Params& p, int i) {
+  Item it;
+  const int r = fdiv(i, p.div_qpairs), qp = i - r * p.qpairs;
+  it.bh = fdiv(r, p.div_nwin);
+  const int win = r - it.bh * p.nwin;
+  const int wy = fdiv(win, p.div_nwx), wx = win - wy * p.nwx;
+  it.x0 = wx * p.win_w;
+  it.y0 = wy * p.win_h;
+  it.x_end = min(it.x0 + p.win_w, p.gridW);
+  it.y_end = min(it.y0 + p.win_h, p.gridH);
+  it.ntiles = p.step_x ? (it.x_end - it.x0 + kTile - 1) / kTile : (it.y_end - it.y0 + p.box_h - 1) / p.box_h;
+  it.qt0 = kQT * qp;
+  return it;
+}
 
 struct __align__(8) Barriers {
   uint64_t q_full[kQT], q_empty[kQT];
@@ -138,15 +169,14 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
   const uint32_t tmem = __shfl_sync(0xffffffffu, bar->tmem_base, 0);
 
   const int item0 = blockIdx.x, item_step = gridDim.x;
-  const int ntiles = p.ntiles, nsteps = 2 * p.ntiles;
 
   if (warp == 0) {
     // ================= TMA producer =================
     // a tile = two boxes of 64 channels x 128 tokens, one per swizzled half
-    auto load_tile = [&](uint32_t dst, const CUtensorMap* map, uint64_t* full, int tok, int h, int b) {
+    auto load_tile = [&](uint32_t dst, const CUtensorMap* map, uint64_t* full, int x, int y, int h, int b) {
       mbar_expect_tx(full, kTileBytes);
-      tma_load_4d(dst, map, full, 0, tok, h, b);
-      tma_load_4d(dst + kHalfBytes, map, full, kHalfD, tok, h, b);
+      tma_load_5d(dst, map, full, 0, x, y, h, b);
+      tma_load_5d(dst + kHalfBytes, map, full, kHalfD, x, y, h, b);
     };
     bool ok = true;
     int n = 0;                 // items seen
@@ -154,23 +184,26 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     uint32_t kpar = 1, vpar = 1;   // parity of the "empty" phase this pass over each ring waits for
     int issued_v = 0;          // for the abort path: V copies issued so far
     for (int i = item0; i < p.total_items && ok; i += item_step) {
-      const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
-      const int b = fdiv(bh, p.div_H), h = bh - b * p.H;   // coordinates of the input tensor maps
+      const Item it = decode_item(p, i);
+      if (it.qt0 >= it.ntiles) continue;
+      const int ntiles = it.ntiles, qt0 = it.qt0;
+      const int b = fdiv(it.bh, p.div_H), h = it.bh - b * p.H;   // coordinates of the input tensor maps
       for (int t = 0; t < kQT && ok; ++t) {
         ok = warp_wait<kSuspendNs>(&bar->q_empty[t], (n & 1) ^ 1, &bar->abort_flag, p.status);
         if (!ok) break;
-        if (qt0 + t < ntiles && elect_one()) load_tile(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], (qt0 + t) * kTile, h, b);
+        if (qt0 + t < ntiles && elect_one())
+          load_tile(sQ + t * kTileBytes, &mapQ, &bar->q_full[t], it.x0 + (qt0 + t) * p.step_x, it.y0 + (qt0 + t) * p.step_y, h, b);
         __syncwarp();
       }
       for (int j = 0; j < ntiles && ok; ++j) {
         ok = warp_wait<kSuspendNs>(&bar->k_empty[ks], kpar, &bar->abort_flag, p.status);
         if (!ok) break;
-        if (elect_one()) load_tile(sK + ks * kTileBytes, &mapK, &bar->k_full[ks], j * kTile, h, b);
+        if (elect_one()) load_tile(sK + ks * kTileBytes, &mapK, &bar->k_full[ks], it.x0 + j * p.step_x, it.y0 + j * p.step_y, h, b);
         __syncwarp();
         if (++ks == kKS) { ks = 0; kpar ^= 1; }
         ok = warp_wait<kSuspendNs>(&bar->v_empty[vs], vpar, &bar->abort_flag, p.status);
         if (!ok) break;
-        if (elect_one()) load_tile(sV + vs * kTileBytes, &mapV, &bar->v_full[vs], j * kTile, h, b);
+        if (elect_one()) load_tile(sV + vs * kTileBytes, &mapV, &bar->v_full[vs], it.x0 + j * p.step_x, it.y0 + j * p.step_y, h, b);
         __syncwarp();
         ++issued_v;
         if (++vs == kVS) { vs = 0; vpar ^= 1; }
@@ -198,8 +231,10 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     uint32_t pcnt[2][2] = {{0, 0}, {0, 0}}; // publications seen so far per tile and buffer: parity of p_full
     uint32_t qcnt[2] = {0, 0};              // items in which the tile existed: parity of q_full
     for (int i = item0; i < p.total_items && ok; i += item_step) {
-      const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
-      const bool ex[2] = {true, qt0 + 1 < ntiles};
+      const Item it = decode_item(p, i);
+      if (it.qt0 >= it.ntiles) continue;
+      const int nsteps = 2 * it.ntiles;
+      const bool ex[2] = {true, it.qt0 + 1 < it.ntiles};
       // Scores of step u: scores_begin waits for the key tile, scores_tile issues tile x's MMAs into buffer
       // u % 2 (the caller has made sure that the buffer is free: its previous P V has been issued, and one
       // thread's MMAs execute in issue order), scores_end hands the key tile and the query tiles back.
@@ -303,14 +338,15 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
     const float sl2 = p.scale_log2;
     const float kLazy = 8.f / sl2;                 // the reference maximum moves only when it grew by > 2^8
     const uint64_t sl2x2 = pack2(sl2, sl2);
-    const int last_valid = p.N - (ntiles - 1) * kTile;         // keys that exist in the last key tile
     bool ok = true;
     uint32_t scnt[2] = {0, 0};        // steps seen by this tile per score buffer: parity of s_full
     uint32_t g = 0;                   // steps seen by this tile in all: phase of pv_done
 
     for (int i = item0; i < p.total_items && ok; i += item_step) {
-      const int bh = fdiv(i, p.div_qgroups), qt0 = kQT * (i - bh * p.qgroups);
-      if (qt0 + t >= ntiles) continue;              // this query tile does not exist
+      const Item it = decode_item(p, i);
+      if (it.qt0 >= it.ntiles) continue;            // an empty item (a short edge window)
+      if (it.qt0 + t >= it.ntiles) continue;        // this query tile does not exist
+      const int nsteps = 2 * it.ntiles;
       float m = -INFINITY, l = 0.f;
       for (int u = 0; u < nsteps; ++u) {
         const uint32_t tS = tS0 + (u & 1) * kSub;
@@ -319,18 +355,31 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
         ++scnt[u & 1];
         tc_fence_after();
         uint32_t va[32], vb2[32];
-        if ((u >> 1) == ntiles - 1 && last_valid < kTile) {
-          // Last key tile of a sequence that is not a multiple of 128: overwrite the scores of keys
-          // that do not exist with -inf in tensor memory, then treat the step like any other.
+        // valid extent of this key tile's box along x and y: a key outside the grid or the window does not exist
+        const int vx = it.x_end - (it.x0 + (u >> 1) * p.step_x), vy = it.y_end - (it.y0 + (u >> 1) * p.step_y);
+        if (vx < p.box_w || vy < p.box_h) {
+          // Edge tile: overwrite the scores of keys that do not exist with -inf in tensor memory, then
+          // treat the step like any other.
 #pragma unroll 1
           for (int c = 0; c < 2; ++c) {
-            const int nv = last_valid - (64 * (u & 1) + 32 * c);      // valid keys among these 32
-            if (nv < 32) {                                             // warp-uniform
+            const int k0 = 64 * (u & 1) + 32 * c;      // first of the 32 keys, as an index into the box
+            uint32_t bits = 0;
+            if (p.box_w >= 32) {                       // the 32 keys lie in one box row
+              const int ly = k0 >> p.lg_box_w, lx0 = k0 & (p.box_w - 1);
+              const int nv = min(32, vx - lx0);
+              if (ly < vy && nv > 0) bits = nv >= 32 ? 0xffffffffu : ((1u << nv) - 1u);
+            } else {                                   // 32 / box_w whole box rows
+              const uint32_t rowbits = (1u << min(vx, p.box_w)) - 1u;
+              const int ly0 = k0 >> p.lg_box_w;
+              for (int rr = 0; rr < (32 >> p.lg_box_w); ++rr)
+                if (ly0 + rr < vy) bits |= rowbits << (rr << p.lg_box_w);
+            }
+            if (bits != 0xffffffffu) {                 // warp-uniform: the mask depends on the tile only
               tmem_ld32(tS + 32 * c, va);
               tmem_wait_ld(va);
 #pragma unroll
               for (int x = 0; x < 32; ++x)
-                if (x >= nv) va[x] = kNegInf;     // exp2(-inf) = 0 and -inf never wins the maximum
+                if (!((bits >> x) & 1u)) va[x] = kNegInf;   // exp2(-inf) = 0 and -inf never wins the maximum
               tmem_st32(tS + 32 * c, va);
             }
           }
@@ -401,14 +450,17 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
-      const int tok = (qt0 + t) * kTile + 32 * q4 + lane;       // this thread's token
-      __nv_bfloat16* dst = p.o + ((size_t)bh * p.N + (size_t)tok) * kD;
+      // this thread's token: row r of the tile's box
+      const int r = 32 * q4 + lane;
+      const int qx = it.x0 + (it.qt0 + t) * p.step_x + (r & (p.box_w - 1)), qy = it.y0 + (it.qt0 + t) * p.step_y + (r >> p.lg_box_w);
+      const bool row_ok = qx < it.x_end && qy < it.y_end;
+      __nv_bfloat16* dst = p.o + ((size_t)it.bh * p.N + (size_t)qy * p.gridW + qx) * kD;
 #pragma unroll 1
       for (int c = 0; c < kD / 32; ++c) {
         uint32_t v[32];
         tmem_ld32(tO + 32 * c, v);
         tmem_wait_ld(v);
-        if (tok < p.N) {
+        if (row_ok) {
 #pragma unroll
           for (int x = 0; x < 4; ++x)
             *reinterpret_cast<uint4*>(dst + 32 * c + 8 * x) =
@@ -433,28 +485,52 @@ attn_d128_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant
 
 }  // namespace
 
-bool attn_d128_supported(const AttnArgs& a) {
-  if (a.dtype != JV_BF16 || a.D != kD) return false;
-  const int64_t N = (int64_t)a.Hg * a.Wg;
-  if (N < kTile) return false;                              // shorter sequences: the generic kernel
-  const int64_t ntiles = (N + kTile - 1) / kTile;
-  if ((ntiles + kQT - 1) / kQT * a.BH > 0x7fffffffll) return false;
+// F (full = true or one window covering the grid): any N >= 128.  W: windows whose width ww is a power of
+// two <= 128 (a tile is a box of ww x 128 / ww tokens), no prefix tokens.
+namespace {
+struct Geometry {
+  int gridW, gridH, win_w, win_h, box_w, box_h, step_x, step_y, nwx, nwy, tiles_per_window;
+};
+bool geometry(const AttnArgs& a, bool full, Geometry* g) {
+  const int N = a.Hg * a.Wg;
+  if (full || (a.wh >= a.Hg && a.ww >= a.Wg)) {
+    *g = Geometry{N, 1, N, 1, kTile, 1, kTile, 0, 1, 1, ceil_div(N, kTile)};
+    return true;
+  }
+  const int ww = a.ww;
+  if (ww < 1 || ww > kTile || (ww & (ww - 1)) != 0) return false;   // box width must divide 128
+  const int bh = kTile / ww;
+  const int wh = a.wh < a.Hg ? a.wh : a.Hg;
+  *g = Geometry{a.Wg, a.Hg, ww, wh, ww, bh, 0, bh, ceil_div(a.Wg, ww), ceil_div(a.Hg, wh), ceil_div(wh, bh)};
+  return true;
+}
+}  // namespace
+
+bool attn_d128_supported(const AttnArgs& a, bool full) {
+  if (a.dtype != JV_BF16 || a.D != kD || a.P != 0) return false;
+  Geometry g;
+  if (!geometry(a, full, &g)) return false;
+  if ((int64_t)a.Hg * a.Wg < kTile) return false;           // tiny problems: the generic kernel
+  if ((int64_t)g.nwx * g.nwy * ceil_div(g.tiles_per_window, kQT) * a.BH > 0x7fffffffll) return false;
   return encode_fn() != nullptr;
 }
 
-cudaError_t launch_attn_d128(const AttnArgs& a, int* status, cudaStream_t st) {
+cudaError_t launch_attn_d128(const AttnArgs& a, bool full, int* status, cudaStream_t st) {
+  Geometry g;
+  if (!geometry(a, full, &g)) return cudaErrorInvalidValue;
   EncodeFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
   const int N = a.Hg * a.Wg;
   CUtensorMap maps[3];
   const void* ptrs[3] = {a.q, a.k, a.v};
-  // the inputs as (d, token, head, batch) with the caller's strides; a box is one 64-channel half of a tile
-  const cuuint64_t idims[4] = {(cuuint64_t)kD, (cuuint64_t)N, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
-  const cuuint64_t istrides[3] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)a.in.head * 2, (cuuint64_t)a.in.batch * 2};
-  const cuuint32_t ibox[4] = {(cuuint32_t)kHalfD, (cuuint32_t)kTile, 1, 1};
-  const cuuint32_t iestr[4] = {1, 1, 1, 1};
+  // the inputs as (d, x, y, head, batch) with the caller's strides; a box is one 64-channel half of a tile
+  const cuuint64_t idims[5] = {(cuuint64_t)kD, (cuuint64_t)g.gridW, (cuuint64_t)g.gridH, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
+  const cuuint64_t istrides[4] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)g.gridW * a.in.tok * 2, (cuuint64_t)a.in.head * 2,
+                                  (cuuint64_t)a.in.batch * 2};
+  const cuuint32_t ibox[5] = {(cuuint32_t)kHalfD, (cuuint32_t)g.box_w, (cuuint32_t)g.box_h, 1, 1};
+  const cuuint32_t iestr[5] = {1, 1, 1, 1, 1};
   for (int i = 0; i < 3; ++i) {
-    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptrs[i]), idims, istrides, ibox, iestr,
+    CUresult r = enc(&maps[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptrs[i]), idims, istrides, ibox, iestr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -468,10 +544,23 @@ cudaError_t launch_attn_d128(const AttnArgs& a, int* status, cudaStream_t st) {
   p.o = (__nv_bfloat16*)a.o;
   p.status = status;
   p.N = N;
-  p.ntiles = ceil_div(N, kTile);
-  p.qgroups = ceil_div(p.ntiles, kQT);
-  p.total_items = p.qgroups * a.BH;
-  p.div_qgroups = make_fastdiv((uint32_t)p.qgroups);
+  p.gridW = g.gridW;
+  p.gridH = g.gridH;
+  p.win_w = g.win_w;
+  p.win_h = g.win_h;
+  p.box_w = g.box_w;
+  p.box_h = g.box_h;
+  p.lg_box_w = 0;
+  while ((1 << p.lg_box_w) < g.box_w) ++p.lg_box_w;
+  p.step_x = g.step_x;
+  p.step_y = g.step_y;
+  p.nwx = g.nwx;
+  p.nwin = g.nwx * g.nwy;
+  p.qpairs = ceil_div(g.tiles_per_window, kQT);
+  p.total_items = p.qpairs * p.nwin * a.BH;
+  p.div_qpairs = make_fastdiv((uint32_t)p.qpairs);
+  p.div_nwin = make_fastdiv((uint32_t)p.nwin);
+  p.div_nwx = make_fastdiv((uint32_t)p.nwx);
   p.H = a.H;
   p.div_H = make_fastdiv((uint32_t)a.H);
   p.scale_log2 = a.scale * 1.4426950408889634f;

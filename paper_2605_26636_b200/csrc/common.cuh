@@ -119,9 +119,10 @@ cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream
 // tcgen05 path for windows of one or two 128-token tiles (bf16, D == 64, no prefix): two windows per CTA
 bool attn_w4_supported(const AttnArgs& a);
 cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st);
-// tcgen05 path for full attention at head_dim 128 (bf16, N >= 128): two query tiles per CTA
-bool attn_d128_supported(const AttnArgs& a);
-cudaError_t launch_attn_d128(const AttnArgs& a, int* status, cudaStream_t st);
+// tcgen05 path at head_dim 128 (bf16, N >= 128, no prefix tokens in W): two query tiles per CTA.
+// full = true: F over all N tokens; else W with windows whose width is a power of two <= 128
+bool attn_d128_supported(const AttnArgs& a, bool full);
+cudaError_t launch_attn_d128(const AttnArgs& a, bool full, int* status, cudaStream_t st);
 // tcgen05 path for full attention over long sequences (bf16, D == 64, N >= 1024): four query tiles per CTA
 bool attn_f4_supported(const AttnArgs& a);
 cudaError_t launch_attn_f4(const AttnArgs& a, int* status, cudaStream_t st);
