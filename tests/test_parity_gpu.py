@@ -153,7 +153,8 @@ def test_linear_dwc_with_poisoned_scratch_and_output(jv, oracle, case):
                          ids=["vitb_64x128", "giant_32x64", "d128_24x40"])
 def test_other_model_shapes(jv, oracle, case):
     """Non-square grids (a 1024x2048 image at patch 16 is 64x128 tokens) with 12 and 24 heads on the
-    tensor-core kernels, and head_dim 128 on the shape-generic kernels; sampled (batch, head) pairs."""
+    tensor-core kernels, and head_dim 128 (F and W on their own tensor-core kernel, L on the shape-generic
+    kernels); sampled (batch, head) pairs."""
     B, H, Hg, Wg, D = case
     q, k, v = inputs.custom_qkv(B, H, Hg * Wg, D, "bf16", seed=H + D)
     dq, dk, dv = _dev((q, k, v))
