@@ -1,4 +1,4 @@
-// Full softmax attention (Eq. 1) and 2-D window attention (Sec. 3.2.3) at head_dim 128 on the
+// Full softmax attention (Eq. 1) and 2-D window attention (Sec. 3.2.2) at head_dim 128 on the
 // 5th-generation tensor cores: two 128-row query tiles per CTA.  bf16 tensors, no prefix tokens in W.
 //
 // The four-tile kernel of head_dim 64 (attn_f4.cu) does not carry over: a 128-column fp32 accumulator

@@ -1,4 +1,4 @@
-// 2-D window attention (Sec. 3.2.3) for windows of one or two 128-token tiles (16 x 16 and the
+// 2-D window attention (Sec. 3.2.2) for windows of one or two 128-token tiles (16 x 16 and the
 // like) on the 5th-generation tensor cores: two windows side by side per CTA, four 128-row query
 // tiles, so that every SM sub-core holds four softmax warps.  bf16 tensors, head_dim 64, no prefix tokens.
 //

@@ -148,6 +148,41 @@ def test_linear_dwc_with_poisoned_scratch_and_output(jv, oracle, case):
         assert rel_err(out, ref) <= TOL["bf16"], rep
 
 
+# ------------------------------------------------------------------ window kernel: every box shape
+WBOX = [  # B, H, Hg, Wg, win_h, win_w: windows of one or two 128-token boxes (box = win_w x 128 / win_w rows)
+    (2, 2, 48, 80, 16, 16),      # two boxes of 16 x 8, whole windows only
+    (1, 3, 41, 70, 16, 16),      # ragged: a bottom row of windows with one box (9 rows), a right column 6 wide
+    (1, 2, 37, 50, 8, 16),       # one box per window; bottom windows of 5 rows, right windows 2 wide
+    (1, 2, 20, 70, 8, 32),       # two boxes of 32 x 4; bottom windows of one box, right windows 6 wide
+    (2, 1, 22, 100, 4, 32),      # one box of 32 x 4; bottom windows of 2 rows
+    (1, 2, 70, 20, 32, 8),       # two boxes of 8 x 16; bottom windows of 6 rows (one box), right windows 4 wide
+    (1, 1, 50, 12, 16, 8),       # one box of 8 x 16
+    (1, 2, 100, 9, 64, 4),       # two boxes of 4 x 32; right windows 1 wide
+    (5, 7, 16, 16, 16, 16),      # 35 windows: fewer than one CTA pair per SM, an odd count (a slot without work)
+]
+
+
+@pytest.mark.parametrize("case", WBOX, ids=lambda c: "x".join(map(str, c)))
+def test_window_kernel_box_shapes(jv, oracle, case):
+    """The two-windows-per-CTA kernel over every tile box it accepts, with ragged grids in both directions
+    (edge windows with one box instead of two, clipped stores, masked keys); one launch per call."""
+    B, H, Hg, Wg, wh, ww = case
+    q, k, v = inputs.custom_qkv(B, H, Hg * Wg, 64, "bf16", seed=7000 + Hg + 3 * Wg + wh)
+    out, check = guarded_empty(q.shape, torch.bfloat16, DEV)
+    out.fill_(float("nan"))
+    launches = jv.launch_count()
+    jv.window_attn(*_dev((q, k, v)), Hg, Wg, wh, ww, out=out)
+    assert jv.launch_count() == launches + 1
+    check()
+    if B * H > 8:
+        out = out.cpu()
+        for b, h in sample_heads(B, H, 6, 9):
+            sl = (slice(b, b + 1), slice(h, h + 1))
+            assert rel_err(out[sl], oracle.window_attn(q[sl], k[sl], v[sl], Hg, Wg, wh, ww)) <= TOL["bf16"], (case, b, h)
+    else:
+        assert rel_err(out, oracle.window_attn(q, k, v, Hg, Wg, wh, ww)) <= TOL["bf16"], case
+
+
 # ------------------------------------------------------------------ other model sizes and grids
 @pytest.mark.parametrize("case", [(1, 12, 64, 128, 64), (1, 24, 32, 64, 64), (1, 4, 24, 40, 128)],
                          ids=["vitb_64x128", "giant_32x64", "d128_24x40"])
