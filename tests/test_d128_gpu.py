@@ -83,6 +83,7 @@ WCASES = [  # B, H, Hg, Wg, win_h, win_w
     (1, 1, 24, 64, 24, 16),      # three tiles per window: the second item of a window holds one
     (1, 2, 12, 96, 4, 32),       # box of 32 x 4 tokens
     (1, 1, 9, 200, 5, 128),      # box of 128 x 1 tokens, five tiles per window, ragged in both directions
+    (1, 2, 40, 9, 16, 16),       # a grid narrower than the window's box
 ]
 
 

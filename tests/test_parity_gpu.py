@@ -159,6 +159,8 @@ WBOX = [  # B, H, Hg, Wg, win_h, win_w: windows of one or two 128-token boxes (b
     (1, 1, 50, 12, 16, 8),       # one box of 8 x 16
     (1, 2, 100, 9, 64, 4),       # two boxes of 4 x 32; right windows 1 wide
     (5, 7, 16, 16, 16, 16),      # 35 windows: fewer than one CTA pair per SM, an odd count (a slot without work)
+    (1, 2, 40, 9, 16, 16),       # a grid narrower than the window's box
+    (2, 1, 5, 70, 8, 16),        # a grid lower than the window's box
 ]
 
 
