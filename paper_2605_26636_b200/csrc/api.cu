@@ -148,7 +148,9 @@ jv_status run_attn(const void* q, const void* k, const void* v, void* o, const j
   if (!g_force_generic.load() && !one_window && attn_w4_supported(a)) {
     int* status = device_status_ptr();
     if (!status) return JV_ERR_CUDA;
-    return from_cuda(launch_attn_w4(a, status, st));
+    const jv_status r = from_cuda(launch_attn_w4(a, status, st));
+    if (r != JV_OK || a.P == 0) return r;
+    return from_cuda(launch_attn_generic(a, st, true));   // the P prefix queries, which attend everything
   }
   if (!g_force_generic.load() && attn_tc_supported(a, full)) {
     int* status = device_status_ptr();

@@ -43,7 +43,11 @@ constexpr int kTile = 128;                  // tokens per tile (MMA M and key-ti
 constexpr int kTileBytes = kTile * kD * 2;  // 16 KB
 constexpr int kSlots = 2;                   // windows in flight per CTA
 constexpr int kQT = 2 * kSlots;             // query tiles per CTA
-constexpr int kKS = 2, kVS = 3;             // K and V ring depths per slot
+constexpr int kKS = 2;                      // K ring depth per slot
+constexpr int kVSMax = 3;                   // V ring depth per slot: 3 without prefix tokens (a stage doubles as the
+                                            // output's staging tile), 2 with them (rows go straight to global memory)
+constexpr int kPreRows = 16;                // prefix keys are one 16-key MMA: P <= 16
+constexpr int kPreBytes = kPreRows * kD * 2;   // 2 KB: the prefix rows of K, or of V
 constexpr int kWarps = 20;
 constexpr int kThreads = kWarps * 32;
 constexpr int kFirstSoftmaxWarp = 4;
@@ -54,6 +58,9 @@ constexpr int kPolyOf8 = 2;                 // of every 8 score pairs, this many
 constexpr uint32_t kColS = 0, kColO = 256;
 
 struct W4Params {
+  __nv_bfloat16* o;      // first grid token of (batch, head) 0 (the prefix variant writes rows itself)
+  int tokens_per_head;   // P + Hg * Wg
+  int P;                 // prefix keys behind every window's own keys (0: none)
   int* status;
   int gridW, gridH;      // token grid
   int win_w, win_h;      // window extent
@@ -87,17 +94,25 @@ __device__ __forceinline__ Item decode_item(const W4Params& p, int r) {
 
 struct __align__(8) Barriers {
   uint64_t q_full[kQT], q_empty[kQT];
-  uint64_t k_full[kSlots][kKS], k_empty[kSlots][kKS], v_full[kSlots][kVS], v_empty[kSlots][kVS];
+  uint64_t k_full[kSlots][kKS], k_empty[kSlots][kKS], v_full[kSlots][kVSMax], v_empty[kSlots][kVSMax];
+  uint64_t pre_full[kSlots], pre_empty[kSlots];       // the slot's prefix rows of K and V
   uint64_t s_full[kQT], p_full[kQT], o_full[kQT];
   uint64_t drain;
   uint32_t tmem_base;
   volatile uint32_t abort_flag;
 };
-constexpr size_t kSmemTiles = (kQT + kSlots * (kKS + kVS)) * (size_t)kTileBytes;   // Q[4] K[2][2] V[2][3]
-constexpr size_t kSmemBytes = kSmemTiles + sizeof(Barriers) + 1024;                 // + alignment slack
+// shared memory: Q[4] | K[2][2] | V[2][kVS] | (prefix variant: per slot the prefix rows of K, then of V) | barriers
+template <bool kPrefix>
+struct Layout {
+  static constexpr int kVS = kPrefix ? 2 : 3;
+  static constexpr size_t kTiles = (kQT + kSlots * (kKS + kVS)) * (size_t)kTileBytes;
+  static constexpr size_t kPre = kPrefix ? (size_t)kSlots * 2 * kPreBytes : 0;
+  static constexpr size_t kBytes = kTiles + kPre + sizeof(Barriers) + 1024;          // + alignment slack
+};
 
 constexpr uint32_t kIdescQK = idesc(kTile, kSub, 0);
 constexpr uint32_t kIdescPV = idesc(kTile, kD, 1);
+constexpr uint32_t kIdescQKpre = idesc(kTile, kPreRows, 0);   // scores against the 16 prefix rows
 
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
   asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
@@ -109,15 +124,26 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 // sequence on its own; ring stages and barrier parities follow running counters.  The second query
 // tile of a window that has one tile only (a bottom edge window) is skipped by its softmax warps;
 // the issuer still frees its Q buffer so that arrival counts hold.
+// kPrefix: every window's queries also attend the P <= 16 prefix tokens of their (batch, head): one more
+// step per window with a 16-key score MMA against the prefix rows of K (kept in shared memory per slot,
+// reloaded per window from L2) and a 16-key P V.  The prefix QUERIES are not this kernel's work.
+template <bool kPrefix>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                const __grid_constant__ CUtensorMap mapV, const __grid_constant__ CUtensorMap mapO,
-               const W4Params p) {
+               const __grid_constant__ CUtensorMap mapKp, const __grid_constant__ CUtensorMap mapVp, const W4Params p) {
+  constexpr int kVS = Layout<kPrefix>::kVS;
+  constexpr size_t kSmemTiles = Layout<kPrefix>::kTiles;
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment by an offset from the array itself, so that accesses stay shared-space loads and stores
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles);
+  Barriers* bar = reinterpret_cast<Barriers*>(smem + kSmemTiles + Layout<kPrefix>::kPre);
   const uint32_t sQ = smem_u32(smem), sK = sQ + kQT * kTileBytes, sV = sK + kSlots * kKS * kTileBytes;
+  const uint32_t sPre = sQ + (uint32_t)kSmemTiles;   // slot s: prefix rows of K at s * 4 KB, of V 2 KB behind them
+
+  // a grid launched behind this one with programmatic serialisation (the prefix queries of W, which
+  // depend on nothing here) may run beside it
+  if (kPrefix) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
 
@@ -142,8 +168,11 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       for (int g = 0; g < kVS; ++g) {
         mbar_init(&bar->v_full[s][g], 1);
-        mbar_init(&bar->v_empty[s][g], 4);   // the four softmax warps that staged their output into it
+        // handed back by the four softmax warps that staged their output into it, or (prefix variant) by the issuer
+        mbar_init(&bar->v_empty[s][g], kPrefix ? 1 : 4);
       }
+      mbar_init(&bar->pre_full[s], 1);
+      mbar_init(&bar->pre_empty[s], 1);
     }
     mbar_init(&bar->drain, kSlots);
     bar->abort_flag = 0;
@@ -203,6 +232,16 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         ++issued_v;
         if (++vs == kVS) { vs = 0; vpar ^= 1; }
       }
+      if (kPrefix && ok) {            // the prefix rows of K and V of this (batch, head): rows past P arrive as zeros
+        ok = warp_wait<kSuspendNs>(&bar->pre_empty[s], (n & 1) ^ 1, &bar->abort_flag, p.status);
+        if (!ok) break;
+        if (elect_one()) {
+          mbar_expect_tx(&bar->pre_full[s], 2 * kPreBytes);
+          tma_load_4d(sPre + s * 2 * kPreBytes, &mapKp, &bar->pre_full[s], 0, 0, h, b);
+          tma_load_4d(sPre + s * 2 * kPreBytes + kPreBytes, &mapVp, &bar->pre_full[s], 0, 0, h, b);
+        }
+        __syncwarp();
+      }
       ++n;
     }
     if (!ok && lane == 0) {
@@ -225,11 +264,14 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     uint32_t phk = 0, phv = 0;              // and their "full" parities
     uint32_t pcnt[2] = {0, 0};              // steps published so far per tile: parity of p_full
     uint32_t qcnt[2] = {0, 0};              // windows in which the tile existed: parity of q_full
+    uint32_t pre_cnt = 0;                   // windows seen: parity of pre_full
     for (int r = kSlots * blockIdx.x + s; r < p.total && ok; r += item_step) {
       const Item it = decode_item(p, r);
-      const int nsteps = 2 * it.ntiles;
-      for (int u = 0; u <= nsteps && ok; ++u) {
-        const bool has_qk = u < nsteps, has_pv = u > 0;
+      const int nsteps = 2 * it.ntiles;               // steps against the window's own keys
+      const int ns = nsteps + (kPrefix ? 1 : 0);      // and, behind them, one against the prefix rows
+      for (int u = 0; u <= ns && ok; ++u) {
+        const bool has_qk = u < nsteps, has_pre_qk = kPrefix && u == nsteps;          // scores of step u
+        const bool has_pv = u > 0 && u <= nsteps, has_pre_pv = kPrefix && u == ns;    // P V of step u - 1
         if (has_qk && (u & 1) == 0) {       // first half of a key tile: its K must have landed
           ok = warp_wait<kSuspendNs>(&bar->k_full[s][sk], phk, &bar->abort_flag, p.status);
           if (!ok) break;
@@ -238,8 +280,14 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           ok = warp_wait<kSuspendNs>(&bar->v_full[s][sv], phv, &bar->abort_flag, p.status);
           if (!ok) break;
         }
+        if (has_pre_qk) {                   // the prefix rows of K and V must have landed
+          ok = warp_wait<kSuspendNs>(&bar->pre_full[s], pre_cnt & 1, &bar->abort_flag, p.status);
+          ++pre_cnt;
+          if (!ok) break;
+        }
         const uint32_t kb = sK + (s * kKS + sk) * kTileBytes + (u & 1) * (kSub * kD * 2);
         const uint32_t vb = sV + (s * kVS + sv) * kTileBytes + ((u - 1) & 1) * (kSub * kD * 2);
+        const uint32_t kpb = sPre + s * 2 * kPreBytes, vpb = kpb + kPreBytes;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           if (x >= it.ntiles) continue;
@@ -261,28 +309,40 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                 mma_ts_1(tmem + kColO + t * kD, tmem + kColS + t * kSub + c * 8, desc_advance(dv, c * 2048), kIdescPV,
                          (u > 1 || c > 0) ? 1u : 0u);
             }
+            if (has_pre_pv)                  // 16 prefix keys: one MMA of K = 16
+              mma_ts_1(tmem + kColO + t * kD, tmem + kColS + t * kSub, smem_desc(vpb), kIdescPV, 1u);
             if (has_qk) {
               const uint64_t dq = smem_desc(sQ + t * kTileBytes), dk = smem_desc(kb);
 #pragma unroll
               for (int c = 0; c < kD / 16; ++c)
                 mma_ss_1(tmem + kColS + t * kSub, desc_advance(dq, c * 32), desc_advance(dk, c * 32), kIdescQK, c > 0);
             }
+            if (has_pre_qk) {                // scores against the prefix rows: 16 columns
+              const uint64_t dq = smem_desc(sQ + t * kTileBytes), dk = smem_desc(kpb);
+#pragma unroll
+              for (int c = 0; c < kD / 16; ++c)
+                mma_ss_1(tmem + kColS + t * kSub, desc_advance(dq, c * 32), desc_advance(dk, c * 32), kIdescQKpre, c > 0);
+            }
           }
           __syncwarp();
-          if (has_qk) tc_commit(&bar->s_full[t]);
+          if (u < ns) tc_commit(&bar->s_full[t]);
           else tc_commit(&bar->o_full[t]);
         }
         if (!ok) break;
-        // a V stage is handed back by the softmax warps that stage their output over it, not here
-        if (has_pv && ((u - 1) & 1) == 1 && ++sv == kVS) { sv = 0; phv ^= 1; }
+        if (has_pv && ((u - 1) & 1) == 1) { // both halves of the V tile are in flight or done
+          // without prefix tokens the stage is handed back by the softmax warps that stage their output over it
+          if (kPrefix) tc_commit(&bar->v_empty[s][sv]);
+          if (++sv == kVS) { sv = 0; phv ^= 1; }
+        }
         if (has_qk && (u & 1) == 1) {
           tc_commit(&bar->k_empty[s][sk]);
-          if (u == nsteps - 1) {            // the window's last scores: its query tiles may be replaced
-            tc_commit(&bar->q_empty[tb]);
-            tc_commit(&bar->q_empty[tb + 1]);
-          }
           if (++sk == kKS) { sk = 0; phk ^= 1; }
         }
+        if (u == ns - 1) {                  // the window's last scores: its query tiles may be replaced
+          tc_commit(&bar->q_empty[tb]);
+          tc_commit(&bar->q_empty[tb + 1]);
+        }
+        if (has_pre_pv) tc_commit(&bar->pre_empty[s]);
       }
     }
     // Teardown: every MMA issued so far must have retired before tensor memory is released.
@@ -330,20 +390,32 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       ++n_all;
       if (it.ntiles == 2) ++n_two;
       if (x >= it.ntiles) {           // this query tile does not exist
-        release();
+        if (!kPrefix) release();
         continue;
       }
-      const int nsteps = 2 * it.ntiles;
+      const int nsteps = 2 * it.ntiles;               // steps against the window's own keys
+      const int ns = nsteps + (kPrefix ? 1 : 0);      // and, behind them, one against the prefix rows
       const int vx = it.x_end - it.x0;                   // valid columns of every box of this window
       float m = -INFINITY, l = 0.f;
-      for (int u = 0; u < nsteps; ++u) {
+      for (int u = 0; u < ns; ++u) {
+        const bool pre = kPrefix && u == nsteps;      // the step of the prefix keys: 16 score columns, P of them keys
         ok = warp_wait<kSuspendNs>(&bar->s_full[t], scnt & 1, &bar->abort_flag, p.status);
         if (!ok) break;
         ++scnt;
         tc_fence_after();
         uint32_t va[32];
         const int vy = it.y_end - (it.y0 + (u >> 1) * p.box_h);    // valid rows of this key tile's box
-        if (vx < p.box_w || vy < p.box_h) {
+        if (pre) {
+          // Columns 0 .. P - 1 hold the scores against the prefix keys; up to column 31 everything else
+          // (scores against the zero rows behind them, the previous step's leftovers) becomes -inf.
+          tmem_ld32(tS, va);
+          tmem_wait_ld(va);
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (i >= p.P) va[i] = kNegInf;
+          tmem_st32(tS, va);
+          tmem_wait_st();
+        } else if (vx < p.box_w || vy < p.box_h) {
           // Edge tile: overwrite the scores of keys outside the grid with -inf in tensor memory, then
           // treat the step like any other.
 #pragma unroll 1
@@ -374,9 +446,11 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         // ---- pass 1: the step's maximum (second half first, so that the first half is the one
         // left in registers for pass 2)
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        tmem_ld32(tS + 32, va);
-        tmem_wait_ld(va);
-        max32(va, mx4);
+        if (!pre) {
+          tmem_ld32(tS + 32, va);
+          tmem_wait_ld(va);
+          max32(va, mx4);
+        }
         tmem_ld32(tS, va);
         tmem_wait_ld(va);
         max32(va, mx4);
@@ -411,10 +485,12 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         uint32_t pk[16];
         exp32<false, kPolyOf8>(va, sl2x2, mnegx2, lsum, pk, mx4);
         tmem_st16(tS, pk);
-        tmem_ld32(tS + 32, va);
-        tmem_wait_ld(va);
-        exp32<false, kPolyOf8>(va, sl2x2, mnegx2, lsum, pk, mx4);
-        tmem_st16(tS + 16, pk);
+        if (!pre) {
+          tmem_ld32(tS + 32, va);
+          tmem_wait_ld(va);
+          exp32<false, kPolyOf8>(va, sl2x2, mnegx2, lsum, pk, mx4);
+          tmem_st16(tS + 16, pk);
+        }
         float a0, a1, b0, b1;
         unpack2(add2(lsum[0], lsum[1]), a0, a1);
         unpack2(add2(lsum[2], lsum[3]), b0, b1);
@@ -423,9 +499,37 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bar->p_full[t]);
-        if (u == 0) release();         // the previous window's store has long read its staging quarter
+        if (!kPrefix && u == 0) release();   // the previous window's store has long read its staging quarter
       }
       if (!ok) break;
+      if (kPrefix) {
+        // ---- epilogue with prefix tokens: O / l -> bf16 -> this thread's row, 128 contiguous bytes of global memory
+        ok = warp_wait<kSuspendNs>(&bar->o_full[t], par_own, &bar->abort_flag, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        const float inv = 1.f / l;
+        const int rr = 32 * q4 + lane;                                     // row of the tile's box
+        const int qx = it.x0 + (rr & (p.box_w - 1)), qy = it.y0 + x * p.box_h + (rr >> p.lg_box_w);
+        const bool row_ok = qx < it.x_end && qy < it.y_end;
+        __nv_bfloat16* dst = p.o + ((size_t)it.bh * p.tokens_per_head + (size_t)qy * p.gridW + qx) * kD;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld32(tO + 32 * c, v);
+          tmem_wait_ld(v);
+          if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              *reinterpret_cast<uint4*>(dst + 32 * c + 8 * i) =
+                  make_uint4(pack_bf16(__uint_as_float(v[8 * i]) * inv, __uint_as_float(v[8 * i + 1]) * inv),
+                             pack_bf16(__uint_as_float(v[8 * i + 2]) * inv, __uint_as_float(v[8 * i + 3]) * inv),
+                             pack_bf16(__uint_as_float(v[8 * i + 4]) * inv, __uint_as_float(v[8 * i + 5]) * inv),
+                             pack_bf16(__uint_as_float(v[8 * i + 6]) * inv, __uint_as_float(v[8 * i + 7]) * inv));
+          }
+        }
+        tc_fence_before();
+        continue;
+      }
       // ---- epilogue: O / l -> bf16 -> this warp's quarter of the V tile x of this window -> one TMA store.
       // Both query tiles' last P V read that V tile: both must have retired.
       ok = warp_wait<kSuspendNs>(&bar->o_full[t], par_own, &bar->abort_flag, p.status);
@@ -463,7 +567,7 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       }
       held = stage;
     }
-    if (ok) release();
+    if (!kPrefix && ok) release();
     // the staging tile must outlive the last store's reads; wait for the writes as well
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
@@ -479,9 +583,11 @@ attn_w4_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
 }  // namespace
 
-// Windows of exactly one or two tile boxes (box = window width x 128 / width rows), no prefix tokens.
+// Windows of exactly one or two tile boxes (box = window width x 128 / width rows); at most 16 prefix tokens
+// (contiguous inputs only: the prefix rows are found behind a.k and a.v).
 bool attn_w4_supported(const AttnArgs& a) {
-  if (a.dtype != JV_BF16 || a.D != kD || a.P != 0) return false;
+  if (a.dtype != JV_BF16 || a.D != kD) return false;
+  if (a.P > kPreRows || (a.P > 0 && a.strided)) return false;
   if (a.wh >= a.Hg && a.ww >= a.Wg) return false;         // one window: full attention's kernels
   const int ww = a.ww;
   if (ww < 1 || ww > 32 || (ww & (ww - 1)) != 0) return false;   // a warp's 32 rows are whole box rows
@@ -495,10 +601,12 @@ bool attn_w4_supported(const AttnArgs& a) {
 cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st) {
   EncodeFn enc = encode_fn();
   if (!enc) return cudaErrorNotSupported;
-  const int N = a.Hg * a.Wg;
+  const int N = a.P + a.Hg * a.Wg;                     // tokens per (batch, head): prefix tokens, then the grid
   const int box_w = a.ww, box_h = kTile / a.ww;
-  CUtensorMap maps[4];
-  const void* ptrs[4] = {a.q, a.k, a.v, a.o};
+  CUtensorMap maps[6];
+  // the grid tokens start behind the prefix rows
+  const size_t grid0 = (size_t)a.P * kD * 2, igrid0 = (size_t)a.P * (size_t)a.in.tok * 2;
+  const void* ptrs[4] = {(const char*)a.q + igrid0, (const char*)a.k + igrid0, (const char*)a.v + igrid0, (char*)a.o + grid0};
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)a.Wg, (cuuint64_t)a.Hg, (cuuint64_t)a.BH};
   const cuuint64_t strides[3] = {(cuuint64_t)kD * 2, (cuuint64_t)a.Wg * kD * 2, (cuuint64_t)N * kD * 2};
   // the output is stored per warp: a quarter of the tile's box (32 tokens)
@@ -519,12 +627,34 @@ cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st) {
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
   }
+  // the P prefix rows of K and V as (d, row, head, batch), a box of 16 rows: rows past P arrive as zeros
+  maps[4] = maps[1];
+  maps[5] = maps[2];
+  if (a.P > 0) {
+    const cuuint64_t pdims[4] = {(cuuint64_t)kD, (cuuint64_t)a.P, (cuuint64_t)a.H, (cuuint64_t)(a.BH / a.H)};
+    const cuuint64_t pstrides[3] = {(cuuint64_t)a.in.tok * 2, (cuuint64_t)a.in.head * 2, (cuuint64_t)a.in.batch * 2};
+    const cuuint32_t pbox[4] = {(cuuint32_t)kD, (cuuint32_t)kPreRows, 1, 1};
+    const void* pptrs[2] = {a.k, a.v};
+    for (int i = 0; i < 2; ++i) {
+      CUresult r = enc(&maps[4 + i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pptrs[i]), pdims, pstrides, pbox,
+                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    }
+  }
   static OncePerDevice smem_opt_in;   // > 48 KB of dynamic shared memory: a per-device function attribute
   cudaError_t e = smem_opt_in.run([] {
-    return cudaFuncSetAttribute(attn_w4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    cudaError_t r = cudaFuncSetAttribute(attn_w4_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)Layout<false>::kBytes);
+    if (r == cudaSuccess)
+      r = cudaFuncSetAttribute(attn_w4_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Layout<true>::kBytes);
+    return r;
   });
   if (e != cudaSuccess) return e;
   W4Params p;
+  p.o = (__nv_bfloat16*)a.o + (size_t)a.P * kD;        // first grid token of (batch, head) 0
+  p.tokens_per_head = N;
+  p.P = a.P;
   p.status = status;
   p.gridW = a.Wg;
   p.gridH = a.Hg;
@@ -545,7 +675,11 @@ cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st) {
   const int num_sms = device_sm_count();
   const int want = ceil_div(p.total, kSlots);
   const int grid = want < num_sms ? want : num_sms;
-  attn_w4_kernel<<<grid, kThreads, kSmemBytes, st>>>(maps[0], maps[1], maps[2], maps[3], p);
+  if (a.P > 0) {
+    attn_w4_kernel<true><<<grid, kThreads, Layout<true>::kBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
+  } else {
+    attn_w4_kernel<false><<<grid, kThreads, Layout<false>::kBytes, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], p);
+  }
   count_launch();
   return cudaGetLastError();
 }

@@ -116,7 +116,7 @@ cudaError_t launch_attn_generic(const AttnArgs& a, cudaStream_t st, bool prefix_
 // windows whose width ww is a power of two <= 128 (a tile is a box of ww x 128/ww tokens).
 bool attn_tc_supported(const AttnArgs& a, bool full);
 cudaError_t launch_attn_tc(const AttnArgs& a, bool full, int* status, cudaStream_t st);
-// tcgen05 path for windows of one or two 128-token tiles (bf16, D == 64, no prefix): two windows per CTA
+// tcgen05 path for windows of one or two 128-token tiles (bf16, D == 64, at most 16 prefix tokens): two windows per CTA
 bool attn_w4_supported(const AttnArgs& a);
 cudaError_t launch_attn_w4(const AttnArgs& a, int* status, cudaStream_t st);
 // tcgen05 path at head_dim 128 (bf16, N >= 128, no prefix tokens in W): two query tiles per CTA.
