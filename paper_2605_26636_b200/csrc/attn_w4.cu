@@ -1,6 +1,6 @@
 // 2-D window attention (Sec. 3.2.2) for windows of one or two 128-token tiles (16 x 16 and the
 // like) on the 5th-generation tensor cores: two windows side by side per CTA, four 128-row query
-// tiles, so that every SM sub-core holds four softmax warps.  bf16 tensors, head_dim 64, no prefix tokens.
+// tiles, so that every SM sub-core holds four softmax warps.  bf16 tensors, head_dim 64, at most 16 prefix tokens.
 //
 // The softmax of attention at head_dim 64 is bound by the SM's ordinary pipes and their latencies, and a
 // window is short work (four 64-key steps per query tile): with two query tiles per CTA (attn_tc.cu) a
@@ -23,6 +23,8 @@
 // the V tile x of its own window once both tiles' last P V have retired; the producer may refill that
 // stage when the four warps that staged into it have seen their stores read it (v_empty counts them),
 // which they check one step into their next window, off the critical path.
+// With prefix tokens (template parameter): one more step per window against the prefix rows of K and V,
+// which take the shared memory of the third V stage; the rows then go straight to global memory.
 //
 // Every mbarrier wait is bounded: a wait that runs out sets the device status word, raises a
 // CTA-wide abort flag, and every role falls through to the common teardown (tensor memory is
